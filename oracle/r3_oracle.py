@@ -1,0 +1,278 @@
+"""CPU oracle for the Rollout Routing Replay (R3) MoE layer.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain, float64 statement of what the
+paper's Section 4.1 defines.  Only the test-suite, the smoke check and the benchmark's
+``cpu_baseline`` / reference arm may import it; the product path (the CUDA library and its
+Python binding) never does, and shares no code, table or constant with it.
+
+Everything is numpy float64.  Inputs are the stored values of the tensors handed to the GPU
+path (bf16 values widened exactly), so the only differences between the two sides are the
+GPU's working precision and summation order.
+
+Notation follows the paper: T tokens, hidden size d, M = E experts, K experts per token,
+``s`` router logits, ``I`` the routing mask (kept as K indices per token), ``g`` gate weights,
+``E_i`` the i-th expert network, ``y`` the layer output.  The expert network is a bias-free
+SwiGLU feed-forward of width F (the paper leaves ``E_i`` abstract; the benchmark
+configuration fixes it).
+
+A library matmul / sort is used as a single step where the definition is a matrix product or
+an ordering; there is no tiling, fusion or reordering beyond what the equations state.
+
+Pins (see tests/test_oracle_pins.py): every public function is pinned to something other than
+itself - closed forms, library routines on special cases, finite differences, brute force over
+all M experts on tiny layers, and the stored golden values derived by hand in
+tests/golden/.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=F64))
+
+
+# ----------------------------------------------------------------------------------------------
+# Section 4.1, first equation: router logits  s = x W_r
+# ----------------------------------------------------------------------------------------------
+def router_logits(x, w_r) -> np.ndarray:
+    """s[t, i] = sum_c x[t, c] * W_r[i, c]   (Section 4.1, first equation).
+
+    ``w_r`` is stored [E, d] (output-major), so the paper's ``x W_r`` is ``x @ w_r.T``.
+    """
+    return _f64(x) @ _f64(w_r).T
+
+
+# ----------------------------------------------------------------------------------------------
+# Section 4.1, second equation: I = TopKMask(s, K)
+# ----------------------------------------------------------------------------------------------
+def topk_indices(s, K: int) -> np.ndarray:
+    """The K experts of TopKMask(s, K) for every token, as indices [T, K].
+
+    Slot order is descending logit; exact ties go to the lower expert index (the paper does not
+    state a tie rule; this is the reading used throughout).  A stable sort of the negated logits
+    gives exactly that order.
+    """
+    s = _f64(s)
+    T, E = s.shape
+    if not 0 < K <= E:
+        raise ValueError("need 0 < K <= E")
+    order = np.argsort(-s, axis=1, kind="stable")
+    return np.ascontiguousarray(order[:, :K]).astype(np.int64)
+
+
+def mask_from_indices(idx, E: int) -> np.ndarray:
+    """Binary mask I in {0,1}^M with exactly K ones per token (Section 4.1: sum_i I_i = K)."""
+    idx = np.asarray(idx, dtype=np.int64)
+    check_record(idx, E)
+    T, K = idx.shape
+    I = np.zeros((T, E), dtype=F64)
+    I[np.arange(T)[:, None], idx] = 1.0
+    return I
+
+
+def check_record(idx, E: int) -> None:
+    """A record is valid when every token lists K distinct experts in [0, E)."""
+    idx = np.asarray(idx)
+    if idx.ndim != 2:
+        raise ValueError("record must be [T, K]")
+    if idx.size and (idx.min() < 0 or idx.max() >= E):
+        raise ValueError("expert index out of range")
+    srt = np.sort(idx, axis=1)
+    if idx.shape[1] > 1 and np.any(srt[:, 1:] == srt[:, :-1]):
+        raise ValueError("duplicate expert in a token's record")
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. (train_gate) / Eq. (replay_gate): softmax of the training logits over a mask
+# ----------------------------------------------------------------------------------------------
+def gate_dense(s, I) -> np.ndarray:
+    """g_i = I_i exp(s_i) / sum_j I_j exp(s_j), all M entries (Eq. train_gate / replay_gate).
+
+    Written exactly as printed, over the dense mask.  The row maximum over the masked entries is
+    subtracted first; that cancels in the ratio.
+    """
+    s = _f64(s)
+    I = _f64(I)
+    m = np.max(np.where(I > 0, s, -np.inf), axis=1, keepdims=True)
+    num = I * np.exp(np.where(I > 0, s - m, 0.0))
+    return num / np.sum(num, axis=1, keepdims=True)
+
+
+def replay_gate(s_train, idx_infer) -> np.ndarray:
+    """Eq. (replay_gate) restricted to the K recorded experts: gates [T, K], slot-aligned.
+
+    g[t, j] = exp(s[t, e_j] - m) / sum_j' exp(s[t, e_j'] - m),  e_j = idx[t, j],
+    m = max_j s[t, e_j].  The M - K other entries of the equation are zero and are not stored.
+    """
+    s = _f64(s_train)
+    idx = np.asarray(idx_infer, dtype=np.int64)
+    check_record(idx, s.shape[1])
+    sel = np.take_along_axis(s, idx, axis=1)
+    z = np.exp(sel - sel.max(axis=1, keepdims=True))
+    return z / z.sum(axis=1, keepdims=True)
+
+
+# ----------------------------------------------------------------------------------------------
+# Expert network E_i (bias-free SwiGLU FFN, width F)
+# ----------------------------------------------------------------------------------------------
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def swiglu_expert(x, w_gate_i, w_up_i, w_down_i) -> np.ndarray:
+    """E_i(x) = W_down,i ( silu(W_gate,i x) * (W_up,i x) ) for rows of x.
+
+    w_gate_i, w_up_i: [F, d]; w_down_i: [d, F]  (all output-major).
+    """
+    x = _f64(x)
+    a = x @ _f64(w_gate_i).T
+    b = x @ _f64(w_up_i).T
+    return (silu(a) * b) @ _f64(w_down_i).T
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. (replay_output):  y = sum_i g_replay,i E_i(x_train)
+# ----------------------------------------------------------------------------------------------
+def expert_outputs(x, idx, w_gate, w_up, w_down) -> np.ndarray:
+    """E_{e_j}(x[t]) for every recorded (token, slot): array [T, K, d].
+
+    These are the only terms of Eq. (replay_output) whose gate is non-zero.  The loop runs over
+    experts i = 1..M as the sum in the equation does, evaluating expert i on the tokens whose
+    mask has I_i = 1.
+    """
+    x = _f64(x)
+    idx = np.asarray(idx, dtype=np.int64)
+    T, K = idx.shape
+    E = len(w_gate)
+    check_record(idx, E)
+    d_out = np.asarray(w_down[0]).shape[0]
+    out = np.zeros((T, K, d_out), dtype=F64)
+    for i in range(E):
+        tt, jj = np.nonzero(idx == i)
+        if tt.size == 0:
+            continue
+        out[tt, jj] = swiglu_expert(x[tt], w_gate[i], w_up[i], w_down[i])
+    return out
+
+
+def replay_output(x, s_train, idx_infer, w_gate, w_up, w_down):
+    """Eq. (replay_output): y[t] = sum_j g[t, j] * E_{e_j}(x[t]).  Returns (y, gates, eo).
+
+    ``eo`` is the [T, K, d] array of expert outputs, returned because the gradient needs it.
+    """
+    g = replay_gate(s_train, idx_infer)
+    eo = expert_outputs(x, idx_infer, w_gate, w_up, w_down)
+    y = np.einsum("tk,tkd->td", g, eo)
+    return y, g, eo
+
+
+def replay_output_dense(x, s_train, I_infer, w_gate, w_up, w_down) -> np.ndarray:
+    """Eq. (replay_output) literally: sum over ALL M experts of g_replay,i E_i(x), dense mask.
+
+    Every expert is evaluated on every token.  Tiny layers only.
+    """
+    x = _f64(x)
+    g = gate_dense(s_train, I_infer)
+    E = g.shape[1]
+    y = np.zeros((x.shape[0], np.asarray(w_down[0]).shape[0]), dtype=F64)
+    for i in range(E):
+        y += g[:, i:i + 1] * swiglu_expert(x, w_gate[i], w_up[i], w_down[i])
+    return y
+
+
+def train_output(x, w_r, K, w_gate, w_up, w_down) -> np.ndarray:
+    """The ordinary MoE layer, Eqs. (train_gate) and (train_output), written on its own:
+    logits, TopKMask, softmax over the selected logits, weighted sum over all M experts."""
+    s = router_logits(x, w_r)
+    I = mask_from_indices(topk_indices(s, K), s.shape[1])
+    return replay_output_dense(x, s, I, w_gate, w_up, w_down)
+
+
+# ----------------------------------------------------------------------------------------------
+# Token dispatch: the (expert, token) ordering implied by evaluating E_i only where I_i = 1
+# ----------------------------------------------------------------------------------------------
+def permutation(idx, E: int):
+    """Stable grouping of the R = T*K (token, slot) pairs by expert.
+
+    Pairs are listed in (t, j) order and stably sorted by key idx[t, j].  Returns
+    counts [E], offsets [E+1] (exclusive scan), row_of_slot [T, K] (destination row of each
+    pair) and slot_of_row [R] (flat pair index t*K + j held by each row), all int32.
+    """
+    idx = np.asarray(idx, dtype=np.int64)
+    check_record(idx, E)
+    T, K = idx.shape
+    flat = idx.reshape(-1)
+    slot_of_row = np.argsort(flat, kind="stable")
+    row_of_slot = np.empty(T * K, dtype=np.int64)
+    row_of_slot[slot_of_row] = np.arange(T * K)
+    counts = np.bincount(flat, minlength=E)
+    offsets = np.concatenate([[0], np.cumsum(counts)])
+    return (counts.astype(np.int32), offsets.astype(np.int32),
+            row_of_slot.reshape(T, K).astype(np.int32), slot_of_row.astype(np.int32))
+
+
+def permute_rows(x, slot_of_row, K: int) -> np.ndarray:
+    """xp[r] = x[token of row r]: the rows each expert reads, grouped by expert."""
+    return np.asarray(x)[np.asarray(slot_of_row, dtype=np.int64) // K]
+
+
+# ----------------------------------------------------------------------------------------------
+# Router-logit gradient through the replayed mask (Section 4.1, purpose (b))
+# ----------------------------------------------------------------------------------------------
+def dgates(dy, eo) -> np.ndarray:
+    """dL/dg[t, j] = <dy[t], E_{e_j}(x[t])>   (chain rule on Eq. replay_output)."""
+    return np.einsum("td,tkd->tk", _f64(dy), _f64(eo))
+
+
+def replay_gate_bwd(g, dg, idx, E: int) -> np.ndarray:
+    """dL/ds_train [T, E] through Eq. (replay_gate) with I_infer held constant.
+
+    On the mask d g_j / d s_{e_j'} = g_j (delta_jj' - g_j'), hence
+    ds[t, e_j] = g_j (dg_j - sum_j' g_j' dg_j');  entries off the mask are zero.
+    """
+    g = _f64(g)
+    dg = _f64(dg)
+    idx = np.asarray(idx, dtype=np.int64)
+    check_record(idx, E)
+    T, K = idx.shape
+    c = np.sum(g * dg, axis=1, keepdims=True)
+    ds = np.zeros((T, E), dtype=F64)
+    ds[np.arange(T)[:, None], idx] = g * (dg - c)
+    return ds
+
+
+def layer_fwd_bwd(x, w_r, idx_infer, w_gate, w_up, w_down, dy):
+    """Whole replayed layer: forward (logits, gate, experts, output) and router-logit backward.
+
+    Returns a dict with s, g, eo, y, dg, ds.
+    """
+    s = router_logits(x, w_r)
+    y, g, eo = replay_output(x, s, idx_infer, w_gate, w_up, w_down)
+    dg = dgates(dy, eo)
+    ds = replay_gate_bwd(g, dg, idx_infer, s.shape[1])
+    return dict(s=s, g=g, eo=eo, y=y, dg=dg, ds=ds)
+
+
+def layer_tokens(x_rows, w_r, idx_rows, w_gate, w_up, w_down, dy_rows):
+    """The same layer evaluated one token at a time, for spot checks at sizes where the whole
+    batch is too slow: for each given token, K expert evaluations straight from the equations.
+    Returns (y [n, d], ds [n, E])."""
+    x_rows = _f64(x_rows)
+    dy_rows = _f64(dy_rows)
+    idx_rows = np.asarray(idx_rows, dtype=np.int64)
+    n, K = idx_rows.shape
+    E = len(w_gate)
+    ys, dss = [], []
+    for t in range(n):
+        xt = x_rows[t:t + 1]
+        s = router_logits(xt, w_r)
+        g = replay_gate(s, idx_rows[t:t + 1])
+        eo = np.stack([swiglu_expert(xt, w_gate[e], w_up[e], w_down[e])[0]
+                       for e in idx_rows[t]])[None]
+        ys.append(np.einsum("tk,tkd->td", g, eo)[0])
+        dg = dgates(dy_rows[t:t + 1], eo)
+        dss.append(replay_gate_bwd(g, dg, idx_rows[t:t + 1], E)[0])
+    return np.stack(ys), np.stack(dss)
