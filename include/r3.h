@@ -1,0 +1,169 @@
+/*
+ * r3.h - C ABI of the replayed-routing MoE layer (Rollout Routing Replay, "R3") for NVIDIA B200.
+ *
+ * The library evaluates one Mixture-of-Experts layer whose expert selection is REPLAYED from a
+ * record made by an inference engine, as defined in Section 4.1 of the paper
+ * "Stabilizing MoE Reinforcement Learning by Aligning Training and Inference Routers":
+ *
+ *   s        = x W_r                                            (router logits, first equation)
+ *   I        = TopKMask(s, K)                                   (second equation; capture side)
+ *   g_i      = I_infer,i exp(s_train,i) / sum_j I_infer,j exp(s_train,j)      (Eq. replay_gate)
+ *   y        = sum_i g_i E_i(x_train)                                          (Eq. replay_output)
+ *
+ * plus the gradient of a loss with respect to s_train through the replayed gate (the mask is a
+ * constant; Section 4.1, purpose (b)).  The expert network E_i is a bias-free SwiGLU feed-forward
+ * network of width F:  E_i(x) = W_down,i ( silu(W_gate,i x) * (W_up,i x) ).
+ *
+ * Notation: T tokens, d hidden size, E (= M) experts, K experts per token, R = T*K rows.
+ *
+ * General rules
+ *  - Every pointer is a DEVICE pointer owned by the caller unless the parameter is documented as
+ *    "host".  The library never allocates, frees or synchronises (except r3_replay_layer_host,
+ *    which synchronises the stream before it returns); each call enqueues its kernels on
+ *    `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and returns.
+ *  - Matrices are row-major and dense.  Weights are stored output-major: W_r [E, d],
+ *    W_gate/W_up [E, F, d], W_down [E, d, F].
+ *  - Activations and expert weights have dtype `act_dtype` (R3_F32 or R3_BF16); W_r has dtype
+ *    `router_w_dtype`; logits, gates and their gradients are always float32.  All accumulation is
+ *    float32.
+ *  - The routing record holds K expert indices per token, `idx_type` R3_IDX_U8 (E <= 256) or
+ *    R3_IDX_I16 (E <= 32767), laid out [layer][token][slot].  Replay accepts the K indices of a
+ *    token in any order; gates are returned in the same slot order.
+ *  - Alignment: all base pointers 16-byte aligned, workspaces 256-byte aligned; d and F
+ *    multiples of 8.
+ *  - Errors the host can see (null pointer, bad shape, workspace too small, failed launch) are
+ *    returned as r3_status and nothing is launched.  Data-dependent problems (index out of range,
+ *    duplicate index within a token, an internal wait that ran out) are written to the optional
+ *    device word `dev_status` (first error wins; 0 = clean; the caller zeroes it); kernels never
+ *    trap, and skip the offending element.
+ *  - T = 0 returns R3_OK without launching.  Experts with no rows are legal.
+ *  - Results are bit-reproducible from run to run: no floating-point atomics are used anywhere.
+ */
+#ifndef R3_H_
+#define R3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    R3_OK = 0,
+    R3_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, K > E, index type too narrow */
+    R3_ERR_UNSUPPORTED = 2,   /* a legal shape this build has no kernel for */
+    R3_ERR_WORKSPACE = 3,     /* workspace missing, too small or misaligned */
+    R3_ERR_CUDA = 4           /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+} r3_status;
+
+enum { R3_F32 = 0, R3_BF16 = 1 };
+enum { R3_IDX_U8 = 1, R3_IDX_I16 = 2 };
+
+/* values written to *dev_status by kernels */
+enum { R3_DEV_OK = 0, R3_DEV_BAD_INDEX = 1, R3_DEV_DUP_INDEX = 2, R3_DEV_TIMEOUT = 3 };
+
+typedef struct {
+    int32_t T, d, E, K, F;
+    int32_t act_dtype;        /* R3_F32 | R3_BF16 : x, dy, xp, h, o, y, expert weights */
+    int32_t router_w_dtype;   /* R3_F32 | R3_BF16 : W_r */
+    int32_t idx_type;         /* R3_IDX_U8 | R3_IDX_I16 */
+} r3_shape;
+
+const char* r3_status_string(r3_status s);
+
+/* Section 4.1, first and second equations: router logits and TopKMask, fused.
+ *   s[t,i] = sum_c x[t,c] W_r[i,c];  idx_out[t, 0..K) = the K experts with the largest s[t,.],
+ *   slot order = descending logit, exact ties to the lower expert index.
+ * x [T,d] act_dtype; w_router [E,d] router_w_dtype; idx_out [T,K] idx_type (may be NULL when only
+ * logits are wanted); logits_out [T,E] float32 or NULL.  At least one output must be non-NULL.
+ * Used on the inference side to make the record, and on the training side (logits_out set) for
+ * s_train.  Supported: E <= 512. */
+r3_status r3_capture_topk(const r3_shape* shape, const void* x, const void* w_router,
+                          void* idx_out, float* logits_out, void* stream);
+
+/* The same for L independent layers in one launch sequence: x [L,T,d], w_router [L,E,d],
+ * idx_out [L,T,K], logits_out [L,T,E] or NULL. */
+r3_status r3_capture_topk_batched(const r3_shape* shape, int32_t L, const void* x,
+                                  const void* w_router, void* idx_out, float* logits_out,
+                                  void* stream);
+
+/* Eq. (replay_gate): softmax of the TRAINING logits over the K RECORDED experts.
+ *   gates[t,j] = exp(s[t,e_j] - m) / sum_j' exp(s[t,e_j'] - m),  e_j = idx[t,j], m = max_j s[t,e_j]
+ * logits [T,E] f32; idx [T,K]; gates [T,K] f32 (slot-aligned with idx).
+ * dev_status (optional): R3_DEV_BAD_INDEX / R3_DEV_DUP_INDEX if a token's record is invalid; the
+ * gates of such a token are written as 0. */
+r3_status r3_replay_gate_fwd(const r3_shape* shape, const float* logits, const void* idx,
+                             float* gates, int32_t* dev_status, void* stream);
+
+/* Gradient through Eq. (replay_gate) with the mask held constant:
+ *   c = sum_j g[t,j] dg[t,j];  dlogits[t,e_j] = g[t,j] (dg[t,j] - c);  dlogits[t,i] = 0 elsewhere.
+ * gates, dgates [T,K] f32; idx [T,K]; dlogits [T,E] f32, every element written. */
+r3_status r3_replay_gate_bwd(const r3_shape* shape, const float* gates, const float* dgates,
+                             const void* idx, float* dlogits, void* stream);
+
+/* Token dispatch implied by Eq. (replay_output): expert i is evaluated only on tokens whose
+ * recorded mask has I_i = 1.  The R (token, slot) pairs are grouped by expert, stably (within an
+ * expert, ascending token).
+ *   counts[e]        = number of pairs with idx = e                       [E]   int32
+ *   offsets          = exclusive scan of counts, offsets[E] = R           [E+1] int32
+ *   row_of_slot[t,j] = destination row of pair (t,j)                      [T,K] int32
+ *   slot_of_row[r]   = t*K + j of the pair stored in row r                [R]   int32
+ *   xp[r]            = x[slot_of_row[r] / K]                              [R,d] act_dtype
+ * x / xp may both be NULL to compute the maps only.  Integer outputs are exact and independent of
+ * scheduling.  workspace: r3_permute_workspace_bytes(shape) bytes.  Supported: E <= 1024.
+ * dev_status (optional): R3_DEV_BAD_INDEX for an index >= E (that pair is dropped). */
+size_t r3_permute_workspace_bytes(const r3_shape* shape);
+r3_status r3_permute(const r3_shape* shape, const void* idx, const void* x, int32_t* counts,
+                     int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* xp,
+                     void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* Expert networks E_i on the grouped rows: for expert e and rows r in [offsets[e], offsets[e+1])
+ *   h[r] = silu(xp[r] W_gate,e^T) * (xp[r] W_up,e^T);   o[r] = h[r] W_down,e^T.
+ * xp [R,d]; offsets [E+1]; w_gate, w_up [E,F,d]; w_down [E,d,F]; o [R,d]; all act_dtype.
+ * bf16: tcgen05 tensor-core grouped GEMMs with fp32 accumulation, h and o rounded to bf16.
+ * f32:  plain fp32 FMA kernels.
+ * workspace: r3_grouped_swiglu_workspace_bytes(shape) bytes (holds h [R,F] and the tile list).
+ * dev_status (optional): R3_DEV_TIMEOUT if an internal bounded wait ran out (outputs invalid). */
+size_t r3_grouped_swiglu_workspace_bytes(const r3_shape* shape);
+r3_status r3_grouped_swiglu(const r3_shape* shape, const void* xp, const int32_t* offsets,
+                            const void* w_gate, const void* w_up, const void* w_down, void* o,
+                            void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* Eq. (replay_output): y[t] = sum_{j=0..K-1} gates[t,j] * o[row_of_slot[t,j]], added in slot
+ * order in fp32 (no atomics), rounded once to act_dtype.  o [R,d]; y [T,d]. */
+r3_status r3_combine(const r3_shape* shape, const void* o, const int32_t* row_of_slot,
+                     const float* gates, void* y, void* stream);
+
+/* Chain rule on Eq. (replay_output): dgates[t,j] = sum_c dy[t,c] * o[row_of_slot[t,j], c].
+ * dy [T,d] act_dtype; dgates [T,K] f32. */
+r3_status r3_combine_bwd_gates(const r3_shape* shape, const void* dy, const void* o,
+                               const int32_t* row_of_slot, float* dgates, void* stream);
+
+/* The whole replayed layer, forward and router-logit backward, enqueued back to back on one
+ * stream: logits -> replay gate -> permute -> experts -> combine -> dgates -> dlogits.
+ * Inputs x [T,d], w_router [E,d], idx [T,K], expert weights, dy [T,d];
+ * outputs y [T,d] act_dtype and dlogits [T,E] f32.  Intermediates live in `workspace`
+ * (r3_replay_layer_workspace_bytes).  Optional outputs (may be NULL): gates_out [T,K] f32. */
+size_t r3_replay_layer_workspace_bytes(const r3_shape* shape);
+r3_status r3_replay_layer(const r3_shape* shape, const void* x, const void* w_router,
+                          const void* idx, const void* w_gate, const void* w_up,
+                          const void* w_down, const void* dy, void* y, float* dlogits,
+                          float* gates_out, void* workspace, size_t ws_bytes,
+                          int32_t* dev_status, void* stream);
+
+/* As r3_replay_layer, with the per-step tensors in HOST memory (pinned memory recommended):
+ * x_host, idx_host, dy_host are copied to the device, y_host and dlogits_host are copied back,
+ * and the stream is synchronised before returning.  Weights stay on the device.  The workspace
+ * must hold r3_replay_layer_host_workspace_bytes(shape) bytes (device staging included). */
+size_t r3_replay_layer_host_workspace_bytes(const r3_shape* shape);
+r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host, const void* w_router,
+                               const void* idx_host, const void* w_gate, const void* w_up,
+                               const void* w_down, const void* dy_host, void* y_host,
+                               float* dlogits_host, void* workspace, size_t ws_bytes,
+                               int32_t* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* R3_H_ */

@@ -1,0 +1,39 @@
+// Internal (non-exported) interfaces between the translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "r3.h"
+
+namespace r3 {
+
+// Device-side tile list of the grouped GEMMs: int32 header[4] = {number of M tiles, BM, 0, 0}
+// followed by one int32[4] entry per M tile = {expert, first row, valid rows, 0}.  Tiles are
+// listed expert by expert, rows ascending; an M tile never spans two experts.
+constexpr int kTileHeaderInts = 4;
+inline size_t tile_list_bytes(long long R, int E, int BM) {
+    const long long max_tiles = R / BM + E + 1;
+    return (size_t)(kTileHeaderInts + 4 * max_tiles) * sizeof(int32_t);
+}
+inline int max_m_tiles(long long R, int E, int BM) {
+    const long long by_rows = R / BM + E;          // each expert adds at most one partial tile
+    const long long by_pairs = R < by_rows ? R : by_rows;   // and no more tiles than rows
+    return (int)(by_pairs > 0 ? by_pairs : 0);
+}
+
+// Builds the tile list from offsets [E+1] (one small kernel).
+r3_status launch_build_tiles(const int32_t* offsets, int E, int BM, int32_t* tiles,
+                             cudaStream_t stream);
+
+// bf16 grouped SwiGLU on the tcgen05 tensor cores (sm_100a).  `tiles` must have been built with
+// BM = tc_block_m().
+int tc_block_m();
+r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const int32_t* tiles,
+                                   const void* w_gate, const void* w_up, const void* w_down,
+                                   void* h, void* o, int32_t* dev_status, cudaStream_t stream);
+
+// Number of SMs of the current device (cached).
+int sm_count();
+
+}  // namespace r3

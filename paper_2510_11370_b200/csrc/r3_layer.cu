@@ -1,0 +1,164 @@
+// The whole replayed layer as one enqueue: logits -> replay gate -> permute -> experts ->
+// combine -> dgates -> dlogits (Section 4.1, Eqs. replay_gate / replay_output and the
+// router-logit gradient), plus a variant whose per-step tensors live in host memory.
+#include "r3_common.cuh"
+
+namespace r3 {
+
+struct LayerWs {
+    float* logits;
+    float* gates;
+    float* dgates;
+    int32_t* counts;
+    int32_t* offsets;
+    int32_t* row_of_slot;
+    int32_t* slot_of_row;
+    void* xp;
+    void* o;
+    void* permute_ws;
+    size_t permute_bytes;
+    void* swiglu_ws;
+    size_t swiglu_bytes;
+    size_t total;
+};
+
+// Carves the workspace; with base == nullptr only the total size is meaningful.
+static LayerWs carve(const r3_shape* s, void* base) {
+    LayerWs w;
+    size_t off = 0;
+    char* b = static_cast<char*>(base);
+    auto take = [&](size_t bytes) {
+        void* p = b ? b + off : nullptr;
+        off += round_up(bytes ? bytes : 1, 256);
+        return p;
+    };
+    const size_t T = s->T, K = s->K, E = s->E, R = T * K;
+    w.logits = static_cast<float*>(take(T * E * 4));
+    w.gates = static_cast<float*>(take(R * 4));
+    w.dgates = static_cast<float*>(take(R * 4));
+    w.counts = static_cast<int32_t*>(take(E * 4));
+    w.offsets = static_cast<int32_t*>(take((E + 1) * 4));
+    w.row_of_slot = static_cast<int32_t*>(take(R * 4));
+    w.slot_of_row = static_cast<int32_t*>(take(R * 4));
+    w.xp = take(R * s->d * act_bytes(s));
+    w.o = take(R * s->d * act_bytes(s));
+    w.permute_bytes = r3_permute_workspace_bytes(s);
+    w.permute_ws = take(w.permute_bytes);
+    w.swiglu_bytes = r3_grouped_swiglu_workspace_bytes(s);
+    w.swiglu_ws = take(w.swiglu_bytes);
+    w.total = off;
+    return w;
+}
+
+}  // namespace r3
+
+extern "C" size_t r3_replay_layer_workspace_bytes(const r3_shape* shape) {
+    if (r3::check_shape(shape) != R3_OK) return 0;
+    return r3::carve(shape, nullptr).total;
+}
+
+extern "C" r3_status r3_replay_layer(const r3_shape* shape, const void* x, const void* w_router,
+                                     const void* idx, const void* w_gate, const void* w_up,
+                                     const void* w_down, const void* dy, void* y, float* dlogits,
+                                     float* gates_out, void* workspace, size_t ws_bytes,
+                                     int32_t* dev_status, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->T == 0) return R3_OK;
+    if (!x || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !y || !dlogits)
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_layer_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    const r3::LayerWs w = r3::carve(shape, workspace);
+    float* gates = gates_out ? gates_out : w.gates;
+
+    // s_train = x W_r (only the logits are needed on the training side)
+    if ((st = r3_capture_topk(shape, x, w_router, nullptr, w.logits, stream)) != R3_OK) return st;
+    if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
+        return st;
+    if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
+                         w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
+        return st;
+    if ((st = r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, w.swiglu_ws,
+                                w.swiglu_bytes, dev_status, stream)) != R3_OK)
+        return st;
+    if ((st = r3_combine(shape, w.o, w.row_of_slot, gates, y, stream)) != R3_OK) return st;
+    if ((st = r3_combine_bwd_gates(shape, dy, w.o, w.row_of_slot, w.dgates, stream)) != R3_OK)
+        return st;
+    return r3_replay_gate_bwd(shape, gates, w.dgates, idx, dlogits, stream);
+}
+
+namespace r3 {
+struct HostWs {
+    void* x; void* idx; void* dy; void* y; float* dlogits; void* inner; size_t inner_bytes;
+    size_t total;
+};
+static HostWs carve_host(const r3_shape* s, void* base) {
+    HostWs h;
+    size_t off = 0;
+    char* b = static_cast<char*>(base);
+    auto take = [&](size_t bytes) {
+        void* p = b ? b + off : nullptr;
+        off += round_up(bytes ? bytes : 1, 256);
+        return p;
+    };
+    const size_t T = s->T, row = (size_t)s->d * act_bytes(s);
+    h.x = take(T * row);
+    h.idx = take(T * s->K * idx_bytes(s));
+    h.dy = take(T * row);
+    h.y = take(T * row);
+    h.dlogits = static_cast<float*>(take(T * s->E * 4));
+    h.inner_bytes = r3_replay_layer_workspace_bytes(s);
+    h.inner = take(h.inner_bytes);
+    h.total = off;
+    return h;
+}
+}  // namespace r3
+
+extern "C" size_t r3_replay_layer_host_workspace_bytes(const r3_shape* shape) {
+    if (r3::check_shape(shape) != R3_OK) return 0;
+    return r3::carve_host(shape, nullptr).total;
+}
+
+extern "C" r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host,
+                                          const void* w_router, const void* idx_host,
+                                          const void* w_gate, const void* w_up,
+                                          const void* w_down, const void* dy_host, void* y_host,
+                                          float* dlogits_host, void* workspace, size_t ws_bytes,
+                                          int32_t* dev_status, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->T == 0) return R3_OK;
+    if (!x_host || !idx_host || !dy_host || !y_host || !dlogits_host) return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_layer_host_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const r3::HostWs h = r3::carve_host(shape, workspace);
+    const size_t T = shape->T, row = (size_t)shape->d * r3::act_bytes(shape);
+    if (cudaMemcpyAsync(h.x, x_host, T * row, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaMemcpyAsync(h.idx, idx_host, T * shape->K * r3::idx_bytes(shape),
+                        cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaMemcpyAsync(h.dy, dy_host, T * row, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+        return R3_ERR_CUDA;
+    st = r3_replay_layer(shape, h.x, w_router, h.idx, w_gate, w_up, w_down, h.dy, h.y, h.dlogits,
+                         nullptr, h.inner, h.inner_bytes, dev_status, stream);
+    if (st != R3_OK) return st;
+    if (cudaMemcpyAsync(y_host, h.y, T * row, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+        cudaMemcpyAsync(dlogits_host, h.dlogits, T * shape->E * 4, cudaMemcpyDeviceToHost, cs) !=
+            cudaSuccess)
+        return R3_ERR_CUDA;
+    return cudaStreamSynchronize(cs) == cudaSuccess ? R3_OK : R3_ERR_CUDA;
+}
+
+extern "C" const char* r3_status_string(r3_status s) {
+    switch (s) {
+        case R3_OK: return "R3_OK";
+        case R3_ERR_INVALID_ARG: return "R3_ERR_INVALID_ARG: null pointer, bad size or dtype code";
+        case R3_ERR_UNSUPPORTED: return "R3_ERR_UNSUPPORTED: no kernel for this shape";
+        case R3_ERR_WORKSPACE: return "R3_ERR_WORKSPACE: workspace missing, too small or misaligned";
+        case R3_ERR_CUDA: return "R3_ERR_CUDA: a CUDA call failed";
+    }
+    return "unknown r3_status";
+}

@@ -1,0 +1,222 @@
+// Token dispatch for the replayed layer: group the R = T*K (token, slot) pairs by recorded
+// expert, stably, and copy each token's row to its K destination rows.
+//
+// Determinism: ranks never depend on the arrival order of atomics.  A CTA owns a chunk of 256
+// consecutive tokens; (1) it counts its pairs per expert (integer atomics on shared counters -
+// the sum does not depend on order), (2) one CTA turns the [expert][chunk] counts into exclusive
+// prefixes and the expert offsets, (3) each CTA marks, per expert, the bitmap of its tokens that
+// chose the expert; the rank of a pair inside the chunk is the number of lower set bits.
+// A pair whose index is out of range, or repeats an earlier slot of the same token, is dropped
+// (row_of_slot = -1) and reported through dev_status.
+#include "r3_common.cuh"
+
+namespace r3 {
+
+constexpr int kChunk = 256;               // tokens per CTA in the counting / ranking kernels
+constexpr int kWords = kChunk / 32;
+
+template <typename IdxT>
+__device__ __forceinline__ bool pair_ok(const IdxT* rec, int j, int E, int& e, int32_t* dev_status) {
+    e = idx_to_int(rec[j]);
+    if (e < 0 || e >= E) { report(dev_status, R3_DEV_BAD_INDEX); return false; }
+    for (int j2 = 0; j2 < j; ++j2)
+        if (idx_to_int(rec[j2]) == e) { report(dev_status, R3_DEV_DUP_INDEX); return false; }
+    return true;
+}
+
+template <typename IdxT>
+__global__ void __launch_bounds__(kChunk)
+permute_count_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ chunk_counts,
+                     int T, int E, int K, int NB, int32_t* dev_status) {
+    extern __shared__ int32_t hist[];
+    for (int e = threadIdx.x; e < E; e += kChunk) hist[e] = 0;
+    __syncthreads();
+    const int t = blockIdx.x * kChunk + threadIdx.x;
+    if (t < T) {
+        const IdxT* rec = idx + (size_t)t * K;
+        for (int j = 0; j < K; ++j) {
+            int e;
+            if (pair_ok(rec, j, E, e, dev_status)) atomicAdd(&hist[e], 1);
+        }
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += kChunk)
+        chunk_counts[(size_t)e * NB + blockIdx.x] = hist[e];
+}
+
+// One CTA.  In place: chunk_counts[e][b] becomes the number of expert-e pairs in chunks < b.
+// Also writes counts[E] and offsets[E+1].
+__global__ void __launch_bounds__(1024)
+permute_scan_kernel(int32_t* __restrict__ chunk_counts, int32_t* __restrict__ counts,
+                    int32_t* __restrict__ offsets, int E, int NB) {
+    __shared__ int32_t total[kMaxExpertsPermute];
+    __shared__ int32_t warp_sum[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int e = warp; e < E; e += 32) {
+        int32_t* row = chunk_counts + (size_t)e * NB;
+        int32_t carry = 0;
+        for (int b0 = 0; b0 < NB; b0 += 256) {
+            int32_t v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int b = b0 + u * 32 + lane;
+                v[u] = b < NB ? row[b] : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                int32_t inc = v[u];
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                const int b = b0 + u * 32 + lane;
+                if (b < NB) row[b] = carry + inc - v[u];
+                carry += __shfl_sync(0xffffffffu, inc, 31);
+            }
+        }
+        if (lane == 0) total[e] = carry;
+    }
+    __syncthreads();
+    // exclusive scan of total[0..E) over the block (E <= 1024 = blockDim)
+    const int e = threadIdx.x;
+    const int32_t mine = e < E ? total[e] : 0;
+    int32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_sum[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int32_t w = warp_sum[lane], winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t n = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += n;
+        }
+        warp_sum[lane] = winc - w;
+    }
+    __syncthreads();
+    const int32_t excl = warp_sum[warp] + inc - mine;
+    if (e < E) {
+        counts[e] = mine;
+        offsets[e] = excl;
+        if (e == E - 1) offsets[E] = excl + mine;
+    }
+}
+
+template <typename IdxT>
+__global__ void __launch_bounds__(kChunk)
+permute_rank_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ chunk_base,
+                    const int32_t* __restrict__ offsets, int32_t* __restrict__ row_of_slot,
+                    int32_t* __restrict__ slot_of_row, int T, int E, int K, int NB) {
+    extern __shared__ uint32_t bits[];            // [E][kWords]
+    for (int i = threadIdx.x; i < E * kWords; i += kChunk) bits[i] = 0u;
+    __syncthreads();
+    const int lt = threadIdx.x;
+    const int t = blockIdx.x * kChunk + lt;
+    const IdxT* rec = idx + (size_t)(t < T ? t : 0) * K;
+    if (t < T) {
+        for (int j = 0; j < K; ++j) {
+            int e;
+            if (pair_ok(rec, j, E, e, nullptr)) atomicOr(&bits[e * kWords + (lt >> 5)], 1u << (lt & 31));
+        }
+    }
+    __syncthreads();
+    if (t < T) {
+        for (int j = 0; j < K; ++j) {
+            int e;
+            int32_t row = -1;
+            if (pair_ok(rec, j, E, e, nullptr)) {
+                const uint32_t* m = bits + e * kWords;
+                int rank = __popc(m[lt >> 5] & ((1u << (lt & 31)) - 1u));
+                for (int w = 0; w < (lt >> 5); ++w) rank += __popc(m[w]);
+                row = offsets[e] + chunk_base[(size_t)e * NB + blockIdx.x] + rank;
+                slot_of_row[row] = t * K + j;
+            }
+            row_of_slot[(size_t)t * K + j] = row;
+        }
+    }
+}
+
+// One warp per token: read x[t] once (16-byte pieces), write it to the token's K rows.
+template <int VEC_BYTES>
+__global__ void __launch_bounds__(256)
+permute_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ row_of_slot,
+                    uint4* __restrict__ xp, int T, int K, int row_vecs) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const uint4* src = x + (size_t)t * row_vecs;
+    const int32_t* rows = row_of_slot + (size_t)t * K;
+    for (int c0 = 0; c0 < row_vecs; c0 += 128) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int c = c0 + u * 32 + lane;
+            if (c < row_vecs) v[u] = src[c];
+        }
+        for (int j = 0; j < K; ++j) {
+            const int32_t r = rows[j];
+            if (r < 0) continue;
+            uint4* dst = xp + (size_t)r * row_vecs;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = c0 + u * 32 + lane;
+                if (c < row_vecs) dst[c] = v[u];
+            }
+        }
+    }
+}
+
+}  // namespace r3
+
+extern "C" size_t r3_permute_workspace_bytes(const r3_shape* shape) {
+    if (r3::check_shape(shape) != R3_OK) return 0;
+    const size_t NB = (shape->T + r3::kChunk - 1) / r3::kChunk;
+    return r3::round_up((size_t)shape->E * (NB ? NB : 1) * sizeof(int32_t), 256);
+}
+
+extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const void* x,
+                                int32_t* counts, int32_t* offsets, int32_t* row_of_slot,
+                                int32_t* slot_of_row, void* xp, void* workspace, size_t ws_bytes,
+                                int32_t* dev_status, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->E > r3::kMaxExpertsPermute) return R3_ERR_UNSUPPORTED;
+    if (!counts || !offsets) return R3_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (shape->T == 0) {
+        // nothing to group: counts and offsets are still defined (all zero)
+        if (cudaMemsetAsync(counts, 0, sizeof(int32_t) * shape->E, cs) != cudaSuccess ||
+            cudaMemsetAsync(offsets, 0, sizeof(int32_t) * (shape->E + 1), cs) != cudaSuccess)
+            return R3_ERR_CUDA;
+        return R3_OK;
+    }
+    if (!idx || !row_of_slot || !slot_of_row) return R3_ERR_INVALID_ARG;
+    if ((x == nullptr) != (xp == nullptr)) return R3_ERR_INVALID_ARG;
+    if (x && (!r3::aligned(x, 16) || !r3::aligned(xp, 16))) return R3_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < r3_permute_workspace_bytes(shape) || !r3::aligned(workspace, 256))
+        return R3_ERR_WORKSPACE;
+
+    const int T = shape->T, E = shape->E, K = shape->K;
+    const int NB = (T + r3::kChunk - 1) / r3::kChunk;
+    int32_t* chunk_counts = static_cast<int32_t*>(workspace);
+    R3_DISPATCH_IDX(shape, IdxT,
+        r3::permute_count_kernel<IdxT><<<NB, r3::kChunk, E * sizeof(int32_t), cs>>>(
+            static_cast<const IdxT*>(idx), chunk_counts, T, E, K, NB, dev_status));
+    r3::permute_scan_kernel<<<1, 1024, 0, cs>>>(chunk_counts, counts, offsets, E, NB);
+    R3_DISPATCH_IDX(shape, IdxT,
+        r3::permute_rank_kernel<IdxT><<<NB, r3::kChunk, E * r3::kWords * sizeof(uint32_t), cs>>>(
+            static_cast<const IdxT*>(idx), chunk_counts, offsets, row_of_slot, slot_of_row,
+            T, E, K, NB));
+    if (x) {
+        const int row_vecs = (int)((size_t)shape->d * r3::act_bytes(shape) / 16);
+        const int wpb = 8;
+        r3::permute_rows_kernel<16><<<(T + wpb - 1) / wpb, wpb * 32, 0, cs>>>(
+            static_cast<const uint4*>(x), row_of_slot, static_cast<uint4*>(xp), T, K, row_vecs);
+    }
+    return r3::launch_status();
+}

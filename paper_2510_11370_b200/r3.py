@@ -1,0 +1,268 @@
+"""Thin ctypes binding over libr3_b200.so (the C ABI declared in include/r3.h).
+
+Argument marshalling only: every step of the replayed layer runs in the CUDA library.  PyTorch
+supplies device memory and the current stream.  There is no CPU fallback: importing this module
+without a built library raises, and every call requires CUDA tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libr3_b200.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2510_11370_b200.build` "
+        "(needs nvcc; there is no CPU fallback)")
+lib = ctypes.CDLL(_LIB_PATH)
+
+R3_OK = 0
+R3_F32, R3_BF16 = 0, 1
+R3_IDX_U8, R3_IDX_I16 = 1, 2
+DEV_OK, DEV_BAD_INDEX, DEV_DUP_INDEX, DEV_TIMEOUT = 0, 1, 2, 3
+
+EXPORTS = [
+    "r3_status_string", "r3_capture_topk", "r3_capture_topk_batched", "r3_replay_gate_fwd",
+    "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute",
+    "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_combine",
+    "r3_combine_bwd_gates", "r3_replay_layer_workspace_bytes", "r3_replay_layer",
+    "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
+]
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int32), ("d", ctypes.c_int32), ("E", ctypes.c_int32),
+                ("K", ctypes.c_int32), ("F", ctypes.c_int32), ("act_dtype", ctypes.c_int32),
+                ("router_w_dtype", ctypes.c_int32), ("idx_type", ctypes.c_int32)]
+
+
+_P = ctypes.c_void_p
+_SP = ctypes.POINTER(Shape)
+lib.r3_status_string.restype = ctypes.c_char_p
+lib.r3_status_string.argtypes = [ctypes.c_int]
+for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
+           "r3_replay_layer_workspace_bytes", "r3_replay_layer_host_workspace_bytes"):
+    getattr(lib, _n).restype = ctypes.c_size_t
+    getattr(lib, _n).argtypes = [_SP]
+lib.r3_capture_topk.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_capture_topk_batched.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P]
+lib.r3_replay_gate_fwd.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_replay_gate_bwd.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_permute.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
+lib.r3_grouped_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
+lib.r3_combine.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
+lib.r3_replay_layer_host.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
+for _n in EXPORTS:
+    if _n not in ("r3_status_string",) and not _n.endswith("_bytes"):
+        getattr(lib, _n).restype = ctypes.c_int
+
+
+class R3Error(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(lib.r3_status_string(code).decode())
+
+
+def _check(code: int) -> None:
+    if code != R3_OK:
+        raise R3Error(code)
+
+
+_ACT = {torch.float32: R3_F32, torch.bfloat16: R3_BF16}
+_IDX = {torch.uint8: R3_IDX_U8, torch.int16: R3_IDX_I16}
+
+
+def make_shape(T, d, E, K, F, act=torch.bfloat16, router=torch.float32, idx=torch.uint8) -> Shape:
+    return Shape(T, d, E, K, F, _ACT[act], _ACT[router], _IDX[idx])
+
+
+def shape_of(w) -> Shape:
+    """Shape of a synth.Workload."""
+    return make_shape(w.T, w.d, w.E, w.K, w.F, w.act_dtype, w.router_dtype, w.idx_dtype)
+
+
+def _act_dtype(s: Shape):
+    return torch.bfloat16 if s.act_dtype == R3_BF16 else torch.float32
+
+
+def _idx_dtype(s: Shape):
+    return torch.uint8 if s.idx_type == R3_IDX_U8 else torch.int16
+
+
+def _ptr(t, host: bool = False):
+    if t is None:
+        return None
+    if not isinstance(t, torch.Tensor):
+        raise TypeError("expected a torch.Tensor")
+    if host:
+        if t.is_cuda:
+            raise ValueError("expected a host tensor")
+    elif not t.is_cuda:
+        raise ValueError("expected a CUDA tensor (there is no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dev(*ts):
+    for t in ts:
+        if isinstance(t, torch.Tensor):
+            return t.device
+    return torch.device("cuda")
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    """Device scratch of at least nbytes, 256-byte aligned (torch's allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def new_status(device) -> torch.Tensor:
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+# ---------------------------------------------------------------------------------------------
+def capture_topk(s: Shape, x, w_router, idx_out=None, logits_out=None, *, want_idx=True,
+                 want_logits=False, stream=None):
+    """Router logits + TopKMask.  Returns (idx [T,K] or None, logits [T,E] or None)."""
+    dev = _dev(x)
+    if idx_out is None and want_idx:
+        idx_out = torch.empty((s.T, s.K), dtype=_idx_dtype(s), device=dev)
+    if logits_out is None and want_logits:
+        logits_out = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
+    _check(lib.r3_capture_topk(ctypes.byref(s), _ptr(x), _ptr(w_router), _ptr(idx_out),
+                               _ptr(logits_out), _stream(stream)))
+    return idx_out, logits_out
+
+
+def capture_topk_batched(s: Shape, L: int, x, w_router, idx_out=None, logits_out=None, *,
+                         want_idx=True, want_logits=False, stream=None):
+    """L layers at once: x [L,T,d], w_router [L,E,d] -> idx [L,T,K], logits [L,T,E]."""
+    dev = _dev(x)
+    if idx_out is None and want_idx:
+        idx_out = torch.empty((L, s.T, s.K), dtype=_idx_dtype(s), device=dev)
+    if logits_out is None and want_logits:
+        logits_out = torch.empty((L, s.T, s.E), dtype=torch.float32, device=dev)
+    _check(lib.r3_capture_topk_batched(ctypes.byref(s), L, _ptr(x), _ptr(w_router),
+                                       _ptr(idx_out), _ptr(logits_out), _stream(stream)))
+    return idx_out, logits_out
+
+
+def replay_gate_fwd(s: Shape, logits, idx, gates=None, dev_status=None, stream=None):
+    if gates is None:
+        gates = torch.empty((s.T, s.K), dtype=torch.float32, device=_dev(logits))
+    _check(lib.r3_replay_gate_fwd(ctypes.byref(s), _ptr(logits), _ptr(idx), _ptr(gates),
+                                  _ptr(dev_status), _stream(stream)))
+    return gates
+
+
+def replay_gate_bwd(s: Shape, gates, dgates, idx, dlogits=None, stream=None):
+    if dlogits is None:
+        dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=_dev(gates))
+    _check(lib.r3_replay_gate_bwd(ctypes.byref(s), _ptr(gates), _ptr(dgates), _ptr(idx),
+                                  _ptr(dlogits), _stream(stream)))
+    return dlogits
+
+
+def permute_workspace_bytes(s: Shape) -> int:
+    return lib.r3_permute_workspace_bytes(ctypes.byref(s))
+
+
+def permute(s: Shape, idx, x=None, *, out=None, ws=None, dev_status=None, stream=None):
+    """Returns (counts, offsets, row_of_slot, slot_of_row, xp or None)."""
+    dev = _dev(idx)
+    R = s.T * s.K
+    if out is None:
+        counts = torch.empty(s.E, dtype=torch.int32, device=dev)
+        offsets = torch.empty(s.E + 1, dtype=torch.int32, device=dev)
+        ros = torch.empty((s.T, s.K), dtype=torch.int32, device=dev)
+        sor = torch.empty(R, dtype=torch.int32, device=dev)
+        xp = torch.empty((R, s.d), dtype=_act_dtype(s), device=dev) if x is not None else None
+    else:
+        counts, offsets, ros, sor, xp = out
+    if ws is None:
+        ws = workspace(permute_workspace_bytes(s), dev)
+    _check(lib.r3_permute(ctypes.byref(s), _ptr(idx), _ptr(x), _ptr(counts), _ptr(offsets),
+                          _ptr(ros), _ptr(sor), _ptr(xp), _ptr(ws), ws.numel(),
+                          _ptr(dev_status), _stream(stream)))
+    return counts, offsets, ros, sor, xp
+
+
+def grouped_swiglu_workspace_bytes(s: Shape) -> int:
+    return lib.r3_grouped_swiglu_workspace_bytes(ctypes.byref(s))
+
+
+def grouped_swiglu(s: Shape, xp, offsets, w_gate, w_up, w_down, o=None, *, ws=None,
+                   dev_status=None, stream=None):
+    dev = _dev(xp)
+    if o is None:
+        o = torch.empty((s.T * s.K, s.d), dtype=_act_dtype(s), device=dev)
+    if ws is None:
+        ws = workspace(grouped_swiglu_workspace_bytes(s), dev)
+    _check(lib.r3_grouped_swiglu(ctypes.byref(s), _ptr(xp), _ptr(offsets), _ptr(w_gate),
+                                 _ptr(w_up), _ptr(w_down), _ptr(o), _ptr(ws), ws.numel(),
+                                 _ptr(dev_status), _stream(stream)))
+    return o
+
+
+def combine(s: Shape, o, row_of_slot, gates, y=None, stream=None):
+    if y is None:
+        y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=_dev(o))
+    _check(lib.r3_combine(ctypes.byref(s), _ptr(o), _ptr(row_of_slot), _ptr(gates), _ptr(y),
+                          _stream(stream)))
+    return y
+
+
+def combine_bwd_gates(s: Shape, dy, o, row_of_slot, dgates=None, stream=None):
+    if dgates is None:
+        dgates = torch.empty((s.T, s.K), dtype=torch.float32, device=_dev(o))
+    _check(lib.r3_combine_bwd_gates(ctypes.byref(s), _ptr(dy), _ptr(o), _ptr(row_of_slot),
+                                    _ptr(dgates), _stream(stream)))
+    return dgates
+
+
+def replay_layer_workspace_bytes(s: Shape) -> int:
+    return lib.r3_replay_layer_workspace_bytes(ctypes.byref(s))
+
+
+def replay_layer(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, y=None, dlogits=None,
+                 gates=None, ws=None, dev_status=None, stream=None):
+    """Forward + router-logit backward of the replayed layer.  Returns (y, dlogits, gates)."""
+    dev = _dev(x)
+    if y is None:
+        y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    if dlogits is None:
+        dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
+    if gates is None:
+        gates = torch.empty((s.T, s.K), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(replay_layer_workspace_bytes(s), dev)
+    _check(lib.r3_replay_layer(ctypes.byref(s), _ptr(x), _ptr(w_router), _ptr(idx), _ptr(w_gate),
+                               _ptr(w_up), _ptr(w_down), _ptr(dy), _ptr(y), _ptr(dlogits),
+                               _ptr(gates), _ptr(ws), ws.numel(), _ptr(dev_status),
+                               _stream(stream)))
+    return y, dlogits, gates
+
+
+def replay_layer_host_workspace_bytes(s: Shape) -> int:
+    return lib.r3_replay_layer_host_workspace_bytes(ctypes.byref(s))
+
+
+def replay_layer_host(s: Shape, x_host, w_router, idx_host, w_gate, w_up, w_down, dy_host,
+                      y_host, dlogits_host, *, ws, dev_status=None, stream=None):
+    """As replay_layer with x, idx, dy, y, dlogits in (pinned) host memory; synchronises."""
+    _check(lib.r3_replay_layer_host(ctypes.byref(s), _ptr(x_host, True), _ptr(w_router),
+                                    _ptr(idx_host, True), _ptr(w_gate), _ptr(w_up), _ptr(w_down),
+                                    _ptr(dy_host, True), _ptr(y_host, True),
+                                    _ptr(dlogits_host, True), _ptr(ws), ws.numel(),
+                                    _ptr(dev_status), _stream(stream)))
+    return y_host, dlogits_host

@@ -194,7 +194,7 @@ def flops_per_token(w: Workload) -> int:
 
 def checksum(t: torch.Tensor) -> int:
     """64-bit order-dependent checksum of a tensor's raw bytes (for logging inputs)."""
-    b = t.detach().contiguous().view(torch.uint8).to("cpu").to(torch.int64)
+    b = t.detach().contiguous().view(torch.uint8).reshape(-1).to("cpu").to(torch.int64)
     n = b.numel()
     wts = (torch.arange(n, dtype=torch.int64) % 251) + 1
     return int((b * wts).sum().item()) & ((1 << 64) - 1)

@@ -1,0 +1,220 @@
+"""Whole replayed layer (forward + router-logit backward) through the C ABI against the oracle,
+on the benchmark configurations.  Small configurations are compared element by element; the
+large ones compare all integer work and the gates exactly/fully, and the expert-dependent
+outputs on sampled tokens that the oracle evaluates one by one."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import r3_oracle as O
+from paper_2510_11370_b200 import synth
+from tests.helpers import Case, f32, f64, rel_err
+from tests.test_gpu_kernels import check_record_against_logits
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 1e-5
+
+
+@pytest.fixture(scope="module")
+def r3():
+    from paper_2510_11370_b200 import r3 as mod
+    return mod
+
+
+def run_layer(r3, case, stepwise=False):
+    s = r3.shape_of(case.w)
+    c = case.cuda()
+    st = r3.new_status("cuda")
+    if not stepwise:
+        y, ds, g = r3.replay_layer(s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"],
+                                   c["w_down"], c["dy"], dev_status=st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        return dict(y=y, ds=ds, g=g)
+    _, logits = r3.capture_topk(s, c["x"], c["w_r"], want_idx=False, want_logits=True)
+    g = r3.replay_gate_fwd(s, logits, c["idx"], dev_status=st)
+    counts, offsets, ros, sor, xp = r3.permute(s, c["idx"], c["x"], dev_status=st)
+    o = r3.grouped_swiglu(s, xp, offsets, c["w_gate"], c["w_up"], c["w_down"], dev_status=st)
+    y = r3.combine(s, o, ros, g)
+    dg = r3.combine_bwd_gates(s, c["dy"], o, ros)
+    ds = r3.replay_gate_bwd(s, g, dg, c["idx"])
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    return dict(y=y, ds=ds, g=g, logits=logits, counts=counts, offsets=offsets, ros=ros, sor=sor,
+                xp=xp, o=o, dg=dg)
+
+
+def check_full(case, got, ref, tol):
+    assert rel_err(f64(got["g"]), ref["g"]) < max(tol * 1e-2, 1e-5)
+    assert rel_err(f64(got["y"]), ref["y"]) < tol
+    assert rel_err(f64(got["ds"]), ref["ds"]) < tol
+    if "sor" in got:
+        counts, offsets, ros, sor = O.permutation(case.idx_np(), case.w.E)
+        assert np.array_equal(got["counts"].cpu().numpy(), counts)
+        assert np.array_equal(got["offsets"].cpu().numpy(), offsets)
+        assert np.array_equal(got["ros"].cpu().numpy(), ros)
+        assert np.array_equal(got["sor"].cpu().numpy(), sor)
+        assert torch.equal(got["xp"].cpu(), case.x[torch.from_numpy(sor.astype(np.int64)) // case.w.K])
+        assert rel_err(got["logits"].cpu().numpy(), ref["s"]) < 1e-5
+        assert rel_err(f64(got["dg"]), ref["dg"]) < tol
+
+
+def test_config1_tiny_fp32_layer(r3):
+    case = Case(synth.WORKLOADS["c1_tiny_fp32"])
+    own = O.topk_indices(case.s, 2)
+    differs = (np.sort(own, axis=1) != np.sort(case.idx_np(), axis=1)).any(axis=1).mean()
+    assert 0.04 < differs < 0.2                        # about 10% of tokens replay another expert
+    ref = case.oracle_layer()
+    check_full(case, run_layer(r3, case, stepwise=True), ref, TOL_F32)
+    check_full(case, run_layer(r3, case), ref, TOL_F32)
+
+
+def test_config1_replay_of_own_topk_is_the_ordinary_layer(r3):
+    """Replaying the record that the library's own capture kernel makes from the training logits
+    reproduces the ordinary MoE layer (Eqs. train_gate / train_output)."""
+    w = synth.WORKLOADS["c1_tiny_fp32"]
+    case = Case(w)
+    s = r3.shape_of(w)
+    c = case.cuda()
+    own, _ = r3.capture_topk(s, c["x"], c["w_r"])
+    assert np.array_equal(own.cpu().numpy().astype(np.int64), O.topk_indices(case.s, w.K))
+    y, _, _ = r3.replay_layer(s, c["x"], c["w_r"], own, c["w_gate"], c["w_up"], c["w_down"],
+                              c["dy"])
+    y_ref = O.train_output(f64(case.x), f64(case.w_r), w.K, f64(case.w_gate), f64(case.w_up),
+                           f64(case.w_down))
+    assert rel_err(f64(y), y_ref) < TOL_F32
+
+
+def test_config2_bf16_layer_full(r3):
+    case = Case(synth.WORKLOADS["c2_layer_bf16"])
+    ref = case.oracle_layer()
+    check_full(case, run_layer(r3, case, stepwise=True), ref, TOL_BF16)
+    got = run_layer(r3, case)
+    check_full(case, got, ref, TOL_BF16)
+    again = run_layer(r3, case)
+    assert torch.equal(got["y"], again["y"]) and torch.equal(got["ds"], again["ds"])
+
+
+def sampled_check(case, got, n_samples, tol, seed=0):
+    """Tokens the oracle evaluates one at a time straight from the equations."""
+    w = case.w
+    rng = np.random.default_rng(seed)
+    sel = np.sort(rng.choice(w.T, size=n_samples, replace=False))
+    y_ref, ds_ref = O.layer_tokens(f64(case.x[sel]), f64(case.w_r), case.idx_np()[sel],
+                                   case.w_gate, case.w_up, case.w_down, f64(case.dy[sel]))
+    y_all, ds_all = f64(got["y"]), f64(got["ds"])
+    assert np.abs(y_all[sel] - y_ref).max() / np.abs(y_ref).max() < tol
+    assert np.abs(ds_all[sel] - ds_ref).max() / np.abs(ds_ref).max() < tol
+
+
+class LazyWeights:
+    """Per-expert float64 view of a stored [E, ...] weight tensor (converted on access)."""
+
+    def __init__(self, t):
+        self.t = t
+
+    def __len__(self):
+        return self.t.shape[0]
+
+    def __getitem__(self, i):
+        return self.t[int(i)].to(torch.float64).numpy()
+
+
+def big_case(w):
+    case = Case(w, device="cuda")
+    case.w_gate, case.w_up, case.w_down = (LazyWeights(t) for t in
+                                           (case.w_gate, case.w_up, case.w_down))
+    return case
+
+
+def run_big(r3, case, raw):
+    s = r3.shape_of(case.w)
+    st = r3.new_status("cuda")
+    c = {k: getattr(case, k).cuda() for k in ("x", "dy", "w_r", "idx")}
+    wg, wu, wd = (t.cuda() for t in raw)
+    _, logits = r3.capture_topk(s, c["x"], c["w_r"], want_idx=False, want_logits=True)
+    g = r3.replay_gate_fwd(s, logits, c["idx"], dev_status=st)
+    counts, offsets, ros, sor, xp = r3.permute(s, c["idx"], c["x"], dev_status=st)
+    o = r3.grouped_swiglu(s, xp, offsets, wg, wu, wd, dev_status=st)
+    y = r3.combine(s, o, ros, g)
+    dg = r3.combine_bwd_gates(s, c["dy"], o, ros)
+    ds = r3.replay_gate_bwd(s, g, dg, c["idx"])
+    y2, ds2, g2 = r3.replay_layer(s, c["x"], c["w_r"], c["idx"], wg, wu, wd, c["dy"],
+                                  dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert torch.equal(y, y2) and torch.equal(ds, ds2) and torch.equal(g, g2)
+    return dict(y=y, ds=ds, g=g, logits=logits, counts=counts, offsets=offsets, ros=ros, sor=sor,
+                xp=xp)
+
+
+def check_big(case, got, tol, n_samples=48):
+    w = case.w
+    counts, offsets, ros, sor = O.permutation(case.idx_np(), w.E)
+    assert np.array_equal(got["counts"].cpu().numpy(), counts)
+    assert np.array_equal(got["offsets"].cpu().numpy(), offsets)
+    assert np.array_equal(got["ros"].cpu().numpy(), ros)
+    assert np.array_equal(got["sor"].cpu().numpy(), sor)
+    assert torch.equal(got["xp"].cpu(), case.x[torch.from_numpy(sor.astype(np.int64)) // w.K])
+    assert rel_err(got["logits"].cpu().numpy(), case.s) < 1e-5
+    assert rel_err(f64(got["g"]), O.replay_gate(case.s, case.idx_np())) < 1e-5
+    sampled_check(case, got, n_samples, tol)
+    return counts
+
+
+def test_config3_skewed_routing_full_size(r3):
+    w = synth.WORKLOADS["c3_skewed"]
+    case = Case(w, device="cuda")
+    raw = (case.w_gate, case.w_up, case.w_down)
+    case.w_gate, case.w_up, case.w_down = (LazyWeights(t) for t in raw)
+    got = run_big(r3, case, raw)
+    counts = check_big(case, got, TOL_BF16)
+    # the Zipf bias really skews the load: a few experts take most rows, some take (almost) none
+    assert counts.max() > 20 * max(1, np.median(counts)) or counts.max() > w.T // 2
+    assert counts.min() < w.T * w.K // w.E // 4
+
+
+def test_config4_capture_then_replay_round_trip(r3):
+    # inference side: 48 layers x 256 decode tokens, bf16 router, uint8 record, one launch
+    wc = synth.WORKLOADS["c4_capture"]
+    L = wc.layers
+    xs = torch.stack([synth.activations(wc, "cpu", l) for l in range(L)])
+    wr = torch.stack([synth.router_weight(wc, "cpu", l) for l in range(L)])
+    s = r3.shape_of(wc)
+    rec, logits = r3.capture_topk_batched(s, L, xs.cuda(), wr.cuda(), want_logits=True)
+    assert rec.dtype == torch.uint8 and rec.shape == (L, wc.T, wc.K)
+    near = 0
+    for l in range(L):
+        ref_s = O.router_logits(f64(xs[l]), f64(wr[l]))
+        assert rel_err(logits[l].cpu().numpy(), ref_s) < 1e-5
+        near += check_record_against_logits(rec[l].cpu().numpy(), ref_s, wc.K)
+    assert near < 0.05 * L * wc.T
+
+    # training side: a recorded 65536-token batch replayed through one layer.  The record is the
+    # library's own capture of that batch; the oracle works from its own TopKMask of the same
+    # inputs, and parity is judged on the tokens where the two records agree bit for bit.
+    wr_ = synth.WORKLOADS["c4_replay"]
+    case = Case(synth.scaled(wr_, record="noise", sigma=0.0), device="cuda")
+    raw = (case.w_gate, case.w_up, case.w_down)
+    case.w_gate, case.w_up, case.w_down = (LazyWeights(t) for t in raw)
+    s2 = r3.shape_of(wr_)
+    xg, wrg = case.x.cuda(), case.w_r.cuda()
+    gpu_rec, _ = r3.capture_topk(s2, xg, wrg)
+    oracle_rec = O.topk_indices(case.s, wr_.K)
+    check_record_against_logits(gpu_rec.cpu().numpy(), case.s, wr_.K)
+    same = (gpu_rec.cpu().numpy().astype(np.int64) == oracle_rec).all(axis=1)
+    assert same.mean() > 0.95
+    st = r3.new_status("cuda")
+    y, ds, g = r3.replay_layer(s2, xg, wrg, gpu_rec, *(t.cuda() for t in raw), case.dy.cuda(),
+                               dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert np.allclose(g.cpu().numpy().sum(axis=1), 1.0, atol=1e-5)
+    rng = np.random.default_rng(1)
+    sel = np.sort(rng.choice(np.nonzero(same)[0], size=32, replace=False))
+    y_ref, ds_ref = O.layer_tokens(f64(case.x[sel]), f64(case.w_r), oracle_rec[sel],
+                                   case.w_gate, case.w_up, case.w_down, f64(case.dy[sel]))
+    assert np.abs(f64(y)[sel] - y_ref).max() / np.abs(y_ref).max() < TOL_BF16
+    assert np.abs(f64(ds)[sel] - ds_ref).max() / np.abs(ds_ref).max() < TOL_BF16
