@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the replayed-routing MoE layer (forward + router-logit backward) on B200.
+
+    python bench.py --gpus 1 --steps 50 --warmup 5                 # this library
+    python bench.py --impl reference --steps 2 --warmup 1          # the CPU oracle, timed
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+
+A step is one pass of the whole path over one synthetic batch: training logits, replay gate,
+permute, grouped SwiGLU experts, combine, dgates, dlogits.  The default workload is the headline
+single bf16 layer (T=4096, d=2048, E=128, K=8, F=768).  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "replayed-MoE-layer tokens/s (fwd+router bwd)"
+UNIT = "tokens/s"
+# kernel launches of one r3_replay_layer call: logits 1, gate 1, permute 4, tile list 1,
+# expert GEMMs 2, combine 1, dgates 1, dlogits 1
+LAUNCHES_PER_STEP = 12
+# DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
+# from the ncu capture summarised in profiles/; None until captured.
+GEMM_UP_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0,
+                source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for (ts, r) in self.rows if t0 - 0.05 <= ts <= t1 + 0.15 and len(r) >= 7]
+        if not rows:
+            rows = [r for (_, r) in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+
+        def num(v):
+            try:
+                return float(v)
+            except ValueError:
+                return None
+        sm = [num(r[0]) for r in rows if num(r[0]) is not None]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower() == "active" for r in rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": num(rows[0][1]), "power_w_max": max((num(r[2]) or 0) for r in rows),
+                "reasons": reasons, "samples": len(rows)}
+
+
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(w, n_tokens, seed_layer=0):
+    """CPU inputs for the first n_tokens of the workload (weights of all experts)."""
+    import torch
+    from paper_2510_11370_b200 import synth
+    from oracle import r3_oracle as O
+    x = synth.activations(w, "cpu", seed_layer)[:n_tokens]
+    dy = synth.upstream_grad(w, "cpu", seed_layer)[:n_tokens]
+    w_r = synth.router_weight(w, "cpu", seed_layer)
+    wg, wu, wd = synth.expert_weights(w, "cpu", seed_layer)
+    f64 = lambda t: t.to(torch.float64).numpy()
+    f32 = lambda t: t.to(torch.float32).numpy()
+    s = O.router_logits(f64(x), f64(w_r))
+    wn = synth.scaled(w, T=n_tokens)
+    idx = synth.make_record(wn, torch.from_numpy(s), seed_layer).to(torch.int64).numpy()
+    return dict(x=f64(x), dy=f64(dy), w_r=f64(w_r), wg=f32(wg), wu=f32(wu), wd=f32(wd), idx=idx)
+
+
+def oracle_step(inp):
+    from oracle import r3_oracle as O
+    return O.layer_fwd_bwd(inp["x"], inp["w_r"], inp["idx"], inp["wg"], inp["wu"], inp["wd"],
+                           inp["dy"])
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle(w, n_tokens, steps, warmup):
+    inp = oracle_sample(w, n_tokens)
+    for _ in range(warmup):
+        oracle_step(inp)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(inp)
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    return n_tokens / dt, dt
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n = min(w.T, args.ref_tokens)
+    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    steps = min(steps, 5)
+    warmup = min(warmup, 1)
+    tps, dt = time_oracle(w, n, steps, warmup)
+    cores = blas_threads()
+    sample = (f"tokens [0,{n}) of {w.name} (all {w.E} experts' weights), whole layer fwd + "
+              f"router-logit bwd in float64 numpy, {steps} timed step(s)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "T": w.T, "d": w.d, "E": w.E, "K": w.K, "F": w.F,
+                   "sample_tokens": n},
+        "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    from paper_2510_11370_b200 import build, dist as r3dist, synth
+    build.build()
+    from paper_2510_11370_b200 import r3
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    rank, world = r3dist.init("nccl")
+    peaks = load_peaks()
+
+    # per-rank synthetic batch (weak scaling: every rank runs the full per-GPU workload)
+    wk = synth.scaled(w, seed=w.seed + rank)
+    s = r3.shape_of(wk)
+    x = synth.activations(wk, dev)
+    dy = synth.upstream_grad(wk, dev)
+    w_r = synth.router_weight(wk, dev)
+    wg, wu, wd = synth.expert_weights(wk, dev)
+    _, logits0 = r3.capture_topk(s, x, w_r, want_idx=False, want_logits=True)
+    idx = synth.make_record(wk, logits0)           # inference-side record emulated from drifted logits
+    del logits0
+    T, K, E, d, F = wk.T, wk.K, wk.E, wk.d, wk.F
+    R = T * K
+    es = 2 if wk.act == "bf16" else 4
+
+    st = r3.new_status(dev)
+    y = torch.empty((T, d), dtype=wk.act_dtype, device=dev)
+    dlogits = torch.empty((T, E), dtype=torch.float32, device=dev)
+    gates = torch.empty((T, K), dtype=torch.float32, device=dev)
+    ws = r3.workspace(r3.replay_layer_workspace_bytes(s), dev)
+
+    def step():
+        r3.replay_layer(s, x, w_r, idx, wg, wu, wd, dy, y=y, dlogits=dlogits, gates=gates, ws=ws,
+                        dev_status=st)
+
+    # ---- whole-path throughput, inputs resident in HBM -----------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r3dist.barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    r3dist.barrier()
+    t_wall1 = time.time()
+    ms_total = r3dist.max_over_ranks(ev0.elapsed_time(ev1), dev)
+    assert st.item() == 0, f"device status {st.item()}"
+    ms_per_step = ms_total / args.steps
+    value = world * T * args.steps / (ms_total * 1e-3)
+
+    # ---- per-kernel segments (same kernels through the per-step entry points, events between) --
+    seg_names = ["logits", "gate_fwd", "permute", "expert_up_swiglu", "expert_down", "combine",
+                 "dgates", "gate_bwd"]
+    logits = torch.empty((T, E), dtype=torch.float32, device=dev)
+    dg = torch.empty((T, K), dtype=torch.float32, device=dev)
+    pout = (torch.empty(E, dtype=torch.int32, device=dev),
+            torch.empty(E + 1, dtype=torch.int32, device=dev),
+            torch.empty((T, K), dtype=torch.int32, device=dev),
+            torch.empty(R, dtype=torch.int32, device=dev),
+            torch.empty((R, d), dtype=wk.act_dtype, device=dev))
+    o = torch.empty((R, d), dtype=wk.act_dtype, device=dev)
+    pws = r3.workspace(r3.permute_workspace_bytes(s), dev)
+    gws = r3.workspace(r3.grouped_swiglu_workspace_bytes(s), dev)
+    seg_steps = min(args.steps, 20)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(seg_names) + 1)]
+           for _ in range(seg_steps)]
+
+    def seg_step(e):
+        e[0].record()
+        r3.capture_topk(s, x, w_r, logits_out=logits, want_idx=False)
+        e[1].record()
+        r3.replay_gate_fwd(s, logits, idx, gates=gates, dev_status=st)
+        e[2].record()
+        r3.permute(s, idx, x, out=pout, ws=pws, dev_status=st)
+        e[3].record()
+        r3.expert_up_swiglu(s, pout[4], pout[1], wg, wu, gws, dev_status=st)
+        e[4].record()
+        r3.expert_down(s, wd, o, gws, dev_status=st)
+        e[5].record()
+        r3.combine(s, o, pout[2], gates, y=y)
+        e[6].record()
+        r3.combine_bwd_gates(s, dy, o, pout[2], dgates=dg)
+        e[7].record()
+        r3.replay_gate_bwd(s, gates, dg, idx, dlogits=dlogits)
+        e[8].record()
+
+    for _ in range(3):
+        seg_step(evs[0])
+    torch.cuda.synchronize()
+    for e in evs:
+        seg_step(e)
+    torch.cuda.synchronize()
+    seg_ms = {n: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs)
+              for i, n in enumerate(seg_names)}
+    algo_bytes = {                                  # algorithmic bytes per call
+        "logits": T * d * es + E * d * (2 if wk.router_w == "bf16" else 4) + T * E * 4,
+        "gate_fwd": T * (E * 4 + K * 1 + K * 4),
+        "permute": T * (K + d * es + K * 8 + K * d * es),
+        "combine": T * (K * d * es + K * 8 + d * es),
+        "dgates": T * (d * es + K * d * es + K * 4 + K * 4),
+        "gate_bwd": T * (K * 9 + E * 4),
+    }
+    flops = {"expert_up_swiglu": 4.0 * R * d * F, "expert_down": 2.0 * R * d * F,
+             "logits": 2.0 * T * d * E}
+    kernels = {}
+    for n in seg_names:
+        ent = {"ms": round(seg_ms[n], 5)}
+        if n in algo_bytes:
+            ent["hbm_gbs"] = round(algo_bytes[n] / (seg_ms[n] * 1e-3) / 1e9, 1)
+            ent["frac_of_measured_hbm"] = round(ent["hbm_gbs"] / peaks["hbm_gbs"], 3)
+        if n in flops:
+            ent["tflops"] = round(flops[n] / (seg_ms[n] * 1e-3) / 1e12, 1)
+        kernels[n] = ent
+
+    # dominant kernel: the up-projection grouped GEMM (4 R d F of the 6 R d F expert FLOPs).
+    # Its events bracket the call, which also holds the one-CTA tile-list kernel (a few us).
+    achieved = flops["expert_up_swiglu"] / (seg_ms["expert_up_swiglu"] * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "grouped_gemm_tc_kernel<0> (gate/up + SwiGLU)",
+                "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": round(achieved / peaks["bf16_tflops"], 4),
+                "peak_kind": f"bf16 matmul burst, {peaks['source']}",
+                "frac_of_sustained": round(achieved / peaks["bf16_tflops_sustained"], 4),
+                "frac_of_nominal_2250": round(achieved / 2250.0, 4),
+                "traffic": GEMM_UP_DRAM_TRAFFIC_BYTES}
+
+    # ---- end to end through the host-buffer entry point -----------------------------------------
+    xh, dyh, idxh = (t.cpu().pin_memory() for t in (x, dy, idx))
+    yh = torch.empty((T, d), dtype=wk.act_dtype).pin_memory()
+    dlh = torch.empty((T, E), dtype=torch.float32).pin_memory()
+    hws = r3.workspace(r3.replay_layer_host_workspace_bytes(s), dev)
+    e2e_steps = min(args.steps, 20)
+    for _ in range(3):
+        r3.replay_layer_host(s, xh, w_r, idxh, wg, wu, wd, dyh, yh, dlh, ws=hws, dev_status=st)
+    r3dist.barrier()
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(e2e_steps):
+        r3.replay_layer_host(s, xh, w_r, idxh, wg, wu, wd, dyh, yh, dlh, ws=hws, dev_status=st)
+    ev1.record()
+    torch.cuda.synchronize()
+    r3dist.barrier()
+    e2e_ms = r3dist.max_over_ranks(ev0.elapsed_time(ev1), dev)
+    assert st.item() == 0
+    assert torch.equal(yh.to(dev), y), "host-buffer path disagrees with the device path"
+    e2e = {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": int(xh.numel() * es + dyh.numel() * es + idxh.numel() * idxh.element_size()),
+           "d2h_bytes_per_step": int(yh.numel() * es + dlh.numel() * 4),
+           "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps}
+
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    # ---- the oracle on this machine's host cores (rank 0, single-GPU runs only) ---------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n = min(wk.T, args.ref_tokens)
+        tps, dt = time_oracle(w, n, 1, 0)
+        cpu_baseline = {"value": tps, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                        "seconds": round(dt, 2),
+                        "sample": f"tokens [0,{n}) of {w.name} (all {w.E} experts' weights), whole "
+                                  f"layer fwd + router-logit bwd, float64 numpy, one pass"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wk.act == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": wk.name, "T": T, "d": d, "E": E, "K": K, "F": F,
+                       "router": "fp32 logits/softmax", "tokens_per_gpu": T,
+                       "l2": "inputs larger than L2: %.2f GB of expert weights stream through "
+                             "the 126 MB L2 every step" % (synth.layer_bytes(wk) / 1e9)},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
+            "kernels": kernels, "peaks": peaks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_layer_bf16")
+    ap.add_argument("--ref-tokens", type=int, default=4096,
+                    help="tokens of the workload the CPU oracle is timed on")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2510_11370_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -130,6 +130,19 @@ r3_status r3_grouped_swiglu(const r3_shape* shape, const void* xp, const int32_t
                             const void* w_gate, const void* w_up, const void* w_down, void* o,
                             void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
 
+/* The two halves of r3_grouped_swiglu as separate calls (same kernels, same workspace), so that a
+ * caller can place other work, or timing events, between them:
+ *   r3_expert_up_swiglu : builds the tile list from offsets and writes h = silu(xp Wg^T)*(xp Wu^T)
+ *                         into the workspace;
+ *   r3_expert_down      : o = h W_down^T, reading h and the tile list that the preceding
+ *                         r3_expert_up_swiglu call left in the SAME workspace.
+ * Expert network E_i of Eq. (replay_output); argument rules as for r3_grouped_swiglu. */
+r3_status r3_expert_up_swiglu(const r3_shape* shape, const void* xp, const int32_t* offsets,
+                              const void* w_gate, const void* w_up, void* workspace,
+                              size_t ws_bytes, int32_t* dev_status, void* stream);
+r3_status r3_expert_down(const r3_shape* shape, const void* w_down, void* o, void* workspace,
+                         size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* Eq. (replay_output): y[t] = sum_{j=0..K-1} gates[t,j] * o[row_of_slot[t,j]], added in slot
  * order in fp32 (no atomics), rounded once to act_dtype.  o [R,d]; y [T,d]. */
 r3_status r3_combine(const r3_shape* shape, const void* o, const int32_t* row_of_slot,

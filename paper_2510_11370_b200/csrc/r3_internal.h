@@ -29,9 +29,12 @@ r3_status launch_build_tiles(const int32_t* offsets, int E, int BM, int32_t* til
 // bf16 grouped SwiGLU on the tcgen05 tensor cores (sm_100a).  `tiles` must have been built with
 // BM = tc_block_m().
 int tc_block_m();
+// phases: bit 0 = gate/up projections + SwiGLU (xp -> h), bit 1 = down projection (h -> o).
+enum { kPhaseUp = 1, kPhaseDown = 2 };
 r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const int32_t* tiles,
                                    const void* w_gate, const void* w_up, const void* w_down,
-                                   void* h, void* o, int32_t* dev_status, cudaStream_t stream);
+                                   void* h, void* o, int32_t* dev_status, int phases,
+                                   cudaStream_t stream);
 
 // Number of SMs of the current device (cached).
 int sm_count();

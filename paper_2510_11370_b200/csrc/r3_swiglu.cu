@@ -142,17 +142,19 @@ simt_grouped_gemm_kernel(const float* __restrict__ A, const float* __restrict__ 
 static r3_status launch_grouped_swiglu_f32(const r3_shape* s, const void* xp, const int32_t* tiles,
                                            const void* w_gate, const void* w_up,
                                            const void* w_down, void* h, void* o,
-                                           cudaStream_t cs) {
+                                           int phases, cudaStream_t cs) {
     const long long R = (long long)s->T * s->K;
     const int mt = max_m_tiles(R, s->E, SBM);
     if (mt == 0) return R3_OK;
     dim3 g1(mt, (s->F + SBN - 1) / SBN), g2(mt, (s->d + SBN - 1) / SBN);
-    simt_grouped_gemm_kernel<true><<<g1, 256, 0, cs>>>(
-        static_cast<const float*>(xp), static_cast<const float*>(w_gate),
-        static_cast<const float*>(w_up), static_cast<float*>(h), tiles, s->d, s->F);
-    simt_grouped_gemm_kernel<false><<<g2, 256, 0, cs>>>(
-        static_cast<const float*>(h), static_cast<const float*>(w_down), nullptr,
-        static_cast<float*>(o), tiles, s->F, s->d);
+    if (phases & kPhaseUp)
+        simt_grouped_gemm_kernel<true><<<g1, 256, 0, cs>>>(
+            static_cast<const float*>(xp), static_cast<const float*>(w_gate),
+            static_cast<const float*>(w_up), static_cast<float*>(h), tiles, s->d, s->F);
+    if (phases & kPhaseDown)
+        simt_grouped_gemm_kernel<false><<<g2, 256, 0, cs>>>(
+            static_cast<const float*>(h), static_cast<const float*>(w_down), nullptr,
+            static_cast<float*>(o), tiles, s->F, s->d);
     return launch_status();
 }
 
@@ -170,29 +172,59 @@ extern "C" size_t r3_grouped_swiglu_workspace_bytes(const r3_shape* shape) {
            r3::round_up(r3::tile_list_bytes(R, shape->E, r3::block_m(shape)), 256);
 }
 
+namespace r3 {
+// Shared body of the three expert entry points.
+static r3_status run_experts(const r3_shape* shape, const void* xp, const int32_t* offsets,
+                             const void* w_gate, const void* w_up, const void* w_down, void* o,
+                             void* workspace, size_t ws_bytes, int32_t* dev_status, int phases,
+                             void* stream) {
+    r3_status st = check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->E > 1024) return R3_ERR_UNSUPPORTED;
+    if (shape->T == 0) return R3_OK;
+    const bool up = phases & kPhaseUp, down = phases & kPhaseDown;
+    if ((up && (!xp || !offsets || !w_gate || !w_up)) || (down && (!w_down || !o)))
+        return R3_ERR_INVALID_ARG;
+    if ((up && (!aligned(xp, 16) || !aligned(w_gate, 16) || !aligned(w_up, 16))) ||
+        (down && (!aligned(o, 16) || !aligned(w_down, 16))))
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || ws_bytes < r3_grouped_swiglu_workspace_bytes(shape) ||
+        !aligned(workspace, 256))
+        return R3_ERR_WORKSPACE;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    void* h = workspace;
+    int32_t* tiles = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + h_bytes(shape));
+    if (up) {
+        st = launch_build_tiles(offsets, shape->E, block_m(shape), tiles, cs);
+        if (st != R3_OK) return st;
+    }
+    if (shape->act_dtype == R3_BF16)
+        return launch_grouped_swiglu_tc(shape, xp, tiles, w_gate, w_up, w_down, h, o, dev_status,
+                                        phases, cs);
+    return launch_grouped_swiglu_f32(shape, xp, tiles, w_gate, w_up, w_down, h, o, phases, cs);
+}
+}  // namespace r3
+
 extern "C" r3_status r3_grouped_swiglu(const r3_shape* shape, const void* xp,
                                        const int32_t* offsets, const void* w_gate,
                                        const void* w_up, const void* w_down, void* o,
                                        void* workspace, size_t ws_bytes, int32_t* dev_status,
                                        void* stream) {
-    r3_status st = r3::check_shape(shape);
-    if (st != R3_OK) return st;
-    if (shape->E > 1024) return R3_ERR_UNSUPPORTED;
-    if (shape->T == 0) return R3_OK;
-    if (!xp || !offsets || !w_gate || !w_up || !w_down || !o) return R3_ERR_INVALID_ARG;
-    if (!r3::aligned(xp, 16) || !r3::aligned(o, 16) || !r3::aligned(w_gate, 16) ||
-        !r3::aligned(w_up, 16) || !r3::aligned(w_down, 16))
-        return R3_ERR_INVALID_ARG;
-    if (!workspace || ws_bytes < r3_grouped_swiglu_workspace_bytes(shape) ||
-        !r3::aligned(workspace, 256))
-        return R3_ERR_WORKSPACE;
-    cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    void* h = workspace;
-    int32_t* tiles = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + r3::h_bytes(shape));
-    st = r3::launch_build_tiles(offsets, shape->E, r3::block_m(shape), tiles, cs);
-    if (st != R3_OK) return st;
-    if (shape->act_dtype == R3_BF16)
-        return r3::launch_grouped_swiglu_tc(shape, xp, tiles, w_gate, w_up, w_down, h, o,
-                                            dev_status, cs);
-    return r3::launch_grouped_swiglu_f32(shape, xp, tiles, w_gate, w_up, w_down, h, o, cs);
+    return r3::run_experts(shape, xp, offsets, w_gate, w_up, w_down, o, workspace, ws_bytes,
+                           dev_status, r3::kPhaseUp | r3::kPhaseDown, stream);
+}
+
+extern "C" r3_status r3_expert_up_swiglu(const r3_shape* shape, const void* xp,
+                                         const int32_t* offsets, const void* w_gate,
+                                         const void* w_up, void* workspace, size_t ws_bytes,
+                                         int32_t* dev_status, void* stream) {
+    return r3::run_experts(shape, xp, offsets, w_gate, w_up, nullptr, nullptr, workspace,
+                           ws_bytes, dev_status, r3::kPhaseUp, stream);
+}
+
+extern "C" r3_status r3_expert_down(const r3_shape* shape, const void* w_down, void* o,
+                                    void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                    void* stream) {
+    return r3::run_experts(shape, nullptr, nullptr, nullptr, nullptr, w_down, o, workspace,
+                           ws_bytes, dev_status, r3::kPhaseDown, stream);
 }

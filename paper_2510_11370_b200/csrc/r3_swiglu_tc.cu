@@ -377,7 +377,8 @@ int tc_block_m() { return tc::BM; }
 
 r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int32_t* tiles,
                                    const void* w_gate, const void* w_up, const void* w_down,
-                                   void* h, void* o, int32_t* dev_status, cudaStream_t cs) {
+                                   void* h, void* o, int32_t* dev_status, int phases,
+                                   cudaStream_t cs) {
     using namespace tc;
     const long long R = (long long)s->T * s->K;
     const int mt = max_m_tiles(R, s->E, BM);
@@ -391,22 +392,30 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int3
             return R3_ERR_CUDA;
         attr_set = true;
     }
-    CUtensorMap m_xp, m_g, m_u, m_h, m_d;
-    if (!make_map_2d(&m_xp, xp, (uint64_t)R, (uint64_t)s->d, BM) ||
-        !make_map_3d(&m_g, w_gate, s->E, s->F, s->d, BN / 2) ||
-        !make_map_3d(&m_u, w_up, s->E, s->F, s->d, BN / 2) ||
-        !make_map_2d(&m_h, h, (uint64_t)R, (uint64_t)s->F, BM) ||
-        !make_map_3d(&m_d, w_down, s->E, s->d, s->F, BN))
-        return R3_ERR_CUDA;
-    const int nb1 = (s->F + BN / 2 - 1) / (BN / 2);
-    const int nb2 = (s->d + BN - 1) / BN;
     const int sms = sm_count();
-    const long long t1 = (long long)mt * nb1, t2 = (long long)mt * nb2;
-    const int g1 = (int)(t1 < sms ? t1 : sms), g2 = (int)(t2 < sms ? t2 : sms);
-    grouped_gemm_tc_kernel<0><<<g1, THREADS, SMEM_BYTES, cs>>>(
-        m_xp, m_g, m_u, tiles, static_cast<__nv_bfloat16*>(h), s->d, s->F, nb1, dev_status);
-    grouped_gemm_tc_kernel<1><<<g2, THREADS, SMEM_BYTES, cs>>>(
-        m_h, m_d, m_d, tiles, static_cast<__nv_bfloat16*>(o), s->F, s->d, nb2, dev_status);
+    if (phases & kPhaseUp) {
+        CUtensorMap m_xp, m_g, m_u;
+        if (!make_map_2d(&m_xp, xp, (uint64_t)R, (uint64_t)s->d, BM) ||
+            !make_map_3d(&m_g, w_gate, s->E, s->F, s->d, BN / 2) ||
+            !make_map_3d(&m_u, w_up, s->E, s->F, s->d, BN / 2))
+            return R3_ERR_CUDA;
+        const int nb1 = (s->F + BN / 2 - 1) / (BN / 2);
+        const long long t1 = (long long)mt * nb1;
+        const int g1 = (int)(t1 < sms ? t1 : sms);
+        grouped_gemm_tc_kernel<0><<<g1, THREADS, SMEM_BYTES, cs>>>(
+            m_xp, m_g, m_u, tiles, static_cast<__nv_bfloat16*>(h), s->d, s->F, nb1, dev_status);
+    }
+    if (phases & kPhaseDown) {
+        CUtensorMap m_h, m_d;
+        if (!make_map_2d(&m_h, h, (uint64_t)R, (uint64_t)s->F, BM) ||
+            !make_map_3d(&m_d, w_down, s->E, s->d, s->F, BN))
+            return R3_ERR_CUDA;
+        const int nb2 = (s->d + BN - 1) / BN;
+        const long long t2 = (long long)mt * nb2;
+        const int g2 = (int)(t2 < sms ? t2 : sms);
+        grouped_gemm_tc_kernel<1><<<g2, THREADS, SMEM_BYTES, cs>>>(
+            m_h, m_d, m_d, tiles, static_cast<__nv_bfloat16*>(o), s->F, s->d, nb2, dev_status);
+    }
     return launch_status();
 }
 

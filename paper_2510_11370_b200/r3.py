@@ -26,7 +26,8 @@ DEV_OK, DEV_BAD_INDEX, DEV_DUP_INDEX, DEV_TIMEOUT = 0, 1, 2, 3
 EXPORTS = [
     "r3_status_string", "r3_capture_topk", "r3_capture_topk_batched", "r3_replay_gate_fwd",
     "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute",
-    "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_combine",
+    "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_expert_up_swiglu",
+    "r3_expert_down", "r3_combine",
     "r3_combine_bwd_gates", "r3_replay_layer_workspace_bytes", "r3_replay_layer",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
 ]
@@ -52,6 +53,8 @@ lib.r3_replay_gate_fwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_gate_bwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_permute.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_grouped_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
+lib.r3_expert_up_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
+lib.r3_expert_down.argtypes = [_SP, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_combine.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
@@ -211,6 +214,20 @@ def grouped_swiglu(s: Shape, xp, offsets, w_gate, w_up, w_down, o=None, *, ws=No
     _check(lib.r3_grouped_swiglu(ctypes.byref(s), _ptr(xp), _ptr(offsets), _ptr(w_gate),
                                  _ptr(w_up), _ptr(w_down), _ptr(o), _ptr(ws), ws.numel(),
                                  _ptr(dev_status), _stream(stream)))
+    return o
+
+
+def expert_up_swiglu(s: Shape, xp, offsets, w_gate, w_up, ws, dev_status=None, stream=None):
+    """First half of grouped_swiglu: tile list + h = silu(xp Wg^T) * (xp Wu^T) into `ws`."""
+    _check(lib.r3_expert_up_swiglu(ctypes.byref(s), _ptr(xp), _ptr(offsets), _ptr(w_gate),
+                                   _ptr(w_up), _ptr(ws), ws.numel(), _ptr(dev_status),
+                                   _stream(stream)))
+
+
+def expert_down(s: Shape, w_down, o, ws, dev_status=None, stream=None):
+    """Second half of grouped_swiglu: o = h W_down^T with h taken from `ws`."""
+    _check(lib.r3_expert_down(ctypes.byref(s), _ptr(w_down), _ptr(o), _ptr(ws), ws.numel(),
+                              _ptr(dev_status), _stream(stream)))
     return o
 
 
