@@ -54,7 +54,8 @@ typedef enum {
     R3_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, K > E, index type too narrow */
     R3_ERR_UNSUPPORTED = 2,   /* a legal shape this build has no kernel for */
     R3_ERR_WORKSPACE = 3,     /* workspace missing, too small or misaligned */
-    R3_ERR_CUDA = 4           /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+    R3_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+    R3_ERR_SCRATCH_LIMIT = 5  /* the problem needs more than the library's fixed on-device scratch */
 } r3_status;
 
 enum { R3_F32 = 0, R3_BF16 = 1 };
@@ -117,6 +118,26 @@ size_t r3_permute_workspace_bytes(const r3_shape* shape);
 r3_status r3_permute(const r3_shape* shape, const void* idx, const void* x, int32_t* counts,
                      int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* xp,
                      void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* r3_permute without a caller-supplied workspace (the paper has no counterpart; this exists for
+ * the integration, not for the method).  Meant for callers that cannot allocate device memory at
+ * the point of the call: for example a host process whose whole device-memory budget belongs to
+ * another component's pool, where a fresh driver allocation may fail or stall the device, or a
+ * step whose memory plan was fixed in advance.  The scratch (per-expert, per-256-token-chunk
+ * counters) lives in a fixed array inside the library, 1 MiB on every GPU that loads the library,
+ * held until the process exits.  Inputs and outputs are the caller's, exactly as for r3_permute,
+ * and the results are identical to r3_permute's.
+ *  - Limit: E * ceil(T / 256) <= 262144 (e.g. E = 128 up to T = 524288); beyond it the call
+ *    returns R3_ERR_SCRATCH_LIMIT and launches nothing.  E <= 1024 as for r3_permute.
+ *  - The call itself allocates and frees nothing, on the host or on the device.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current) and caches it; make that first call outside any stream capture.
+ *  - Every call uses the same array, and it keeps the previous call's contents (no part of it
+ *    has to be cleared: each call overwrites all the counters it later reads).  Calls that may
+ *    overlap on the GPU - different streams or host threads - race on it; serialise them. */
+r3_status r3_permute_static(const r3_shape* shape, const void* idx, const void* x, int32_t* counts,
+                            int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row,
+                            void* xp, int32_t* dev_status, void* stream);
 
 /* Expert networks E_i on the grouped rows: for expert e and rows r in [offsets[e], offsets[e+1])
  *   h[r] = silu(xp[r] W_gate,e^T) * (xp[r] W_up,e^T);   o[r] = h[r] W_down,e^T.

@@ -220,3 +220,54 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
     }
     return r3::launch_status();
 }
+
+// ---------------------------------------------------------------------------------------------
+// r3_permute_static: the same dispatch with its scratch in a fixed device array of this library.
+//
+// For callers that have no way to hand over scratch memory: a host whose device memory is owned
+// entirely by another component's pool (asking the driver for more would fail, fragment the pool
+// or stall the device, since a driver allocation synchronises it), or a step that must not touch
+// the allocator because its memory budget was fixed up front.  They still pass inputs and outputs;
+// only the [expert][chunk] counters live here.
+//
+// The array is part of the loaded library image: every GPU that loads the library carries these
+// kStaticScratchInts * 4 bytes until the process exits.  All calls share it and it keeps whatever
+// the last call left; nothing in it needs to start at zero because the counting kernel overwrites
+// every counter the later kernels read.  Two calls that overlap on the GPU (different streams, or
+// different host threads) would race on it.
+// ---------------------------------------------------------------------------------------------
+namespace r3 {
+constexpr int kStaticScratchInts = 1 << 18;            // 1 MiB: E * ceil(T / 256) <= 262144
+static __device__ __align__(256) int32_t g_permute_scratch[kStaticScratchInts];
+
+// In host code the array's name only stands for the symbol; the device address has to be asked
+// for, per device, with that device current.  Cached after the first call on each device.
+static r3_status static_scratch_ptr(int32_t** out) {
+    constexpr int kMaxDevices = 64;
+    static int32_t* cached[kMaxDevices] = {nullptr};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return R3_ERR_CUDA;
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_permute_scratch) != cudaSuccess || !p) return R3_ERR_CUDA;
+        cached[dev] = static_cast<int32_t*>(p);
+    }
+    *out = cached[dev];
+    return R3_OK;
+}
+}  // namespace r3
+
+extern "C" r3_status r3_permute_static(const r3_shape* shape, const void* idx, const void* x,
+                                       int32_t* counts, int32_t* offsets, int32_t* row_of_slot,
+                                       int32_t* slot_of_row, void* xp, int32_t* dev_status,
+                                       void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->E > r3::kMaxExpertsPermute) return R3_ERR_UNSUPPORTED;
+    const long long NB = ((long long)shape->T + r3::kChunk - 1) / r3::kChunk;
+    if ((long long)shape->E * NB > r3::kStaticScratchInts) return R3_ERR_SCRATCH_LIMIT;
+    int32_t* scratch = nullptr;
+    if ((st = r3::static_scratch_ptr(&scratch)) != R3_OK) return st;
+    return r3_permute(shape, idx, x, counts, offsets, row_of_slot, slot_of_row, xp, scratch,
+                      sizeof(int32_t) * r3::kStaticScratchInts, dev_status, stream);
+}

@@ -19,13 +19,14 @@ if not os.path.exists(_LIB_PATH):
 lib = ctypes.CDLL(_LIB_PATH)
 
 R3_OK = 0
+R3_ERR_SCRATCH_LIMIT = 5
 R3_F32, R3_BF16 = 0, 1
 R3_IDX_U8, R3_IDX_I16 = 1, 2
 DEV_OK, DEV_BAD_INDEX, DEV_DUP_INDEX, DEV_TIMEOUT = 0, 1, 2, 3
 
 EXPORTS = [
     "r3_status_string", "r3_capture_topk", "r3_capture_topk_batched", "r3_replay_gate_fwd",
-    "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute",
+    "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute", "r3_permute_static",
     "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_expert_up_swiglu",
     "r3_expert_down", "r3_combine",
     "r3_combine_bwd_gates", "r3_replay_layer_workspace_bytes", "r3_replay_layer",
@@ -52,6 +53,7 @@ lib.r3_capture_topk_batched.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P]
 lib.r3_replay_gate_fwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_gate_bwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_permute.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
+lib.r3_permute_static.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, _P]
 lib.r3_grouped_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_expert_up_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_expert_down.argtypes = [_SP, _P, _P, _P, ctypes.c_size_t, _P, _P]
@@ -198,6 +200,18 @@ def permute(s: Shape, idx, x=None, *, out=None, ws=None, dev_status=None, stream
                           _ptr(ros), _ptr(sor), _ptr(xp), _ptr(ws), ws.numel(),
                           _ptr(dev_status), _stream(stream)))
     return counts, offsets, ros, sor, xp
+
+
+def permute_static(s: Shape, idx, x, counts, offsets, row_of_slot, slot_of_row, xp, *,
+                   dev_status=None, stream=None):
+    """r3_permute with the scratch inside the library: for callers that cannot allocate device
+    memory where they call from (their memory belongs to someone else's pool, or was budgeted
+    ahead of time).  All outputs are passed in; nothing is allocated here either.  Raises
+    R3Error(R3_ERR_SCRATCH_LIMIT) when E * ceil(T / 256) > 262144.  Do not overlap calls."""
+    _check(lib.r3_permute_static(ctypes.byref(s), _ptr(idx), _ptr(x), _ptr(counts),
+                                 _ptr(offsets), _ptr(row_of_slot), _ptr(slot_of_row), _ptr(xp),
+                                 _ptr(dev_status), _stream(stream)))
+    return counts, offsets, row_of_slot, slot_of_row, xp
 
 
 def grouped_swiglu_workspace_bytes(s: Shape) -> int:
