@@ -26,9 +26,9 @@ if ROOT not in sys.path:
 
 METRIC = "replayed-MoE-layer tokens/s (fwd+router bwd)"
 UNIT = "tokens/s"
-# kernel launches of one r3_replay_layer call: logits 1, gate 1, permute 4, tile list 1,
-# expert GEMMs 2, combine 1, dgates 1, dlogits 1
-LAUNCHES_PER_STEP = 12
+# kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, gate 1, permute 4,
+# tile list 1, expert GEMMs 2, combine 1, dgates 1, dlogits 1
+LAUNCHES_PER_STEP = 13
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
 # from the ncu capture summarised in profiles/; None until captured.
 GEMM_UP_DRAM_TRAFFIC_BYTES = 993.5e6   # 947.5 MB read + 46.0 MB written
@@ -196,7 +196,7 @@ def run_ours(args, w):
     dy = synth.upstream_grad(wk, dev)
     w_r = synth.router_weight(wk, dev)
     wg, wu, wd = synth.expert_weights(wk, dev)
-    _, logits0 = r3.capture_topk(s, x, w_r, want_idx=False, want_logits=True)
+    _, logits0 = r3.capture_topk_ws(s, 1, x, w_r, want_idx=False, want_logits=True)
     idx = synth.make_record(wk, logits0)           # inference-side record emulated from drifted logits
     del logits0
     T, K, E, d, F = wk.T, wk.K, wk.E, wk.d, wk.F
@@ -250,13 +250,14 @@ def run_ours(args, w):
     o = torch.empty((R, d), dtype=wk.act_dtype, device=dev)
     pws = r3.workspace(r3.permute_workspace_bytes(s), dev)
     gws = r3.workspace(r3.grouped_swiglu_workspace_bytes(s), dev)
+    rws = r3.workspace(r3.capture_topk_workspace_bytes(s, 1), dev)
     seg_steps = min(args.steps, 20)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(seg_names) + 1)]
            for _ in range(seg_steps)]
 
     def seg_step(e):
         e[0].record()
-        r3.capture_topk(s, x, w_r, logits_out=logits, want_idx=False)
+        r3.capture_topk_ws(s, 1, x, w_r, logits_out=logits, want_idx=False, ws=rws)
         e[1].record()
         r3.replay_gate_fwd(s, logits, idx, gates=gates, dev_status=st)
         e[2].record()

@@ -79,7 +79,8 @@ const char* r3_status_string(r3_status s);
  * x [T,d] act_dtype; w_router [E,d] router_w_dtype; idx_out [T,K] idx_type (may be NULL when only
  * logits are wanted); logits_out [T,E] float32 or NULL.  At least one output must be non-NULL.
  * Used on the inference side to make the record, and on the training side (logits_out set) for
- * s_train.  Supported: E <= 512. */
+ * s_train.  bf16 activations with bf16 router weights (E a multiple of 16 up to 256, K <= 16)
+ * run on the tensor cores; other combinations use a float32 FMA kernel (E <= 512). */
 r3_status r3_capture_topk(const r3_shape* shape, const void* x, const void* w_router,
                           void* idx_out, float* logits_out, void* stream);
 
@@ -88,6 +89,18 @@ r3_status r3_capture_topk(const r3_shape* shape, const void* x, const void* w_ro
 r3_status r3_capture_topk_batched(const r3_shape* shape, int32_t L, const void* x,
                                   const void* w_router, void* idx_out, float* logits_out,
                                   void* stream);
+
+/* The same with caller scratch, which lets float32 router weights use the tensor cores too: the
+ * weights are split into three bf16 planes (hi + mid + lo = all 24 mantissa bits) in the
+ * workspace and the three products are accumulated in fp32, so the logits keep float32-level
+ * accuracy.  workspace: r3_capture_topk_workspace_bytes(shape, L) bytes (0 when none is needed:
+ * bf16 router weights, or a shape the tensor-core kernel does not cover).  Without a workspace
+ * (or through r3_capture_topk / _batched) float32 router weights take the float32 FMA kernel.
+ * Tensor-core kernel: bf16 activations, E a multiple of 16 up to 256, K <= 16. */
+size_t r3_capture_topk_workspace_bytes(const r3_shape* shape, int32_t L);
+r3_status r3_capture_topk_ws(const r3_shape* shape, int32_t L, const void* x,
+                             const void* w_router, void* idx_out, float* logits_out,
+                             void* workspace, size_t ws_bytes, void* stream);
 
 /* Eq. (replay_gate): softmax of the TRAINING logits over the K RECORDED experts.
  *   gates[t,j] = exp(s[t,e_j] - m) / sum_j' exp(s[t,e_j'] - m),  e_j = idx[t,j], m = max_j s[t,e_j]

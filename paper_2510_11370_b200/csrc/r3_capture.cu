@@ -6,6 +6,7 @@
 // widened exactly), keeps that tile in shared memory, optionally streams it out, and selects the
 // top K of each row with warp-wide argmax rounds.
 #include "r3_common.cuh"
+#include "r3_internal.h"
 
 namespace r3 {
 
@@ -151,21 +152,50 @@ static r3_status capture_dispatch(const r3_shape* s, int L, const void* x, const
 
 }  // namespace r3
 
+namespace r3 {
+// Shared body: tensor-core kernel when the shape allows it (and, for float32 router weights, when
+// the caller supplied scratch for the bf16 planes), otherwise the float32 FMA kernel.
+static r3_status capture_any(const r3_shape* shape, int32_t L, const void* x, const void* w_router,
+                             void* idx_out, float* logits_out, void* workspace, size_t ws_bytes,
+                             void* stream) {
+    r3_status st = check_shape(shape);
+    if (st != R3_OK) return st;
+    if (L < 0 || L > 65535) return R3_ERR_INVALID_ARG;
+    if (shape->T == 0 || L == 0) return R3_OK;
+    if (!x || !w_router || (!idx_out && !logits_out)) return R3_ERR_INVALID_ARG;
+    if (!aligned(x, 16) || !aligned(w_router, 16)) return R3_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (router_tc_supported(shape)) {
+        const size_t need = router_tc_workspace_bytes(shape, L);
+        if (need == 0) return launch_router_tc(shape, L, x, w_router, idx_out, logits_out, nullptr, cs);
+        if (workspace) {
+            if (ws_bytes < need || !aligned(workspace, 256)) return R3_ERR_WORKSPACE;
+            return launch_router_tc(shape, L, x, w_router, idx_out, logits_out, workspace, cs);
+        }
+    }
+    if (shape->E > kMaxExpertsCapture) return R3_ERR_UNSUPPORTED;
+    return capture_dispatch(shape, L, x, w_router, idx_out, logits_out, cs);
+}
+}  // namespace r3
+
+extern "C" size_t r3_capture_topk_workspace_bytes(const r3_shape* shape, int32_t L) {
+    if (r3::check_shape(shape) != R3_OK || L <= 0) return 0;
+    return r3::router_tc_workspace_bytes(shape, L);
+}
+
+extern "C" r3_status r3_capture_topk_ws(const r3_shape* shape, int32_t L, const void* x,
+                                        const void* w_router, void* idx_out, float* logits_out,
+                                        void* workspace, size_t ws_bytes, void* stream) {
+    return r3::capture_any(shape, L, x, w_router, idx_out, logits_out, workspace, ws_bytes, stream);
+}
+
 extern "C" r3_status r3_capture_topk_batched(const r3_shape* shape, int32_t L, const void* x,
                                              const void* w_router, void* idx_out,
                                              float* logits_out, void* stream) {
-    r3_status st = r3::check_shape(shape);
-    if (st != R3_OK) return st;
-    if (L < 0 || L > 65535) return R3_ERR_INVALID_ARG;
-    if (shape->E > r3::kMaxExpertsCapture) return R3_ERR_UNSUPPORTED;
-    if (shape->T == 0 || L == 0) return R3_OK;
-    if (!x || !w_router || (!idx_out && !logits_out)) return R3_ERR_INVALID_ARG;
-    if (!r3::aligned(x, 16) || !r3::aligned(w_router, 16)) return R3_ERR_INVALID_ARG;
-    return r3::capture_dispatch(shape, L, x, w_router, idx_out, logits_out,
-                                static_cast<cudaStream_t>(stream));
+    return r3::capture_any(shape, L, x, w_router, idx_out, logits_out, nullptr, 0, stream);
 }
 
 extern "C" r3_status r3_capture_topk(const r3_shape* shape, const void* x, const void* w_router,
                                      void* idx_out, float* logits_out, void* stream) {
-    return r3_capture_topk_batched(shape, 1, x, w_router, idx_out, logits_out, stream);
+    return r3::capture_any(shape, 1, x, w_router, idx_out, logits_out, nullptr, 0, stream);
 }

@@ -36,6 +36,14 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const 
                                    void* h, void* o, int32_t* dev_status, int phases,
                                    cudaStream_t stream);
 
+// Router logits + top-K on the tensor cores (bf16 activations, E a multiple of 16 up to 256,
+// K <= 16).  float32 router weights need router_tc_workspace_bytes() of scratch for their three
+// bf16 planes; bf16 router weights need none.
+bool router_tc_supported(const r3_shape* shape);
+size_t router_tc_workspace_bytes(const r3_shape* shape, int L);
+r3_status launch_router_tc(const r3_shape* shape, int L, const void* x, const void* w_router,
+                           void* idx_out, float* logits_out, void* workspace, cudaStream_t stream);
+
 // Number of SMs of the current device (cached).
 int sm_count();
 

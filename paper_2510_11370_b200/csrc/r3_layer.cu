@@ -19,6 +19,8 @@ struct LayerWs {
     size_t permute_bytes;
     void* swiglu_ws;
     size_t swiglu_bytes;
+    void* router_ws;
+    size_t router_bytes;
     size_t total;
 };
 
@@ -46,6 +48,8 @@ static LayerWs carve(const r3_shape* s, void* base) {
     w.permute_ws = take(w.permute_bytes);
     w.swiglu_bytes = r3_grouped_swiglu_workspace_bytes(s);
     w.swiglu_ws = take(w.swiglu_bytes);
+    w.router_bytes = r3_capture_topk_workspace_bytes(s, 1);
+    w.router_ws = w.router_bytes ? take(w.router_bytes) : nullptr;
     w.total = off;
     return w;
 }
@@ -74,7 +78,9 @@ extern "C" r3_status r3_replay_layer(const r3_shape* shape, const void* x, const
     float* gates = gates_out ? gates_out : w.gates;
 
     // s_train = x W_r (only the logits are needed on the training side)
-    if ((st = r3_capture_topk(shape, x, w_router, nullptr, w.logits, stream)) != R3_OK) return st;
+    if ((st = r3_capture_topk_ws(shape, 1, x, w_router, nullptr, w.logits, w.router_ws,
+                                 w.router_bytes, stream)) != R3_OK)
+        return st;
     if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
         return st;
     if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,

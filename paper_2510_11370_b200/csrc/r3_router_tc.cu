@@ -1,0 +1,242 @@
+// Router logits + TopKMask on the tcgen05 tensor cores (Section 4.1, first two equations), for
+// bf16 activations.
+//
+//   s[t, i] = sum_c x[t, c] W_r[i, c]
+//
+// bf16 router weights are used as they are (one MMA pass).  float32 router weights are first
+// split into three bf16 planes  w = hi + mid + lo  (hi = bf16(w), mid = bf16(w - hi),
+// lo = bf16(w - hi - mid); 24 mantissa bits in all), and the three products are accumulated into
+// the same fp32 TMEM accumulator: x is exact in bf16, so the logits keep float32-level accuracy
+// while the contraction runs on the tensor pipe.
+//
+// One CTA per 128-token tile: warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer, warps 2-5
+// = epilogue.  Each epilogue thread owns one token: it streams its E logits out of TMEM 32 at a
+// time, writes them (optionally) to logits_out and keeps a sorted top-K list in registers
+// (strict comparisons in ascending expert order, so exact ties keep the lower index first).
+#include "r3_common.cuh"
+#include "r3_internal.h"
+#include "r3_tc.cuh"
+
+namespace r3 {
+namespace rt {
+
+using namespace tc;
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int UK = 16;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int THREADS = 6 * 32;
+constexpr int BAR_BYTES = 256;
+constexpr int MAX_STAGES = 4;
+constexpr int KMAX = 16;                 // longest record the register top-K list supports
+constexpr int SMEM_LIMIT = 227 * 1024;
+
+__global__ void __launch_bounds__(256)
+split_router_weight_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ planes,
+                           long long per_layer, long long total) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const long long l = i / per_layer, r = i - l * per_layer;
+    const float v = w[i];
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    __nv_bfloat16* base = planes + l * 3 * per_layer + r;
+    base[0] = hi;
+    base[per_layer] = mid;
+    base[2 * per_layer] = lo;
+}
+
+template <typename IdxT, int KM>
+__global__ void __launch_bounds__(THREADS, 1)
+router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                 IdxT* __restrict__ idx_out, float* __restrict__ logits_out, int T, int d, int E,
+                 int K, int planes, int stages, uint32_t tmem_cols) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const int b_bytes = planes * E * BK * 2;
+    const int stage_bytes = A_BYTES + b_bytes;
+    const uint32_t bar0 = base + stages * stage_bytes;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
+    const uint32_t acc_bar = bar0 + 8u * (2 * MAX_STAGES);
+    volatile uint32_t* tmem_slot =
+        reinterpret_cast<volatile uint32_t*>(base_ptr + stages * stage_bytes + 128);
+    volatile int* abort_flag =
+        reinterpret_cast<volatile int*>(base_ptr + stages * stage_bytes + 132);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int layer = blockIdx.y;
+    const int t0 = blockIdx.x * BM;
+    const int kblocks = (d + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(acc_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, nullptr)) break;
+                const uint32_t sa = base + stage * stage_bytes, sb = sa + A_BYTES;
+                mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
+                tma_load_2d(sa, &tmX, kb * BK, layer * T + t0, full_bar(stage));
+                for (int p = 0; p < planes; ++p)
+                    tma_load_2d(sb + p * E * BK * 2, &tmW, kb * BK, (layer * planes + p) * E,
+                                full_bar(stage));
+                if (++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc_bf16(BM, E);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                if (!mbar_wait(full_bar(stage), phase, abort_flag, nullptr)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = base + stage * stage_bytes, sb = sa + A_BYTES;
+                const uint64_t da = smem_desc_sw128(sa);
+                for (int p = 0; p < planes; ++p) {
+                    const uint64_t db = smem_desc_sw128(sb + p * E * BK * 2);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UK; ++kk)
+                        tc_mma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
+                                    idesc, (kb | p | kk) != 0 ? 1u : 0u);
+                }
+                tc_commit(empty_bar(stage));
+                if (++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) tc_commit(acc_bar);
+        }
+    } else {
+        const int q = warp & 3;
+        const int r_in = q * 32 + lane;
+        const int t = t0 + r_in;
+        const bool row_ok = t < T;
+        if (mbar_wait(acc_bar, 0u, abort_flag, nullptr)) {
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+            float tv[KM];
+            int ti[KM];
+#pragma unroll
+            for (int j = 0; j < KM; ++j) { tv[j] = -INFINITY; ti[j] = 0; }
+            float* lrow = logits_out ? logits_out + ((size_t)layer * T + (row_ok ? t : 0)) * E
+                                     : nullptr;
+            for (int c = 0; c < E; c += 32) {
+                float v[32];
+                tc_ld32(taddr + c, v);
+                tc_wait_ld();
+                if (lrow && row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        if (c + i < E)
+                            *reinterpret_cast<float4*>(lrow + c + i) =
+                                make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                }
+                if (idx_out) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (c + i < E && v[i] > tv[KM - 1]) {
+                            tv[KM - 1] = v[i];
+                            ti[KM - 1] = c + i;
+#pragma unroll
+                            for (int j = KM - 1; j > 0; --j) {
+                                if (tv[j] > tv[j - 1]) {
+                                    const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
+                                    const int iv = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = iv;
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            if (idx_out && row_ok) {
+                IdxT* rec = idx_out + ((size_t)layer * T + t) * K;
+#pragma unroll
+                for (int j = 0; j < KM; ++j)
+                    if (j < K) rec[j] = (IdxT)ti[j];
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+}  // namespace rt
+
+bool router_tc_supported(const r3_shape* s) {
+    return s->act_dtype == R3_BF16 && s->E % 16 == 0 && s->E >= 16 && s->E <= 256 &&
+           s->K <= rt::KMAX;
+}
+
+size_t router_tc_workspace_bytes(const r3_shape* s, int L) {
+    if (!router_tc_supported(s) || s->router_w_dtype == R3_BF16) return 0;
+    return round_up((size_t)L * 3 * s->E * s->d * sizeof(__nv_bfloat16), 256);
+}
+
+r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* w_router,
+                           void* idx_out, float* logits_out, void* workspace, cudaStream_t cs) {
+    using namespace rt;
+    const int planes = s->router_w_dtype == R3_BF16 ? 1 : 3;
+    const void* wplanes = w_router;
+    if (planes == 3) {
+        const long long per_layer = (long long)s->E * s->d, total = per_layer * L;
+        split_router_weight_kernel<<<(unsigned)((total + 255) / 256), 256, 0, cs>>>(
+            static_cast<const float*>(w_router), static_cast<__nv_bfloat16*>(workspace), per_layer,
+            total);
+        wplanes = workspace;
+    }
+    const int stage_bytes = A_BYTES + planes * s->E * BK * 2;
+    int stages = (SMEM_LIMIT - BAR_BYTES - 1024) / stage_bytes;
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    if (stages < 2) return R3_ERR_UNSUPPORTED;
+    const int smem = stages * stage_bytes + BAR_BYTES + 1024;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < s->E) tmem_cols <<= 1;
+
+    CUtensorMap mx, mw;
+    if (!make_map_2d(&mx, x, (uint64_t)L * s->T, (uint64_t)s->d, BM) ||
+        !make_map_2d(&mw, wplanes, (uint64_t)L * planes * s->E, (uint64_t)s->d, (uint32_t)s->E))
+        return R3_ERR_CUDA;
+    dim3 grid((s->T + BM - 1) / BM, L);
+#define R3_RT(IDX, KM)                                                                          \
+    do {                                                                                        \
+        auto kern = router_tc_kernel<IDX, KM>;                                                  \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=    \
+            cudaSuccess)                                                                        \
+            return R3_ERR_CUDA;                                                                 \
+        kern<<<grid, THREADS, smem, cs>>>(mx, mw, static_cast<IDX*>(idx_out), logits_out, s->T, \
+                                          s->d, s->E, s->K, planes, stages, tmem_cols);         \
+    } while (0)
+    const bool u8 = s->idx_type == R3_IDX_U8;
+    if (s->K <= 8) { if (u8) R3_RT(uint8_t, 8); else R3_RT(int16_t, 8); }
+    else { if (u8) R3_RT(uint8_t, 16); else R3_RT(int16_t, 16); }
+#undef R3_RT
+    return launch_status();
+}
+
+}  // namespace r3

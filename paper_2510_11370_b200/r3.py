@@ -25,7 +25,8 @@ R3_IDX_U8, R3_IDX_I16 = 1, 2
 DEV_OK, DEV_BAD_INDEX, DEV_DUP_INDEX, DEV_TIMEOUT = 0, 1, 2, 3
 
 EXPORTS = [
-    "r3_status_string", "r3_capture_topk", "r3_capture_topk_batched", "r3_replay_gate_fwd",
+    "r3_status_string", "r3_capture_topk", "r3_capture_topk_batched",
+    "r3_capture_topk_workspace_bytes", "r3_capture_topk_ws", "r3_replay_gate_fwd",
     "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute", "r3_permute_static",
     "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_expert_up_swiglu",
     "r3_expert_down", "r3_combine",
@@ -50,6 +51,9 @@ for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
     getattr(lib, _n).argtypes = [_SP]
 lib.r3_capture_topk.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_capture_topk_batched.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P]
+lib.r3_capture_topk_workspace_bytes.restype = ctypes.c_size_t
+lib.r3_capture_topk_workspace_bytes.argtypes = [_SP, ctypes.c_int32]
+lib.r3_capture_topk_ws.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, ctypes.c_size_t, _P]
 lib.r3_replay_gate_fwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_gate_bwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_permute.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
@@ -159,6 +163,26 @@ def capture_topk_batched(s: Shape, L: int, x, w_router, idx_out=None, logits_out
         logits_out = torch.empty((L, s.T, s.E), dtype=torch.float32, device=dev)
     _check(lib.r3_capture_topk_batched(ctypes.byref(s), L, _ptr(x), _ptr(w_router),
                                        _ptr(idx_out), _ptr(logits_out), _stream(stream)))
+    return idx_out, logits_out
+
+
+def capture_topk_workspace_bytes(s: Shape, L: int = 1) -> int:
+    return lib.r3_capture_topk_workspace_bytes(ctypes.byref(s), L)
+
+
+def capture_topk_ws(s: Shape, L: int, x, w_router, idx_out=None, logits_out=None, *, ws=None,
+                    want_idx=True, want_logits=False, stream=None):
+    """capture_topk with scratch, so that float32 router weights run on the tensor cores too."""
+    dev = _dev(x)
+    lead = (L,) if x.dim() == 3 else ()
+    if idx_out is None and want_idx:
+        idx_out = torch.empty(lead + (s.T, s.K), dtype=_idx_dtype(s), device=dev)
+    if logits_out is None and want_logits:
+        logits_out = torch.empty(lead + (s.T, s.E), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(capture_topk_workspace_bytes(s, L), dev)
+    _check(lib.r3_capture_topk_ws(ctypes.byref(s), L, _ptr(x), _ptr(w_router), _ptr(idx_out),
+                                  _ptr(logits_out), _ptr(ws), ws.numel(), _stream(stream)))
     return idx_out, logits_out
 
 

@@ -154,6 +154,44 @@ def test_capture_exact_arithmetic_with_planted_ties(r3, act, rw):
     assert np.array_equal(idx.cpu().numpy().astype(np.int64), O.topk_indices(ref_s, K))
 
 
+@pytest.mark.parametrize("rw", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T,d,E,K", [(333, 64, 32, 6), (1000, 200, 128, 8), (130, 2048, 256, 16)])
+def test_capture_tensor_core_exact_arithmetic_with_planted_ties(r3, rw, T, d, E, K):
+    """The tcgen05 router kernel (bf16 activations, E a multiple of 16) on small-integer data:
+    sums are exact, so logits and record must equal the oracle's bit for bit, ties included.
+    float32 weights go through the three-plane split (the integers sit entirely in the top plane)."""
+    rng = np.random.default_rng(T + E)
+    x = torch.from_numpy(rng.integers(-3, 4, (T, d)).astype(np.float32)).to(torch.bfloat16)
+    w = torch.from_numpy(rng.integers(-2, 3, (E, d)).astype(np.float32)).to(rw)
+    w[5] = w[2]
+    w[17] = w[2]
+    w[E - 1] = w[0]
+    s = r3.make_shape(T, d, E, K, 8, router=rw)
+    idx, logits = r3.capture_topk_ws(s, 1, x.cuda(), w.cuda(), want_logits=True)
+    ref_s = O.router_logits(f64(x), f64(w))
+    assert np.array_equal(logits.cpu().numpy().astype(np.float64), ref_s)
+    assert np.array_equal(idx.cpu().numpy().astype(np.int64), O.topk_indices(ref_s, K))
+
+
+@pytest.mark.parametrize("T,d,E,K,L", [(4096, 2048, 128, 8, 1), (300, 520, 64, 4, 3),
+                                       (129, 2048, 256, 8, 2)])
+def test_capture_tensor_core_fp32_router_weights_keep_fp32_accuracy(r3, T, d, E, K, L):
+    x = torch.randn(L, T, d).to(torch.bfloat16)
+    w = torch.randn(L, E, d) * 0.02
+    s = r3.make_shape(T, d, E, K, 8)
+    assert r3.capture_topk_workspace_bytes(s, L) >= L * 3 * E * d * 2
+    idx, logits = r3.capture_topk_ws(s, L, x.cuda(), w.cuda(), want_logits=True)
+    near = 0
+    for l in range(L):
+        ref_s = O.router_logits(f64(x[l]), f64(w[l]))
+        assert rel_err(logits[l].cpu().numpy(), ref_s) < TOL_F32
+        near += check_record_against_logits(idx[l].cpu().numpy(), ref_s, K)
+    assert near < 0.05 * L * T
+    # logits only / record only give the same values
+    only_idx, _ = r3.capture_topk_ws(s, L, x.cuda(), w.cuda())
+    assert torch.equal(only_idx, idx)
+
+
 def check_record_against_logits(idx_gpu, s_ref, K, tau=1e-3):
     """Margin rule for floating-point near-ties: where the oracle's K-th and (K+1)-th logits are
     at least tau apart the sets must be equal; elsewhere the chosen set must be within tau of

@@ -33,7 +33,7 @@ def run_layer(r3, case, stepwise=False):
         torch.cuda.synchronize()
         assert st.item() == 0
         return dict(y=y, ds=ds, g=g)
-    _, logits = r3.capture_topk(s, c["x"], c["w_r"], want_idx=False, want_logits=True)
+    _, logits = r3.capture_topk_ws(s, 1, c["x"], c["w_r"], want_idx=False, want_logits=True)
     g = r3.replay_gate_fwd(s, logits, c["idx"], dev_status=st)
     counts, offsets, ros, sor, xp = r3.permute(s, c["idx"], c["x"], dev_status=st)
     o = r3.grouped_swiglu(s, xp, offsets, c["w_gate"], c["w_up"], c["w_down"], dev_status=st)
@@ -134,7 +134,7 @@ def run_big(r3, case, raw):
     st = r3.new_status("cuda")
     c = {k: getattr(case, k).cuda() for k in ("x", "dy", "w_r", "idx")}
     wg, wu, wd = (t.cuda() for t in raw)
-    _, logits = r3.capture_topk(s, c["x"], c["w_r"], want_idx=False, want_logits=True)
+    _, logits = r3.capture_topk_ws(s, 1, c["x"], c["w_r"], want_idx=False, want_logits=True)
     g = r3.replay_gate_fwd(s, logits, c["idx"], dev_status=st)
     counts, offsets, ros, sor, xp = r3.permute(s, c["idx"], c["x"], dev_status=st)
     o = r3.grouped_swiglu(s, xp, offsets, wg, wu, wd, dev_status=st)
