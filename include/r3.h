@@ -182,6 +182,12 @@ r3_status r3_expert_down(const r3_shape* shape, const void* w_down, void* o, voi
 r3_status r3_combine(const r3_shape* shape, const void* o, const int32_t* row_of_slot,
                      const float* gates, void* y, void* stream);
 
+/* The same with a residual: y[t] = residual[t] + sum_j gates[t,j] * o[row_of_slot[t,j]] (the sum is
+ * formed first, the residual added last, all in fp32, one rounding).  residual [T,d] act_dtype or
+ * NULL (then identical to r3_combine).  Used by r3_replay_stack for x_{l+1} = x_l + y_l. */
+r3_status r3_combine_residual(const r3_shape* shape, const void* o, const int32_t* row_of_slot,
+                              const float* gates, const void* residual, void* y, void* stream);
+
 /* Chain rule on Eq. (replay_output): dgates[t,j] = sum_c dy[t,c] * o[row_of_slot[t,j], c].
  * dy [T,d] act_dtype; dgates [T,K] f32. */
 r3_status r3_combine_bwd_gates(const r3_shape* shape, const void* dy, const void* o,
@@ -198,6 +204,30 @@ r3_status r3_replay_layer(const r3_shape* shape, const void* x, const void* w_ro
                           const void* w_down, const void* dy, void* y, float* dlogits,
                           float* gates_out, void* workspace, size_t ws_bytes,
                           int32_t* dev_status, void* stream);
+
+/* L independent replayed MoE blocks enqueued back to back: block l is r3_replay_layer on its own
+ * input x[l], record idx[l], weights and upstream gradient dy[l] (a model's MoE blocks with the
+ * sublayers between them left out, so that every block's input is given).  All tensors carry a
+ * leading layer axis: x, dy, y [L,T,d]; w_router [L,E,d]; idx [L,T,K]; w_gate/w_up [L,E,F,d];
+ * w_down [L,E,d,F]; dlogits [L,T,E] f32.  workspace: r3_replay_layer_workspace_bytes(shape). */
+r3_status r3_replay_blocks(const r3_shape* shape, int32_t L, const void* x, const void* w_router,
+                           const void* idx, const void* w_gate, const void* w_up,
+                           const void* w_down, const void* dy, void* y, float* dlogits,
+                           void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* A stack of L replayed MoE blocks (no attention) with residual connections,
+ *   x_{l+1} = x_l + y_replay,l(x_l),   l = 0..L-1,
+ * each block being Eq. (replay_output) with its own weights and its own record, plus the
+ * router-logit gradient of every block for one upstream gradient dy [T,d] shared by all blocks
+ * (the gradient that reaches a block's output through the identity path of the later blocks).
+ * Per-layer tensors are stacked on a leading layer axis: w_router [L,E,d], idx [L,T,K],
+ * w_gate/w_up [L,E,F,d], w_down [L,E,d,F]; x0 [T,d]; outputs x_out [T,d] = x_L and
+ * dlogits [L,T,E] f32.  workspace: r3_replay_stack_workspace_bytes(shape) (independent of L). */
+size_t r3_replay_stack_workspace_bytes(const r3_shape* shape);
+r3_status r3_replay_stack(const r3_shape* shape, int32_t L, const void* x0, const void* w_router,
+                          const void* idx, const void* w_gate, const void* w_up,
+                          const void* w_down, const void* dy, void* x_out, float* dlogits,
+                          void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /* As r3_replay_layer, with the per-step tensors in HOST memory (pinned memory recommended):
  * x_host, idx_host, dy_host are copied to the device, y_host and dlogits_host are copied back,

@@ -276,3 +276,25 @@ def layer_tokens(x_rows, w_r, idx_rows, w_gate, w_up, w_down, dy_rows):
         dg = dgates(dy_rows[t:t + 1], eo)
         dss.append(replay_gate_bwd(g, dg, idx_rows[t:t + 1], E)[0])
     return np.stack(ys), np.stack(dss)
+
+
+# ----------------------------------------------------------------------------------------------
+# A stack of replayed MoE blocks with residual connections (benchmark configuration 5)
+# ----------------------------------------------------------------------------------------------
+def replay_stack_tokens(x_rows, layers, dy_rows, store=None):
+    """Follows the given tokens through L residual blocks  x_{l+1} = store(x_l + y_replay,l(x_l)).
+
+    Tokens are independent of each other in every step of the path, so a subset can be followed
+    on its own.  ``layers`` is a sequence of (w_r, idx_rows, w_gate, w_up, w_down) per block, with
+    idx_rows the record rows of these tokens.  ``dy_rows`` is the upstream gradient used for every
+    block (the gradient arriving through the identity path).  ``store`` models the rounding of
+    the stored activations (None = keep float64).  Returns (x_L rows, [ds_l rows for each l])."""
+    x = _f64(x_rows)
+    dss = []
+    for (w_r, idx_rows, w_gate, w_up, w_down) in layers:
+        y, ds = layer_tokens(x, w_r, idx_rows, w_gate, w_up, w_down, dy_rows)
+        dss.append(ds)
+        x = x + y
+        if store is not None:
+            x = _f64(store(x))
+    return x, dss

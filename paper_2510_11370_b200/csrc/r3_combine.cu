@@ -10,7 +10,8 @@ constexpr int kSlotBatch = 8;     // slots gathered together (their loads are is
 template <typename ActT, int TPT>
 __global__ void __launch_bounds__(256)
 combine_kernel(const ActT* __restrict__ o, const int32_t* __restrict__ row_of_slot,
-               const float* __restrict__ gates, ActT* __restrict__ y, int T, int K, int d) {
+               const float* __restrict__ gates, const ActT* __restrict__ residual,
+               ActT* __restrict__ y, int T, int K, int d) {
     using V = Vec16<ActT>;
     constexpr int N = V::N;
     const int team = threadIdx.x / TPT, tl = threadIdx.x % TPT;
@@ -47,6 +48,12 @@ combine_kernel(const ActT* __restrict__ o, const int32_t* __restrict__ row_of_sl
                     for (int i = 0; i < N; ++i) acc[i] = fmaf(gj[u], f[i], acc[i]);
                 }
             }
+        }
+        if (residual) {                      // y = residual + sum (one extra fp32 add per element)
+            float f[N];
+            reinterpret_cast<const V*>(residual)[(size_t)t * row_vecs + c].unpack(f);
+#pragma unroll
+            for (int i = 0; i < N; ++i) acc[i] += f[i];
         }
         V out;
         out.pack(acc);
@@ -125,17 +132,18 @@ static int pick_team(int row_vecs) {
 
 template <typename ActT>
 static void launch_combine(const r3_shape* s, const void* o, const int32_t* row_of_slot,
-                           const float* gates, void* y, cudaStream_t cs) {
+                           const float* gates, const void* residual, void* y, cudaStream_t cs) {
     const int T = s->T, K = s->K, d = s->d;
     const int tpt = pick_team(d / Vec16<ActT>::N);
     const unsigned grid = (unsigned)((T + 256 / tpt - 1) / (256 / tpt));
     const ActT* op = static_cast<const ActT*>(o);
     ActT* yp = static_cast<ActT*>(y);
+    const ActT* rp = static_cast<const ActT*>(residual);
     switch (tpt) {
-        case 32: combine_kernel<ActT, 32><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, yp, T, K, d); break;
-        case 64: combine_kernel<ActT, 64><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, yp, T, K, d); break;
-        case 128: combine_kernel<ActT, 128><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, yp, T, K, d); break;
-        default: combine_kernel<ActT, 256><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, yp, T, K, d); break;
+        case 32: combine_kernel<ActT, 32><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, rp, yp, T, K, d); break;
+        case 64: combine_kernel<ActT, 64><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, rp, yp, T, K, d); break;
+        case 128: combine_kernel<ActT, 128><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, rp, yp, T, K, d); break;
+        default: combine_kernel<ActT, 256><<<grid, 256, 0, cs>>>(op, row_of_slot, gates, rp, yp, T, K, d); break;
     }
 }
 
@@ -157,16 +165,24 @@ static void launch_combine_bwd(const r3_shape* s, const void* dy, const void* o,
 
 }  // namespace r3
 
-extern "C" r3_status r3_combine(const r3_shape* shape, const void* o, const int32_t* row_of_slot,
-                                const float* gates, void* y, void* stream) {
+extern "C" r3_status r3_combine_residual(const r3_shape* shape, const void* o,
+                                         const int32_t* row_of_slot, const float* gates,
+                                         const void* residual, void* y, void* stream) {
     r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
     if (shape->T == 0) return R3_OK;
     if (!o || !row_of_slot || !gates || !y) return R3_ERR_INVALID_ARG;
-    if (!r3::aligned(o, 16) || !r3::aligned(y, 16)) return R3_ERR_INVALID_ARG;
+    if (!r3::aligned(o, 16) || !r3::aligned(y, 16) || !r3::aligned(residual, 16))
+        return R3_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    R3_DISPATCH_ACT(shape, ActT, r3::launch_combine<ActT>(shape, o, row_of_slot, gates, y, cs));
+    R3_DISPATCH_ACT(shape, ActT,
+                    r3::launch_combine<ActT>(shape, o, row_of_slot, gates, residual, y, cs));
     return r3::launch_status();
+}
+
+extern "C" r3_status r3_combine(const r3_shape* shape, const void* o, const int32_t* row_of_slot,
+                                const float* gates, void* y, void* stream) {
+    return r3_combine_residual(shape, o, row_of_slot, gates, nullptr, y, stream);
 }
 
 extern "C" r3_status r3_combine_bwd_gates(const r3_shape* shape, const void* dy, const void* o,

@@ -61,6 +61,36 @@ extern "C" size_t r3_replay_layer_workspace_bytes(const r3_shape* shape) {
     return r3::carve(shape, nullptr).total;
 }
 
+namespace r3 {
+// One replayed layer; `residual` (may be null) is added to the combined output.
+static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_router,
+                           const void* idx, const void* w_gate, const void* w_up,
+                           const void* w_down, const void* dy, const void* residual, void* y,
+                           float* dlogits, float* gates_out, void* workspace,
+                           int32_t* dev_status, void* stream) {
+    const LayerWs w = carve(shape, workspace);
+    float* gates = gates_out ? gates_out : w.gates;
+    r3_status st;
+    // s_train = x W_r (only the logits are needed on the training side)
+    if ((st = r3_capture_topk_ws(shape, 1, x, w_router, nullptr, w.logits, w.router_ws,
+                                 w.router_bytes, stream)) != R3_OK)
+        return st;
+    if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
+        return st;
+    if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
+                         w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
+        return st;
+    if ((st = r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, w.swiglu_ws,
+                                w.swiglu_bytes, dev_status, stream)) != R3_OK)
+        return st;
+    if ((st = r3_combine_residual(shape, w.o, w.row_of_slot, gates, residual, y, stream)) != R3_OK)
+        return st;
+    if ((st = r3_combine_bwd_gates(shape, dy, w.o, w.row_of_slot, w.dgates, stream)) != R3_OK)
+        return st;
+    return r3_replay_gate_bwd(shape, gates, w.dgates, idx, dlogits, stream);
+}
+}  // namespace r3
+
 extern "C" r3_status r3_replay_layer(const r3_shape* shape, const void* x, const void* w_router,
                                      const void* idx, const void* w_gate, const void* w_up,
                                      const void* w_down, const void* dy, void* y, float* dlogits,
@@ -74,25 +104,89 @@ extern "C" r3_status r3_replay_layer(const r3_shape* shape, const void* x, const
     if (!workspace || !r3::aligned(workspace, 256) ||
         ws_bytes < r3_replay_layer_workspace_bytes(shape))
         return R3_ERR_WORKSPACE;
-    const r3::LayerWs w = r3::carve(shape, workspace);
-    float* gates = gates_out ? gates_out : w.gates;
+    return r3::run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y, dlogits,
+                         gates_out, workspace, dev_status, stream);
+}
 
-    // s_train = x W_r (only the logits are needed on the training side)
-    if ((st = r3_capture_topk_ws(shape, 1, x, w_router, nullptr, w.logits, w.router_ws,
-                                 w.router_bytes, stream)) != R3_OK)
-        return st;
-    if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
-        return st;
-    if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
-                         w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
-        return st;
-    if ((st = r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, w.swiglu_ws,
-                                w.swiglu_bytes, dev_status, stream)) != R3_OK)
-        return st;
-    if ((st = r3_combine(shape, w.o, w.row_of_slot, gates, y, stream)) != R3_OK) return st;
-    if ((st = r3_combine_bwd_gates(shape, dy, w.o, w.row_of_slot, w.dgates, stream)) != R3_OK)
-        return st;
-    return r3_replay_gate_bwd(shape, gates, w.dgates, idx, dlogits, stream);
+// ---- a stack of L replayed MoE blocks with residual connections ------------------------------
+extern "C" size_t r3_replay_stack_workspace_bytes(const r3_shape* shape) {
+    if (r3::check_shape(shape) != R3_OK) return 0;
+    const size_t xb = r3::round_up((size_t)shape->T * shape->d * r3::act_bytes(shape), 256);
+    return 2 * xb + r3_replay_layer_workspace_bytes(shape);
+}
+
+extern "C" r3_status r3_replay_stack(const r3_shape* shape, int32_t L, const void* x0,
+                                     const void* w_router, const void* idx, const void* w_gate,
+                                     const void* w_up, const void* w_down, const void* dy,
+                                     void* x_out, float* dlogits, void* workspace, size_t ws_bytes,
+                                     int32_t* dev_status, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (L <= 0) return R3_ERR_INVALID_ARG;
+    if (shape->T == 0) return R3_OK;
+    if (!x0 || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !x_out || !dlogits)
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_stack_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    const size_t T = shape->T, d = shape->d, E = shape->E, F = shape->F, K = shape->K;
+    const size_t es = r3::act_bytes(shape);
+    const size_t xb = r3::round_up(T * d * es, 256);
+    char* ws = static_cast<char*>(workspace);
+    void* ping[2] = {ws, ws + xb};
+    void* inner = ws + 2 * xb;
+    const size_t rw = E * d * (shape->router_w_dtype == R3_BF16 ? 2 : 4);
+    const char* wr = static_cast<const char*>(w_router);
+    const char* wg = static_cast<const char*>(w_gate);
+    const char* wu = static_cast<const char*>(w_up);
+    const char* wd = static_cast<const char*>(w_down);
+    const char* rec = static_cast<const char*>(idx);
+    const void* cur = x0;
+    for (int32_t l = 0; l < L; ++l) {
+        void* nxt = (l == L - 1) ? x_out : ping[l & 1];
+        // x_{l+1} = x_l + y_l : the block input is also the residual
+        st = r3::run_layer(shape, cur, wr + (size_t)l * rw, rec + (size_t)l * T * K * r3::idx_bytes(shape),
+                           wg + (size_t)l * E * F * d * es, wu + (size_t)l * E * F * d * es,
+                           wd + (size_t)l * E * d * F * es, dy, cur, nxt,
+                           dlogits + (size_t)l * T * E, nullptr, inner, dev_status, stream);
+        if (st != R3_OK) return st;
+        cur = nxt;
+    }
+    return R3_OK;
+}
+
+// ---- L independent replayed MoE blocks (each with its own input) -----------------------------
+extern "C" r3_status r3_replay_blocks(const r3_shape* shape, int32_t L, const void* x,
+                                      const void* w_router, const void* idx, const void* w_gate,
+                                      const void* w_up, const void* w_down, const void* dy,
+                                      void* y, float* dlogits, void* workspace, size_t ws_bytes,
+                                      int32_t* dev_status, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (L <= 0) return R3_ERR_INVALID_ARG;
+    if (shape->T == 0) return R3_OK;
+    if (!x || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !y || !dlogits)
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_layer_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    const size_t T = shape->T, d = shape->d, E = shape->E, F = shape->F, K = shape->K;
+    const size_t es = r3::act_bytes(shape);
+    const size_t rw = E * d * (shape->router_w_dtype == R3_BF16 ? 2 : 4);
+    const size_t act = T * d * es, ew = E * F * d * es;
+    for (int32_t l = 0; l < L; ++l) {
+        st = r3::run_layer(shape, static_cast<const char*>(x) + l * act,
+                           static_cast<const char*>(w_router) + l * rw,
+                           static_cast<const char*>(idx) + l * T * K * r3::idx_bytes(shape),
+                           static_cast<const char*>(w_gate) + l * ew,
+                           static_cast<const char*>(w_up) + l * ew,
+                           static_cast<const char*>(w_down) + l * ew,
+                           static_cast<const char*>(dy) + l * act, nullptr,
+                           static_cast<char*>(y) + l * act, dlogits + l * T * E, nullptr,
+                           workspace, dev_status, stream);
+        if (st != R3_OK) return st;
+    }
+    return R3_OK;
 }
 
 namespace r3 {

@@ -30,7 +30,8 @@ EXPORTS = [
     "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute", "r3_permute_static",
     "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_expert_up_swiglu",
     "r3_expert_down", "r3_combine",
-    "r3_combine_bwd_gates", "r3_replay_layer_workspace_bytes", "r3_replay_layer",
+    "r3_combine_residual", "r3_combine_bwd_gates", "r3_replay_layer_workspace_bytes",
+    "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
 ]
 
@@ -46,6 +47,7 @@ _SP = ctypes.POINTER(Shape)
 lib.r3_status_string.restype = ctypes.c_char_p
 lib.r3_status_string.argtypes = [ctypes.c_int]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
+           "r3_replay_stack_workspace_bytes",
            "r3_replay_layer_workspace_bytes", "r3_replay_layer_host_workspace_bytes"):
     getattr(lib, _n).restype = ctypes.c_size_t
     getattr(lib, _n).argtypes = [_SP]
@@ -62,6 +64,9 @@ lib.r3_grouped_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size
 lib.r3_expert_up_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_expert_down.argtypes = [_SP, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_combine.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_combine_residual.argtypes = [_SP, _P, _P, _P, _P, _P, _P]
+lib.r3_replay_blocks.argtypes = [_SP, ctypes.c_int32] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
+lib.r3_replay_stack.argtypes = [_SP, ctypes.c_int32] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_layer_host.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
@@ -275,6 +280,54 @@ def combine(s: Shape, o, row_of_slot, gates, y=None, stream=None):
     _check(lib.r3_combine(ctypes.byref(s), _ptr(o), _ptr(row_of_slot), _ptr(gates), _ptr(y),
                           _stream(stream)))
     return y
+
+
+def combine_residual(s: Shape, o, row_of_slot, gates, residual, y=None, stream=None):
+    """y = residual + sum_j gates[:, j] * o[row_of_slot[:, j]]."""
+    if y is None:
+        y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=_dev(o))
+    _check(lib.r3_combine_residual(ctypes.byref(s), _ptr(o), _ptr(row_of_slot), _ptr(gates),
+                                   _ptr(residual), _ptr(y), _stream(stream)))
+    return y
+
+
+def replay_blocks(s: Shape, L: int, x, w_router, idx, w_gate, w_up, w_down, dy, *, y=None,
+                  dlogits=None, ws=None, dev_status=None, stream=None):
+    """L independent replayed blocks, all tensors stacked on a leading layer axis.
+    Returns (y [L,T,d], dlogits [L,T,E])."""
+    dev = _dev(x)
+    if y is None:
+        y = torch.empty((L, s.T, s.d), dtype=_act_dtype(s), device=dev)
+    if dlogits is None:
+        dlogits = torch.empty((L, s.T, s.E), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(replay_layer_workspace_bytes(s), dev)
+    _check(lib.r3_replay_blocks(ctypes.byref(s), L, _ptr(x), _ptr(w_router), _ptr(idx),
+                                _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(dy), _ptr(y),
+                                _ptr(dlogits), _ptr(ws), ws.numel(), _ptr(dev_status),
+                                _stream(stream)))
+    return y, dlogits
+
+
+def replay_stack_workspace_bytes(s: Shape) -> int:
+    return lib.r3_replay_stack_workspace_bytes(ctypes.byref(s))
+
+
+def replay_stack(s: Shape, L: int, x0, w_router, idx, w_gate, w_up, w_down, dy, *, x_out=None,
+                 dlogits=None, ws=None, dev_status=None, stream=None):
+    """L residual MoE blocks with replayed routing.  Returns (x_L [T,d], dlogits [L,T,E])."""
+    dev = _dev(x0)
+    if x_out is None:
+        x_out = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    if dlogits is None:
+        dlogits = torch.empty((L, s.T, s.E), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(replay_stack_workspace_bytes(s), dev)
+    _check(lib.r3_replay_stack(ctypes.byref(s), L, _ptr(x0), _ptr(w_router), _ptr(idx),
+                               _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(dy), _ptr(x_out),
+                               _ptr(dlogits), _ptr(ws), ws.numel(), _ptr(dev_status),
+                               _stream(stream)))
+    return x_out, dlogits
 
 
 def combine_bwd_gates(s: Shape, dy, o, row_of_slot, dgates=None, stream=None):

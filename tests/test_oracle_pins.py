@@ -344,6 +344,36 @@ def test_per_token_evaluation_matches_batched():
     assert np.allclose(ds, out["ds"][sel], atol=1e-13)
 
 
+def test_residual_stack_against_dense_definition_per_block():
+    """Two residual blocks: every block's output is checked with the all-experts form of
+    Eq. (replay_output) evaluated at that block's input, and x_L - x_0 is the sum of the outputs."""
+    r = rng(500)
+    T, d, E, F, K, L = 5, 4, 3, 3, 2, 3
+    x0 = r.standard_normal((T, d))
+    dy = r.standard_normal((T, d))
+    layers, dense = [], []
+    for l in range(L):
+        _, w_r, wg, wu, wd, _ = tiny_layer(510 + l, T, d, E, F)
+        idx = np.stack([r.permutation(E)[:K] for _ in range(T)])
+        layers.append((w_r, idx, wg, wu, wd))
+    xL, dss = O.replay_stack_tokens(x0, layers, dy)
+    x = x0.copy()
+    for l, (w_r, idx, wg, wu, wd) in enumerate(layers):
+        s = O.router_logits(x, w_r)
+        y = O.replay_output_dense(x, s, O.mask_from_indices(idx, E), wg, wu, wd)
+        out = O.layer_fwd_bwd(x, w_r, idx, wg, wu, wd, dy)
+        assert np.allclose(dss[l], out["ds"], atol=1e-13)
+        x = x + y
+    assert np.allclose(xL, x, atol=1e-12)
+    # a subset of tokens followed on its own gives the same rows; `store` is applied per block
+    sub = [1, 3]
+    xs, _ = O.replay_stack_tokens(x0[sub], [(a, b[sub], c, e, f) for a, b, c, e, f in layers],
+                                  dy[sub])
+    assert np.allclose(xs, xL[sub], atol=1e-13)
+    xr, _ = O.replay_stack_tokens(x0, layers, dy, store=lambda v: np.round(v, 2))
+    assert np.array_equal(xr, np.round(xr, 2)) and not np.allclose(xr, xL, atol=1e-6)
+
+
 # ------------------------------------------------------------------ planted mistakes are caught
 def test_pins_catch_planted_mistakes(monkeypatch):
     """A wrong sign in silu, a transposed router weight or gates taken from the inference
