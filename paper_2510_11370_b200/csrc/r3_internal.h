@@ -26,14 +26,15 @@ inline int max_m_tiles(long long R, int E, int BM) {
 r3_status launch_build_tiles(const int32_t* offsets, int E, int BM, int32_t* tiles,
                              cudaStream_t stream);
 
-// bf16 grouped SwiGLU on the tcgen05 tensor cores (sm_100a).  `tiles` must have been built with
-// BM = tc_block_m().
-int tc_block_m();
+// bf16 grouped SwiGLU on the tcgen05 tensor cores (sm_100a, two CTAs per MMA).  `work` is
+// tc_work_bytes() of scratch for the two device-built work lists (the up phase builds both from
+// `offsets`; the down phase reads the list the up phase left there).
+size_t tc_work_bytes(const r3_shape* shape);
 // phases: bit 0 = gate/up projections + SwiGLU (xp -> h), bit 1 = down projection (h -> o).
 enum { kPhaseUp = 1, kPhaseDown = 2 };
-r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const int32_t* tiles,
+r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const int32_t* offsets,
                                    const void* w_gate, const void* w_up, const void* w_down,
-                                   void* h, void* o, int32_t* dev_status, int phases,
+                                   void* h, void* o, void* work, int32_t* dev_status, int phases,
                                    cudaStream_t stream);
 
 // Router logits + top-K on the tensor cores (bf16 activations, E a multiple of 16 up to 256,

@@ -161,15 +161,17 @@ static r3_status launch_grouped_swiglu_f32(const r3_shape* s, const void* xp, co
 static size_t h_bytes(const r3_shape* s) {
     return round_up((size_t)s->T * s->K * s->F * act_bytes(s), 256);
 }
-static int block_m(const r3_shape* s) { return s->act_dtype == R3_BF16 ? tc_block_m() : SBM; }
+// scratch after h: the tensor-core work lists (bf16) or the row-tile list (float32)
+static size_t list_bytes(const r3_shape* s) {
+    if (s->act_dtype == R3_BF16) return tc_work_bytes(s);
+    return round_up(tile_list_bytes((long long)s->T * s->K, s->E, SBM), 256);
+}
 
 }  // namespace r3
 
 extern "C" size_t r3_grouped_swiglu_workspace_bytes(const r3_shape* shape) {
     if (r3::check_shape(shape) != R3_OK) return 0;
-    const long long R = (long long)shape->T * shape->K;
-    return r3::h_bytes(shape) +
-           r3::round_up(r3::tile_list_bytes(R, shape->E, r3::block_m(shape)), 256);
+    return r3::h_bytes(shape) + r3::list_bytes(shape);
 }
 
 namespace r3 {
@@ -194,13 +196,13 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const int32_
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     void* h = workspace;
     int32_t* tiles = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + h_bytes(shape));
+    if (shape->act_dtype == R3_BF16)
+        return launch_grouped_swiglu_tc(shape, xp, offsets, w_gate, w_up, w_down, h, o, tiles,
+                                        dev_status, phases, cs);
     if (up) {
-        st = launch_build_tiles(offsets, shape->E, block_m(shape), tiles, cs);
+        st = launch_build_tiles(offsets, shape->E, SBM, tiles, cs);
         if (st != R3_OK) return st;
     }
-    if (shape->act_dtype == R3_BF16)
-        return launch_grouped_swiglu_tc(shape, xp, tiles, w_gate, w_up, w_down, h, o, dev_status,
-                                        phases, cs);
     return launch_grouped_swiglu_f32(shape, xp, tiles, w_gate, w_up, w_down, h, o, phases, cs);
 }
 }  // namespace r3

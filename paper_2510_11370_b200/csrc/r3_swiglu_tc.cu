@@ -1,20 +1,34 @@
-// bf16 grouped SwiGLU expert GEMMs on the Blackwell tensor cores (sm_100a).
+// bf16 grouped SwiGLU expert GEMMs on the Blackwell tensor cores (sm_100a), two CTAs per MMA.
 //
-// Two persistent, warp-specialised kernels share one template:
-//   MODE 0:  h[r, f]  = silu(xp[r] . W_gate,e[f]) * (xp[r] . W_up,e[f])      (K = d, N = F)
-//   MODE 1:  o[r, c]  = h[r] . W_down,e[c]                                    (K = F, N = d)
-// A CTA owns output tiles of 128 rows x 256 accumulator columns.  In MODE 0 the 256 columns are
-// 128 gate columns followed by the 128 up columns of the same F slice (two TMA loads into one
-// B tile), so the SwiGLU product is formed in the epilogue without repacking weights.
+//   MODE 0:  h[r, f]  = silu(xp[r] . W_gate,e[f]) * (xp[r] . W_up,e[f])      (K = d, out = F)
+//   MODE 1:  o[r, c]  = h[r] . W_down,e[c]                                    (K = F, out = d)
 //
-// Roles (320 threads): warp 0 lane 0 = TMA producer (cp.async.bulk.tensor into a 4-stage ring of
-// 128B-swizzled tiles), warp 1 lane 0 = tcgen05.mma issuer (accumulators in TMEM, two stages of
-// 256 columns so the epilogue of a tile overlaps the main loop of the next), warps 2..9 =
-// epilogue (tcgen05.ld -> registers -> bf16 -> global).  Rows that belong to the next expert or
-// lie beyond R are computed but never stored.
+// Orientation.  The WEIGHT rows are the M side of the MMA and the TOKEN rows are the N side, so
+// the accumulator holds out^T: tensor-memory lane = output feature, column = token.  M is fixed
+// by the hardware (256 per CTA pair) while N may be any multiple of 16 up to 256, so an expert
+// with an awkward number of rows costs MMA time in proportion to its rows (padding to 16), not
+// to the next multiple of a fixed row tile.
+//
+// A work item is (expert, token tile of N <= 256 rows, feature tile).  The two CTAs of a cluster
+// share it (tcgen05 cta_group::2, UMMA 256 x N x 16): each CTA loads 128 weight rows and N/2
+// token rows per 64-wide k block (32 KB per stage instead of the 48 KB a single-CTA 128x256 tile
+// needs for the same MMA time), and receives 128 features x N tokens in its own tensor memory.
+// In MODE 0 the 128 weight rows of a CTA are 64 gate rows followed by the 64 up rows of the same
+// features, so lanes 0-63 hold the gate pre-activations and lanes 64-127 the up projections; the
+// epilogue exchanges them through shared memory to form the SwiGLU product.
+//
+// Items are ordered (expert, feature tile, token tile) so that consecutive items re-use a weight
+// tile from L2, and are dealt to the clusters as contiguous ranges of equal estimated cost
+// (build_work_kernel), so each cluster walks its own range with no atomics.
+//
+// Roles (192 threads per CTA): warp 0 lane 0 = TMA producer (both CTAs, into a 6-stage ring of
+// 128B-swizzled tiles), warp 1 lane 0 of the leader CTA = MMA issuer (two accumulator stages of
+// 256 columns, so the epilogue of an item overlaps the main loop of the next), warps 2..5 =
+// epilogue (tcgen05.ld -> transpose through shared memory -> 16-byte global stores).
 //
 // Every mbarrier wait is bounded by a clock limit; when a wait runs out the CTA raises a shared
-// abort flag, reports R3_DEV_TIMEOUT, lets the other roles drain, frees its TMEM and returns.
+// abort flag, reports R3_DEV_TIMEOUT, lets the other roles drain (they keep their barrier
+// protocol but skip the work), frees its tensor memory and returns.
 #include "r3_common.cuh"
 #include "r3_internal.h"
 #include "r3_tc.cuh"
@@ -22,116 +36,237 @@
 namespace r3 {
 namespace tc {
 
-constexpr int BM = 128;            // rows per tile (UMMA M)
-constexpr int BN = 256;            // accumulator columns per tile (UMMA N)
+constexpr int BMF = 128;           // weight rows (output features) per CTA; UMMA M = 2 * BMF
+constexpr int BNT = 256;           // most token rows per item (UMMA N)
 constexpr int BK = 64;             // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int UK = 16;             // k per tcgen05.mma (bf16)
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int ACC_STAGES = 2;
-constexpr int TMEM_COLS = ACC_STAGES * BN;       // 512 = all of tensor memory
-constexpr int A_BYTES = BM * BK * 2;             // 16 KB
-constexpr int B_BYTES = BN * BK * 2;             // 32 KB
+constexpr int TMEM_COLS = ACC_STAGES * BNT;      // 512 = all of tensor memory
+constexpr int A_BYTES = BMF * BK * 2;            // 16 KB of weights per CTA and stage
+constexpr int B_BYTES = (BNT / 2) * BK * 2;      // up to 16 KB of tokens per CTA and stage
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 4;
 constexpr int THREADS = (2 + EPI_WARPS) * 32;
+constexpr int EPI_BYTES = 20 * 1024;             // transpose / exchange buffers of the epilogue
 constexpr int BAR_BYTES = 256;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;   // + alignment slack
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + 1024;  // + alignment
+constexpr int FEAT0 = BMF;         // h features per item in MODE 0 (64 per CTA, gate + up rows)
+constexpr int FEAT1 = 2 * BMF;     // o features per item in MODE 1
+constexpr int kMaxClusters = 254;
 
-constexpr uint32_t kInstrDesc = instr_desc_bf16(BM, BN);
+// Tensor maps of one launch.  b[i] loads a token box of 8 * (i + 1) rows.
+struct alignas(64) PairMaps {
+    CUtensorMap a0, a1;
+    CUtensorMap b[BNT / 16];
+};
 
-__device__ __forceinline__ void store8(__nv_bfloat16* dst, const float* f) {
-    uint4 v;
-    __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-    *reinterpret_cast<uint4*>(dst) = v;
+// ---- work list -------------------------------------------------------------------------------
+// Per list: int32 ranges[kRangeInts] (ranges[p] .. ranges[p+1] = items of cluster p), then one
+// int4 per item = {expert | feature tile << 16, first row, N (multiple of 16), valid rows}.
+constexpr int kRangeInts = 256;
+
+__host__ __device__ inline int split_tiles(int cnt) { return (cnt + BNT - 1) / BNT; }
+__host__ __device__ inline int split_rows(int cnt, int nt) {      // rows per tile, multiple of 16
+    return (((cnt + nt - 1) / nt) + 15) & ~15;
+}
+// Estimated duration of an item in units of one token column of MMA time: the MMA time grows
+// with N, but below about 128 columns the weight tile's load time dominates.
+__host__ __device__ inline int item_cost(int n) { return (n < 128 ? 128 : n) + 24; }
+
+struct ExpertSplit {
+    int lo, cnt, nt, q, n_last;
+    long long cost_f;              // cost of the expert's token tiles for one feature tile
+};
+__device__ __forceinline__ ExpertSplit split_of(const int32_t* offsets, int e) {
+    ExpertSplit s;
+    s.lo = offsets[e];
+    s.cnt = offsets[e + 1] - s.lo;
+    s.nt = split_tiles(s.cnt);
+    s.q = s.nt ? split_rows(s.cnt, s.nt) : 0;
+    s.n_last = s.nt ? ((s.cnt - (s.nt - 1) * s.q + 15) & ~15) : 0;
+    s.cost_f = s.nt ? (long long)(s.nt - 1) * item_cost(s.q) + item_cost(s.n_last) : 0;
+    return s;
 }
 
+// One CTA per list (blockIdx.x = 0: up projection with nf0 feature tiles, 1: down with nf1).
+__global__ void __launch_bounds__(1024)
+build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1, int P,
+                  int32_t* __restrict__ list0, int32_t* __restrict__ list1) {
+    __shared__ int32_t s_items[1025];
+    __shared__ long long s_cost[1025];
+    __shared__ int32_t w_items[32];
+    __shared__ long long w_cost[32];
+    const int nf = blockIdx.x == 0 ? nf0 : nf1;
+    int32_t* ranges = blockIdx.x == 0 ? list0 : list1;
+    int4* items = reinterpret_cast<int4*>(ranges + kRangeInts);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    int32_t my_items = 0;
+    long long my_cost = 0;
+    if (tid < E) {
+        const ExpertSplit s = split_of(offsets, tid);
+        my_items = s.nt * nf;
+        my_cost = s.cost_f * nf;
+    }
+    int32_t ii = my_items;
+    long long cc = my_cost;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t a = __shfl_up_sync(0xffffffffu, ii, o);
+        const long long b = __shfl_up_sync(0xffffffffu, cc, o);
+        if (lane >= o) { ii += a; cc += b; }
+    }
+    if (lane == 31) { w_items[warp] = ii; w_cost[warp] = cc; }
+    __syncthreads();
+    if (warp == 0) {
+        const int32_t a0 = w_items[lane];
+        const long long b0 = w_cost[lane];
+        int32_t a = a0;
+        long long b = b0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t x = __shfl_up_sync(0xffffffffu, a, o);
+            const long long y = __shfl_up_sync(0xffffffffu, b, o);
+            if (lane >= o) { a += x; b += y; }
+        }
+        w_items[lane] = a - a0;
+        w_cost[lane] = b - b0;
+    }
+    __syncthreads();
+    s_items[tid] = w_items[warp] + ii - my_items;      // exclusive prefixes
+    s_cost[tid] = w_cost[warp] + cc - my_cost;
+    if (tid == 1023) { s_items[1024] = w_items[warp] + ii; s_cost[1024] = w_cost[warp] + cc; }
+    __syncthreads();
+    const int32_t I = s_items[1024];
+    const long long C = s_cost[1024];
+
+    // start cost, owner cluster and fields of item i
+    auto describe = [&](int32_t i, int4* out) -> int {
+        int lo = 0, hi = E;                      // last e with s_items[e] <= i
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_items[mid] <= i) lo = mid; else hi = mid;
+        }
+        const int e = lo;
+        const ExpertSplit s = split_of(offsets, e);
+        const int k = i - s_items[e];
+        const int f = k / s.nt, j = k - f * s.nt;
+        const long long cs = s_cost[e] + (long long)f * s.cost_f + (long long)j * item_cost(s.q);
+        if (out) {
+            const int n = (j == s.nt - 1) ? s.n_last : s.q;
+            const int valid = min(s.q, s.cnt - j * s.q);
+            *out = make_int4(e | (f << 16), s.lo + j * s.q, n, valid);
+        }
+        int owner = (int)((cs * P) / C);
+        return owner < P ? owner : P - 1;
+    };
+    for (int32_t i = tid; i < I; i += 1024) {
+        int4 it;
+        const int owner = describe(i, &it);
+        items[i] = it;
+        const int prev = i == 0 ? -1 : describe(i - 1, nullptr);
+        for (int p = prev + 1; p <= owner; ++p) ranges[p] = i;
+    }
+    if (tid == 0) {
+        const int last = I > 0 ? describe(I - 1, nullptr) : -1;
+        for (int p = last + 1; p <= P; ++p) ranges[p] = I;
+    }
+}
+
+// ---- the GEMM kernel --------------------------------------------------------------------------
 template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
-grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
-                       const __grid_constant__ CUtensorMap tmB0,
-                       const __grid_constant__ CUtensorMap tmB1,
-                       const int32_t* __restrict__ tiles, __nv_bfloat16* __restrict__ out,
-                       int Kdim, int Nout, int n_blocks, int32_t* dev_status) {
+grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* __restrict__ list,
+                         __nv_bfloat16* __restrict__ out, int Kdim, int Nout,
+                         int32_t* dev_status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bar0 = base + STAGES * STAGE_BYTES;
+    uint8_t* epi_ptr = base_ptr + STAGES * STAGE_BYTES;
+    const uint32_t bar0 = base + STAGES * STAGE_BYTES + EPI_BYTES;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + ACC_STAGES + a); };
-    volatile uint32_t* tmem_slot =
-        reinterpret_cast<volatile uint32_t*>(base_ptr + STAGES * STAGE_BYTES + 128);
-    volatile int* abort_flag =
-        reinterpret_cast<volatile int*>(base_ptr + STAGES * STAGE_BYTES + 132);
+    uint8_t* misc = epi_ptr + EPI_BYTES + 128;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_mtiles = tiles[0];
-    const int total = num_mtiles * n_blocks;
+    const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
+    const int pair = blockIdx.x >> 1;
+    const int w_step = gridDim.x >> 1;
+    const int w_begin = pair, w_end = list[w_step];
+    const int4* items = reinterpret_cast<const int4*>(list + kRangeInts);
     const int kblocks = (Kdim + BK - 1) / BK;
-    const int4* ents = reinterpret_cast<const int4*>(tiles + kTileHeaderInts);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < ACC_STAGES; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), EPI_WARPS);
+            mbar_init(tempty_bar(a), 2 * EPI_WARPS);       // epilogue warps of both CTAs
         }
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_barrier_init();
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ------------------------------ TMA producer ------------------------------------------
+        // ------------------------------ TMA producer (each CTA loads its own halves) -----------
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
-                const int4 ent = ents[w / n_blocks];
-                const int n_blk = w % n_blocks;
+            for (int w = w_begin; ok && w < w_end; w += w_step) {
+                const int4 it = items[w];
+                const int e = it.x & 0xffff, f = it.x >> 16, n = it.z, half = n >> 1;
+                const CUtensorMap* bmap = &maps.b[(half >> 3) - 1];
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) {
                         ok = false;
                         break;
                     }
                     const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-                    tma_load_2d(sa, &tmA, kb * BK, ent.y, full_bar(stage));
+                    const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
+                    if (rank == 0)                      // bytes of both CTAs: 2 x (A + n/2 rows)
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(2 * A_BYTES + n * BK * 2));
                     if (MODE == 0) {
-                        tma_load_3d(sb, &tmB0, kb * BK, n_blk * (BN / 2), ent.x, full_bar(stage));
-                        tma_load_3d(sb + B_BYTES / 2, &tmB1, kb * BK, n_blk * (BN / 2), ent.x,
-                                    full_bar(stage));
+                        const int f0 = f * FEAT0 + (int)rank * (BMF / 2);
+                        tma_load_3d_pair(sa, &maps.a0, kb * BK, f0, e, lead_full);
+                        tma_load_3d_pair(sa + A_BYTES / 2, &maps.a1, kb * BK, f0, e, lead_full);
                     } else {
-                        tma_load_3d(sb, &tmB0, kb * BK, n_blk * BN, ent.x, full_bar(stage));
+                        tma_load_3d_pair(sa, &maps.a0, kb * BK, f * FEAT1 + (int)rank * BMF, e,
+                                         lead_full);
                     }
+                    tma_load_2d_pair(sb, bmap, kb * BK, it.y + (int)rank * half, lead_full);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            // Tail: every stage's release (signalled from the leader's tensor core, also into the
+            // peer CTA) must have landed before this CTA may leave.
+            for (int s = 0; ok && s < STAGES; ++s) {
+                ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
         }
     } else if (warp == 1) {
-        // ------------------------------ MMA issuer ---------------------------------------------
-        if (lane == 0) {
+        // ------------------------------ MMA issuer (leader CTA only) ---------------------------
+        if (lane == 0 && rank == 0) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int w = blockIdx.x; ok && w < total; w += gridDim.x) {
+            for (int w = w_begin; ok && w < w_end; w += w_step) {
+                const int n = items[w].z;
+                const uint32_t idesc = instr_desc_bf16(2 * BMF, n);
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNT);
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, abort_flag, dev_status)) {
                         ok = false;
@@ -143,69 +278,108 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
 #pragma unroll
                     for (int kk = 0; kk < BK / UK; ++kk) {
                         // 16 bf16 = 32 bytes further along k inside the swizzled row
-                        tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
-                                    kInstrDesc, (kb | kk) != 0 ? 1u : 0u);
+                        tc_mma_bf16_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
+                                         idesc, (kb | kk) != 0 ? 1u : 0u);
                     }
-                    tc_commit(empty_bar(stage));      // frees the stage when these MMAs retire
+                    tc_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(tfull_bar(acc));            // accumulator complete
+                tc_commit_pair(tfull_bar(acc), 3);         // accumulator complete, both CTAs
                 if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
             }
         }
     } else {
         // ------------------------------ epilogue -----------------------------------------------
         const int q = warp & 3;                       // TMEM lane quadrant this warp may read
-        const int half = (warp - 2) >> 2;             // which half of the columns it handles
         int acc = 0;
         uint32_t acc_phase = 0;
-        for (int w = blockIdx.x; w < total; w += gridDim.x) {
-            const int4 ent = ents[w / n_blocks];
-            const int n_blk = w % n_blocks;
-            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status)) break;
+        int chunk_no = 0;
+        bool alive = true;                            // false after a wait ran out: the barrier
+                                                      // protocol goes on, the work is skipped
+        for (int w = w_begin; w < w_end; w += w_step) {
+            const int4 it = items[w];
+            const int f = it.x >> 16, row0 = it.y, n = it.z, valid = it.w;
+            if (alive) {
+                const bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status);
+                alive = __all_sync(0xffffffffu, ok);
+            }
             tc_fence_after();
-            const int r_in = q * 32 + lane;
-            const bool row_ok = r_in < ent.z;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-            __nv_bfloat16* orow = out + (size_t)(ent.y + r_in) * Nout;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BNT);
             if (MODE == 0) {
-                constexpr int HALF_N = BN / 2;        // 128 h columns per tile
+                // Quadrants 0,1 hold the gate rows of features p*32 + lane, quadrants 2,3 the up
+                // rows of the same features.  Per chunk of 32 tokens the two warps swap halves
+                // through shared memory (two buffers, one named barrier per chunk): the gate warp
+                // finishes tokens 0-15, the up warp tokens 16-31.
+                const int p = q & 1;
+                const bool gate = q < 2;
+                float* xpair = reinterpret_cast<float*>(epi_ptr + p * 8192);      // 2 x [2][16][32]
+                __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(epi_ptr + 16384 + q * 1024);
+                const int feat = f * FEAT0 + (int)rank * (BMF / 2) + p * 32 + (lane & 3) * 8;
+                const int own = gate ? 0 : 16;        // first of the 16 tokens this warp finishes
 #pragma unroll 1
-                for (int c = 0; c < HALF_N / 2; c += 32) {
-                    const int col = half * (HALF_N / 2) + c;
-                    float g[32], u[32];
-                    tc_ld32(taddr + col, g);
-                    tc_ld32(taddr + HALF_N + col, u);
-                    tc_wait_ld();
+                for (int c = 0; c < n; c += 32, ++chunk_no) {
+                    float v[32];
+                    if (alive) {
+                        tc_ld32(taddr + c, v);
+                        tc_wait_ld();
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        g[i] = __fdividef(g[i], 1.f + __expf(-g[i])) * u[i];
-                    const int n0 = n_blk * HALF_N + col;
-                    if (row_ok) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 8)
-                            if (n0 + i + 8 <= Nout) store8(orow + n0 + i, g + i);
+                        for (int i = 0; i < 32; ++i) v[i] = 0.f;
                     }
+                    float* xb = xpair + (chunk_no & 1) * 1024;
+                    float* send = xb + (gate ? 0 : 512);
+                    const float* recv = xb + (gate ? 512 : 0);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) send[i * 32 + lane] = gate ? v[16 + i] : v[i];
+                    named_bar_sync(1 + p, 64);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float other = recv[i * 32 + lane];
+                        const float g = gate ? v[i] : other;
+                        const float u = gate ? other : v[16 + i];
+                        hb[i * 32 + lane] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const int tl = (lane >> 2) + 8 * rr;
+                        const uint4 val = *reinterpret_cast<const uint4*>(hb + tl * 32 + (lane & 3) * 8);
+                        const int tok = c + own + tl;
+                        if (alive && tok < valid && feat + 8 <= Nout)
+                            *reinterpret_cast<uint4*>(out + (size_t)(row0 + tok) * Nout + feat) = val;
+                    }
+                    __syncwarp();
                 }
             } else {
+                __nv_bfloat16* tbuf = reinterpret_cast<__nv_bfloat16*>(epi_ptr + q * 2048);
+                const int feat0 = f * FEAT1 + (int)rank * BMF + q * 32;
 #pragma unroll 1
-                for (int c = 0; c < BN / 2; c += 32) {
-                    const int col = half * (BN / 2) + c;
-                    float v[32];
-                    tc_ld32(taddr + col, v);
-                    tc_wait_ld();
-                    const int n0 = n_blk * BN + col;
-                    if (row_ok) {
+                for (int c = 0; c < n; c += 32) {
+                    if (alive) {
+                        float v[32];
+                        tc_ld32(taddr + c, v);
+                        tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; i += 8)
-                            if (n0 + i + 8 <= Nout) store8(orow + n0 + i, v + i);
+                        for (int i = 0; i < 32; ++i) tbuf[i * 32 + lane] = __float2bfloat16_rn(v[i]);
+                        __syncwarp();
+#pragma unroll
+                        for (int rr = 0; rr < 4; ++rr) {
+                            const int tok = (lane >> 2) + 8 * rr;
+                            const uint4 val = *reinterpret_cast<const uint4*>(
+                                tbuf + tok * 32 + (lane & 3) * 8);
+                            const int feat = feat0 + (lane & 3) * 8;
+                            if (c + tok < valid && feat + 8 <= Nout)
+                                *reinterpret_cast<uint4*>(out + (size_t)(row0 + c + tok) * Nout +
+                                                          feat) = val;
+                        }
+                        __syncwarp();
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (lane == 0 && alive) mbar_arrive_cluster(mapa_shared(tempty_bar(acc), 0));
             if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -218,57 +392,138 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA,
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         __syncthreads();
     }
+    cluster_sync_all();            // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                     ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+// Tensor maps of the token operand are encoded once per (pointer, shape) and re-used.
+struct TokenMapCache {
+    const void* ptr = nullptr;
+    uint64_t rows = 0, cols = 0;
+    CUtensorMap b[BNT / 16];
+};
+
+static bool token_maps(TokenMapCache* c, const void* ptr, uint64_t rows, uint64_t cols,
+                       PairMaps* out) {
+    if (c->ptr != ptr || c->rows != rows || c->cols != cols) {
+        for (int i = 0; i < BNT / 16; ++i)
+            if (!make_map_2d(&c->b[i], ptr, rows, cols, 8u * (i + 1))) return false;
+        c->ptr = ptr;
+        c->rows = rows;
+        c->cols = cols;
+    }
+    for (int i = 0; i < BNT / 16; ++i) out->b[i] = c->b[i];
+    return true;
+}
+
+// Number of CTA pairs that can be resident at once (one CTA per SM), cached per device.
+template <typename Kern>
+static int resident_pairs(Kern kern) {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (cached[dev] == 0) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3(2 * (sm_count() / 2));
+        cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = SMEM_BYTES;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return 0;
+        const int by_sm = sm_count() / 2;
+        n = n < by_sm ? n : by_sm;
+        cached[dev] = n < kMaxClusters ? n : kMaxClusters;
+    }
+    return cached[dev];
+}
+
+template <int MODE>
+static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* list, void* out,
+                             int Kdim, int Nout, int32_t* dev_status, cudaStream_t cs) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = cs;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<MODE>, maps, list,
+                              static_cast<__nv_bfloat16*>(out), Kdim, Nout,
+                              dev_status) == cudaSuccess ? R3_OK : R3_ERR_CUDA;
 }
 
 }  // namespace tc
 
-int tc_block_m() { return tc::BM; }
+static long long max_items(long long R, int E, int nf) {
+    return (R / tc::BNT + E) * (long long)nf;       // each expert adds at most one partial tile
+}
+static int feat_tiles_up(const r3_shape* s) { return (s->F + tc::FEAT0 - 1) / tc::FEAT0; }
+static int feat_tiles_down(const r3_shape* s) { return (s->d + tc::FEAT1 - 1) / tc::FEAT1; }
+static size_t list_bytes(long long R, int E, int nf) {
+    return round_up(sizeof(int32_t) * tc::kRangeInts + 16 * (size_t)max_items(R, E, nf), 256);
+}
 
-r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int32_t* tiles,
+size_t tc_work_bytes(const r3_shape* s) {
+    const long long R = (long long)s->T * s->K;
+    return list_bytes(R, s->E, feat_tiles_up(s)) + list_bytes(R, s->E, feat_tiles_down(s));
+}
+
+r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int32_t* offsets,
                                    const void* w_gate, const void* w_up, const void* w_down,
-                                   void* h, void* o, int32_t* dev_status, int phases,
+                                   void* h, void* o, void* work, int32_t* dev_status, int phases,
                                    cudaStream_t cs) {
     using namespace tc;
     const long long R = (long long)s->T * s->K;
-    const int mt = max_m_tiles(R, s->E, BM);
-    if (mt == 0) return R3_OK;
+    if (R == 0) return R3_OK;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(grouped_gemm_tc_kernel<0>,
+        if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<0>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(grouped_gemm_tc_kernel<1>,
+            cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return R3_ERR_CUDA;
         attr_set = true;
     }
-    const int sms = sm_count();
+    const int pairs = resident_pairs(grouped_gemm_pair_kernel<0>);
+    if (pairs <= 0) return R3_ERR_CUDA;
+    const int nf0 = feat_tiles_up(s), nf1 = feat_tiles_down(s);
+    int32_t* list0 = static_cast<int32_t*>(work);
+    int32_t* list1 = reinterpret_cast<int32_t*>(static_cast<char*>(work) +
+                                                list_bytes(R, s->E, nf0));
+    static TokenMapCache cache_xp, cache_h;
     if (phases & kPhaseUp) {
-        CUtensorMap m_xp, m_g, m_u;
-        if (!make_map_2d(&m_xp, xp, (uint64_t)R, (uint64_t)s->d, BM) ||
-            !make_map_3d(&m_g, w_gate, s->E, s->F, s->d, BN / 2) ||
-            !make_map_3d(&m_u, w_up, s->E, s->F, s->d, BN / 2))
+        build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, pairs, list0, list1);
+        PairMaps m;
+        if (!make_map_3d(&m.a0, w_gate, s->E, s->F, s->d, BMF / 2) ||
+            !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2) ||
+            !token_maps(&cache_xp, xp, (uint64_t)R, (uint64_t)s->d, &m))
             return R3_ERR_CUDA;
-        const int nb1 = (s->F + BN / 2 - 1) / (BN / 2);
-        const long long t1 = (long long)mt * nb1;
-        const int g1 = (int)(t1 < sms ? t1 : sms);
-        grouped_gemm_tc_kernel<0><<<g1, THREADS, SMEM_BYTES, cs>>>(
-            m_xp, m_g, m_u, tiles, static_cast<__nv_bfloat16*>(h), s->d, s->F, nb1, dev_status);
+        const r3_status st = launch_pair<0>(m, pairs, list0, h, s->d, s->F, dev_status, cs);
+        if (st != R3_OK) return st;
     }
     if (phases & kPhaseDown) {
-        CUtensorMap m_h, m_d;
-        if (!make_map_2d(&m_h, h, (uint64_t)R, (uint64_t)s->F, BM) ||
-            !make_map_3d(&m_d, w_down, s->E, s->d, s->F, BN))
+        PairMaps m;
+        if (!make_map_3d(&m.a0, w_down, s->E, s->d, s->F, BMF) ||
+            !token_maps(&cache_h, h, (uint64_t)R, (uint64_t)s->F, &m))
             return R3_ERR_CUDA;
-        const int nb2 = (s->d + BN - 1) / BN;
-        const long long t2 = (long long)mt * nb2;
-        const int g2 = (int)(t2 < sms ? t2 : sms);
-        grouped_gemm_tc_kernel<1><<<g2, THREADS, SMEM_BYTES, cs>>>(
-            m_h, m_d, m_d, tiles, static_cast<__nv_bfloat16*>(o), s->F, s->d, nb2, dev_status);
+        m.a1 = m.a0;
+        const r3_status st = launch_pair<1>(m, pairs, list1, o, s->F, s->d, dev_status, cs);
+        if (st != R3_OK) return st;
     }
     return launch_status();
 }
