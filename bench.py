@@ -239,7 +239,7 @@ def run_ours(args, w):
 
     # ---- per-kernel segments (same kernels through the per-step entry points, events between) --
     seg_names = ["logits", "gate_fwd", "permute", "expert_up_swiglu", "expert_down", "combine",
-                 "dgates", "gate_bwd"]
+                 "dgates", "gate_bwd", "finish_fused"]
     logits = torch.empty((T, E), dtype=torch.float32, device=dev)
     dg = torch.empty((T, K), dtype=torch.float32, device=dev)
     pout = (torch.empty(E, dtype=torch.int32, device=dev),
@@ -273,6 +273,10 @@ def run_ours(args, w):
         e[7].record()
         r3.replay_gate_bwd(s, gates, dg, idx, dlogits=dlogits)
         e[8].record()
+        # what r3_replay_layer runs instead of gate_fwd + combine + dgates + gate_bwd (K <= 8)
+        r3.replay_finish(s, logits, idx, o, pout[2], dy, y=y, gates=gates, dlogits=dlogits,
+                         dev_status=st)
+        e[9].record()
 
     for _ in range(3):
         seg_step(evs[0])
@@ -289,6 +293,7 @@ def run_ours(args, w):
         "combine": T * (K * d * es + K * 8 + d * es),
         "dgates": T * (d * es + K * d * es + K * 4 + K * 4),
         "gate_bwd": T * (K * 9 + E * 4),
+        "finish_fused": T * (K * d * es + 2 * d * es + K * 9 + K * 4 + E * 4),
     }
     flops = {"expert_up_swiglu": 4.0 * R * d * F, "expert_down": 2.0 * R * d * F,
              "logits": 2.0 * T * d * E}

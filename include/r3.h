@@ -193,6 +193,24 @@ r3_status r3_combine_residual(const r3_shape* shape, const void* o, const int32_
 r3_status r3_combine_bwd_gates(const r3_shape* shape, const void* dy, const void* o,
                                const int32_t* row_of_slot, float* dgates, void* stream);
 
+/* Everything that follows the expert networks, in one pass over the expert outputs: the replay
+ * gate of Eq. (replay_gate), the combine of Eq. (replay_output), the gate gradient and the
+ * router-logit gradient (Section 4.1, purpose (b): the mask is a constant).  Per token,
+ *   g      = softmax of logits[t, idx[t, .]]                       (as r3_replay_gate_fwd)
+ *   y[t]   = residual[t] + sum_j g_j o[row_of_slot[t,j]]           (as r3_combine_residual)
+ *   dg_j   = <dy[t], o[row_of_slot[t,j]]>                          (as r3_combine_bwd_gates)
+ *   dlogits[t, idx[t,j]] = g_j (dg_j - sum_j' g_j' dg_j'), 0 elsewhere   (as r3_replay_gate_bwd)
+ * with the same arithmetic and summation orders as those four calls, so y, gates and dlogits are
+ * bit-identical to theirs, but each expert-output row is read once instead of twice.
+ * logits [T,E] f32; idx [T,K]; o [R,d]; row_of_slot [T,K]; dy [T,d]; residual [T,d] or NULL;
+ * outputs y [T,d], gates_out [T,K] f32 or NULL, dlogits [T,E] f32 (every element written).
+ * Supported for K <= 8 (R3_ERR_UNSUPPORTED beyond; use the four calls).  dev_status as for
+ * r3_replay_gate_fwd. */
+r3_status r3_replay_finish(const r3_shape* shape, const float* logits, const void* idx,
+                           const void* o, const int32_t* row_of_slot, const void* dy,
+                           const void* residual, void* y, float* gates_out, float* dlogits,
+                           int32_t* dev_status, void* stream);
+
 /* The whole replayed layer, forward and router-logit backward, enqueued back to back on one
  * stream: logits -> replay gate -> permute -> experts -> combine -> dgates -> dlogits.
  * Inputs x [T,d], w_router [E,d], idx [T,K], expert weights, dy [T,d];

@@ -1,0 +1,231 @@
+// One pass over the expert outputs that does everything after the expert networks:
+//   replay gate (Eq. replay_gate)            g[t,j]  = softmax over the K recorded logits
+//   combine     (Eq. replay_output)          y[t]    = sum_j g[t,j] o[row_of_slot[t,j]] (+ residual)
+//   gate gradient                            dg[t,j] = <dy[t], o[row_of_slot[t,j]]>
+//   router-logit gradient                    ds[t,e_j] = g_j (dg_j - sum_j' g_j' dg_j'), 0 elsewhere
+// The separate kernels (r3_replay_gate_fwd, r3_combine, r3_combine_bwd_gates, r3_replay_gate_bwd)
+// read every expert-output row twice and need four launches; here a team of threads owns a token,
+// gathers its K rows once, and keeps the same arithmetic and the same summation orders as those
+// kernels, so the results are bit-identical to theirs.  No atomics.
+#include "r3_common.cuh"
+
+namespace r3 {
+
+constexpr int kFusedMaxK = 8;     // slots held in registers per thread
+
+template <typename ActT, typename IdxT, int TPT>
+__global__ void __launch_bounds__(256, 3)
+replay_finish_kernel(const float* __restrict__ logits, const IdxT* __restrict__ idx,
+                     const ActT* __restrict__ o, const int32_t* __restrict__ row_of_slot,
+                     const ActT* __restrict__ dy, const ActT* __restrict__ residual,
+                     ActT* __restrict__ y, float* __restrict__ gates_out,
+                     float* __restrict__ dlogits, int T, int E, int K, int d, int W,
+                     int32_t* dev_status) {
+    using V = Vec16<ActT>;
+    constexpr int N = V::N;
+    constexpr int TEAMS = 256 / TPT;
+    constexpr int WPT = TPT / 32;                      // warps per team
+    __shared__ float g_s[TEAMS][kFusedMaxK];
+    __shared__ float dg_s[TEAMS][kFusedMaxK];
+    __shared__ float part[256 / 32][kFusedMaxK];
+
+    const int team = threadIdx.x / TPT, tl = threadIdx.x % TPT;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * TEAMS + team;
+    const bool live = t < T;                           // no early exit: block-wide barriers below
+    const int tt = live ? t : T - 1;
+    const IdxT* rec = idx + (size_t)tt * K;
+
+    // The K row gathers of the first column piece do not depend on the gates: they are issued
+    // first, so that they are in flight while the team's first warp works out the gates.
+    const int row_vecs = d / N;
+    const int32_t* rows = row_of_slot + (size_t)tt * K;
+    const V* ov = reinterpret_cast<const V*>(o);
+    const V* dyv = reinterpret_cast<const V*>(dy) + (size_t)tt * row_vecs;
+    V* yv = reinterpret_cast<V*>(y) + (size_t)tt * row_vecs;
+    unsigned have = 0;                                  // bit u: slot u has a row
+    V v[kFusedMaxK], dv;
+    {
+        int32_t r[kFusedMaxK];
+#pragma unroll
+        for (int u = 0; u < kFusedMaxK; ++u) {
+            r[u] = u < K ? rows[u] : -1;
+            if (r[u] >= 0) have |= 1u << u;
+        }
+        if (tl < row_vecs) {
+#pragma unroll
+            for (int u = 0; u < kFusedMaxK; ++u)
+                if (r[u] >= 0) v[u] = ov[(size_t)r[u] * row_vecs + tl];
+            dv = dyv[tl];
+        }
+    }
+
+    // ---- replay gate: the first W lanes of the team, one slot each (K <= W <= 32) ------------
+    int my_e = -1;
+    if (tl < 32) {
+        const float* row = logits + (size_t)tt * E;
+        int bad = 0;
+        float s = -INFINITY;
+        if (tl < K) {
+            my_e = idx_to_int(rec[tl]);
+            if (my_e < 0 || my_e >= E) bad |= 1;
+            for (int j2 = 0; j2 < tl; ++j2)
+                if (idx_to_int(rec[j2]) == my_e) bad |= 2;
+            s = row[min(max(my_e, 0), E - 1)];
+        }
+        for (int ofs = W / 2; ofs > 0; ofs >>= 1) bad |= __shfl_xor_sync(0xffffffffu, bad, ofs, W);
+        if (bad && live && tl == 0)
+            report(dev_status, (bad & 1) ? R3_DEV_BAD_INDEX : R3_DEV_DUP_INDEX);
+        float m = s;
+        for (int ofs = W / 2; ofs > 0; ofs >>= 1)
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, ofs, W));
+        const float ex = tl < K ? expf(s - m) : 0.f;
+        float sum = ex;
+        for (int ofs = W / 2; ofs > 0; ofs >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, ofs, W);
+        const float inv = bad ? 0.f : 1.f / sum;
+        if (tl < K) {
+            const float g = ex * inv;
+            g_s[team][tl] = g;
+            if (gates_out && live) gates_out[(size_t)t * K + tl] = g;
+        }
+    }
+    __syncthreads();
+
+    // ---- combine and <dy, o_j> from the gathered rows -------------------------------------------
+    float dacc[kFusedMaxK];
+#pragma unroll
+    for (int u = 0; u < kFusedMaxK; ++u) dacc[u] = 0.f;
+    for (int c = tl; c < row_vecs; c += TPT) {
+        if (c != tl) {                       // later column pieces (d wider than one pass)
+#pragma unroll
+            for (int u = 0; u < kFusedMaxK; ++u)
+                if (have >> u & 1u) v[u] = ov[(size_t)rows[u] * row_vecs + c];
+            dv = dyv[c];
+        }
+        float gr[N];
+        dv.unpack(gr);
+        float acc[N];
+#pragma unroll
+        for (int i = 0; i < N; ++i) acc[i] = 0.f;
+#pragma unroll
+        for (int u = 0; u < kFusedMaxK; ++u) {
+            if (have >> u & 1u) {
+                const float gu = g_s[team][u];
+                float f[N];
+                v[u].unpack(f);
+#pragma unroll
+                for (int i = 0; i < N; ++i) acc[i] = fmaf(gu, f[i], acc[i]);
+#pragma unroll
+                for (int i = 0; i < N; ++i) dacc[u] = fmaf(gr[i], f[i], dacc[u]);
+            }
+        }
+        if (residual) {                      // y = residual + sum (one extra fp32 add per element)
+            float f[N];
+            reinterpret_cast<const V*>(residual)[(size_t)tt * row_vecs + c].unpack(f);
+#pragma unroll
+            for (int i = 0; i < N; ++i) acc[i] += f[i];
+        }
+        if (live) {
+            V out;
+            out.pack(acc);
+            yv[c] = out;
+        }
+    }
+
+    // ---- dg: warp shuffles, then the team's warps in a fixed order ------------------------------
+#pragma unroll
+    for (int u = 0; u < kFusedMaxK; ++u) {
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) dacc[u] += __shfl_xor_sync(0xffffffffu, dacc[u], s);
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int u = 0; u < kFusedMaxK; ++u) part[warp][u] = dacc[u];
+    }
+    __syncthreads();
+    if (tl < kFusedMaxK) {
+        float s = 0.f;
+        for (int w = 0; w < WPT; ++w) s += part[team * WPT + w][tl];   // fixed order
+        dg_s[team][tl] = s;
+    }
+    __syncthreads();
+
+    // ---- router-logit gradient: the team's first warp writes the dense row once ----------------
+    if (tl < 32 && live) {
+        const float g = tl < K ? g_s[team][tl] : 0.f;
+        const float dg = tl < K ? dg_s[team][tl] : 0.f;
+        float c = g * dg;
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) c += __shfl_xor_sync(0xffffffffu, c, s);
+        const float v = g * (dg - c);
+        float* out = dlogits + (size_t)t * E;
+        const int nchunk = (E + 3) >> 2;
+        for (int ch = tl; ch < ((nchunk + 31) & ~31); ch += 32) {
+            float q[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < K; ++j) {
+                const int ej = __shfl_sync(0xffffffffu, my_e, j);
+                const float vj = __shfl_sync(0xffffffffu, v, j);
+                if ((ej >> 2) == ch) q[ej & 3] = vj;
+            }
+            if (ch < nchunk) {
+                const int e0 = ch << 2;
+                if (e0 + 3 < E && (E & 3) == 0) {
+                    *reinterpret_cast<float4*>(out + e0) = make_float4(q[0], q[1], q[2], q[3]);
+                } else {
+                    for (int i = 0; i < 4 && e0 + i < E; ++i) out[e0 + i] = q[i];
+                }
+            }
+        }
+    }
+}
+
+static int pick_team_fused(int row_vecs) {
+    int tpt = 32;
+    while (tpt < 256 && tpt < row_vecs) tpt <<= 1;
+    return tpt;
+}
+
+template <typename ActT, typename IdxT>
+static void launch_finish(const r3_shape* s, const float* logits, const void* idx, const void* o,
+                          const int32_t* row_of_slot, const void* dy, const void* residual,
+                          void* y, float* gates_out, float* dlogits, int32_t* dev_status,
+                          cudaStream_t cs) {
+    const int T = s->T, K = s->K, d = s->d, E = s->E;
+    int W = 1;
+    while (W < K && W < 32) W <<= 1;
+    const int tpt = pick_team_fused(d / Vec16<ActT>::N);
+    const unsigned grid = (unsigned)((T + 256 / tpt - 1) / (256 / tpt));
+#define R3_FIN(TPT)                                                                              \
+    replay_finish_kernel<ActT, IdxT, TPT><<<grid, 256, 0, cs>>>(                                 \
+        logits, static_cast<const IdxT*>(idx), static_cast<const ActT*>(o), row_of_slot,         \
+        static_cast<const ActT*>(dy), static_cast<const ActT*>(residual), static_cast<ActT*>(y), \
+        gates_out, dlogits, T, E, K, d, W, dev_status)
+    switch (tpt) {
+        case 32: R3_FIN(32); break;
+        case 64: R3_FIN(64); break;
+        case 128: R3_FIN(128); break;
+        default: R3_FIN(256); break;
+    }
+#undef R3_FIN
+}
+
+}  // namespace r3
+
+extern "C" r3_status r3_replay_finish(const r3_shape* shape, const float* logits, const void* idx,
+                                      const void* o, const int32_t* row_of_slot, const void* dy,
+                                      const void* residual, void* y, float* gates_out,
+                                      float* dlogits, int32_t* dev_status, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->K > r3::kFusedMaxK) return R3_ERR_UNSUPPORTED;
+    if (shape->T == 0) return R3_OK;
+    if (!logits || !idx || !o || !row_of_slot || !dy || !y || !dlogits) return R3_ERR_INVALID_ARG;
+    if (!r3::aligned(o, 16) || !r3::aligned(dy, 16) || !r3::aligned(y, 16) ||
+        !r3::aligned(residual, 16))
+        return R3_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    R3_DISPATCH_ACT(shape, ActT, R3_DISPATCH_IDX(shape, IdxT,
+        (r3::launch_finish<ActT, IdxT>(shape, logits, idx, o, row_of_slot, dy, residual, y,
+                                       gates_out, dlogits, dev_status, cs))));
+    return r3::launch_status();
+}

@@ -75,7 +75,11 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
     if ((st = r3_capture_topk_ws(shape, 1, x, w_router, nullptr, w.logits, w.router_ws,
                                  w.router_bytes, stream)) != R3_OK)
         return st;
-    if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
+    // K <= 8: gate, combine and both gradients in one pass over the expert outputs; wider records
+    // take the four separate kernels (same results).
+    const bool fused = shape->K <= 8;
+    if (!fused &&
+        (st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
         return st;
     if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
                          w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
@@ -83,6 +87,9 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
     if ((st = r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, w.swiglu_ws,
                                 w.swiglu_bytes, dev_status, stream)) != R3_OK)
         return st;
+    if (fused)
+        return r3_replay_finish(shape, w.logits, idx, w.o, w.row_of_slot, dy, residual, y,
+                                gates_out, dlogits, dev_status, stream);
     if ((st = r3_combine_residual(shape, w.o, w.row_of_slot, gates, residual, y, stream)) != R3_OK)
         return st;
     if ((st = r3_combine_bwd_gates(shape, dy, w.o, w.row_of_slot, w.dgates, stream)) != R3_OK)

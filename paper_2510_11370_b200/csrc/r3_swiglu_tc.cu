@@ -17,9 +17,11 @@
 // features, so lanes 0-63 hold the gate pre-activations and lanes 64-127 the up projections; the
 // epilogue exchanges them through shared memory to form the SwiGLU product.
 //
-// Items are ordered (expert, feature tile, token tile) so that consecutive items re-use a weight
-// tile from L2, and are dealt to the clusters as contiguous ranges of equal estimated cost
-// (build_work_kernel), so each cluster walks its own range with no atomics.
+// Items are ordered (expert, feature tile, token tile) and dealt to the clusters round-robin, so
+// the clusters running at any moment work on neighbouring items: their copies of a shared weight
+// tile or token tile meet in L2, and the weights stream from HBM once.  (Handing the items out
+// from a device counter instead balanced the clusters better but drained the copy ring at every
+// item boundary, because the peer CTA learns its next item late; it was slower.)
 //
 // Roles (192 threads per CTA): warp 0 lane 0 = TMA producer (both CTAs, into a 6-stage ring of
 // 128B-swizzled tiles), warp 1 lane 0 of the leader CTA = MMA issuer (two accumulator stages of
@@ -53,7 +55,6 @@ constexpr int BAR_BYTES = 256;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + 1024;  // + alignment
 constexpr int FEAT0 = BMF;         // h features per item in MODE 0 (64 per CTA, gate + up rows)
 constexpr int FEAT1 = 2 * BMF;     // o features per item in MODE 1
-constexpr int kMaxClusters = 254;
 
 // Tensor maps of one launch.  b[i] loads a token box of 8 * (i + 1) rows.
 struct alignas(64) PairMaps {
@@ -62,115 +63,66 @@ struct alignas(64) PairMaps {
 };
 
 // ---- work list -------------------------------------------------------------------------------
-// Per list: int32 ranges[kRangeInts] (ranges[p] .. ranges[p+1] = items of cluster p), then one
-// int4 per item = {expert | feature tile << 16, first row, N (multiple of 16), valid rows}.
-constexpr int kRangeInts = 256;
+// Per list: int32 header[kHeaderInts] = {number of items, ...}, then one int4 per item =
+// {expert | feature tile << 16, first row, N (multiple of 16), valid rows}, ordered
+// (expert, feature tile, token tile).  An expert with cnt rows is cut into nt = ceil(cnt / 256)
+// token tiles of equal size q (rounded up to 16; the last one holds what is left).
+constexpr int kHeaderInts = 4;
 
 __host__ __device__ inline int split_tiles(int cnt) { return (cnt + BNT - 1) / BNT; }
 __host__ __device__ inline int split_rows(int cnt, int nt) {      // rows per tile, multiple of 16
     return (((cnt + nt - 1) / nt) + 15) & ~15;
 }
-// Estimated duration of an item in units of one token column of MMA time: the MMA time grows
-// with N, but below about 128 columns the weight tile's load time dominates.
-__host__ __device__ inline int item_cost(int n) { return (n < 128 ? 128 : n) + 24; }
-
-struct ExpertSplit {
-    int lo, cnt, nt, q, n_last;
-    long long cost_f;              // cost of the expert's token tiles for one feature tile
-};
-__device__ __forceinline__ ExpertSplit split_of(const int32_t* offsets, int e) {
-    ExpertSplit s;
-    s.lo = offsets[e];
-    s.cnt = offsets[e + 1] - s.lo;
-    s.nt = split_tiles(s.cnt);
-    s.q = s.nt ? split_rows(s.cnt, s.nt) : 0;
-    s.n_last = s.nt ? ((s.cnt - (s.nt - 1) * s.q + 15) & ~15) : 0;
-    s.cost_f = s.nt ? (long long)(s.nt - 1) * item_cost(s.q) + item_cost(s.n_last) : 0;
-    return s;
-}
 
 // One CTA per list (blockIdx.x = 0: up projection with nf0 feature tiles, 1: down with nf1).
 __global__ void __launch_bounds__(1024)
-build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1, int P,
+build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
                   int32_t* __restrict__ list0, int32_t* __restrict__ list1) {
     __shared__ int32_t s_items[1025];
-    __shared__ long long s_cost[1025];
     __shared__ int32_t w_items[32];
-    __shared__ long long w_cost[32];
     const int nf = blockIdx.x == 0 ? nf0 : nf1;
-    int32_t* ranges = blockIdx.x == 0 ? list0 : list1;
-    int4* items = reinterpret_cast<int4*>(ranges + kRangeInts);
+    int32_t* list = blockIdx.x == 0 ? list0 : list1;
+    int4* items = reinterpret_cast<int4*>(list + kHeaderInts);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    int32_t my_items = 0;
-    long long my_cost = 0;
-    if (tid < E) {
-        const ExpertSplit s = split_of(offsets, tid);
-        my_items = s.nt * nf;
-        my_cost = s.cost_f * nf;
-    }
+    const int32_t my_items = tid < E ? split_tiles(offsets[tid + 1] - offsets[tid]) * nf : 0;
     int32_t ii = my_items;
-    long long cc = my_cost;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int32_t a = __shfl_up_sync(0xffffffffu, ii, o);
-        const long long b = __shfl_up_sync(0xffffffffu, cc, o);
-        if (lane >= o) { ii += a; cc += b; }
+        if (lane >= o) ii += a;
     }
-    if (lane == 31) { w_items[warp] = ii; w_cost[warp] = cc; }
+    if (lane == 31) w_items[warp] = ii;
     __syncthreads();
     if (warp == 0) {
         const int32_t a0 = w_items[lane];
-        const long long b0 = w_cost[lane];
         int32_t a = a0;
-        long long b = b0;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int32_t x = __shfl_up_sync(0xffffffffu, a, o);
-            const long long y = __shfl_up_sync(0xffffffffu, b, o);
-            if (lane >= o) { a += x; b += y; }
+            if (lane >= o) a += x;
         }
         w_items[lane] = a - a0;
-        w_cost[lane] = b - b0;
     }
     __syncthreads();
-    s_items[tid] = w_items[warp] + ii - my_items;      // exclusive prefixes
-    s_cost[tid] = w_cost[warp] + cc - my_cost;
-    if (tid == 1023) { s_items[1024] = w_items[warp] + ii; s_cost[1024] = w_cost[warp] + cc; }
+    s_items[tid] = w_items[warp] + ii - my_items;      // exclusive prefix
+    if (tid == 1023) s_items[1024] = w_items[warp] + ii;
     __syncthreads();
     const int32_t I = s_items[1024];
-    const long long C = s_cost[1024];
-
-    // start cost, owner cluster and fields of item i
-    auto describe = [&](int32_t i, int4* out) -> int {
+    if (tid == 0) list[0] = I;
+    for (int32_t i = tid; i < I; i += 1024) {
         int lo = 0, hi = E;                      // last e with s_items[e] <= i
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if (s_items[mid] <= i) lo = mid; else hi = mid;
         }
         const int e = lo;
-        const ExpertSplit s = split_of(offsets, e);
+        const int row_lo = offsets[e], cnt = offsets[e + 1] - row_lo;
+        const int nt = split_tiles(cnt), q = split_rows(cnt, nt);
         const int k = i - s_items[e];
-        const int f = k / s.nt, j = k - f * s.nt;
-        const long long cs = s_cost[e] + (long long)f * s.cost_f + (long long)j * item_cost(s.q);
-        if (out) {
-            const int n = (j == s.nt - 1) ? s.n_last : s.q;
-            const int valid = min(s.q, s.cnt - j * s.q);
-            *out = make_int4(e | (f << 16), s.lo + j * s.q, n, valid);
-        }
-        int owner = (int)((cs * P) / C);
-        return owner < P ? owner : P - 1;
-    };
-    for (int32_t i = tid; i < I; i += 1024) {
-        int4 it;
-        const int owner = describe(i, &it);
-        items[i] = it;
-        const int prev = i == 0 ? -1 : describe(i - 1, nullptr);
-        for (int p = prev + 1; p <= owner; ++p) ranges[p] = i;
-    }
-    if (tid == 0) {
-        const int last = I > 0 ? describe(I - 1, nullptr) : -1;
-        for (int p = last + 1; p <= P; ++p) ranges[p] = I;
+        const int f = k / nt, j = k - f * nt;
+        const int valid = min(q, cnt - j * q);
+        items[i] = make_int4(e | (f << 16), row_lo + j * q, (valid + 15) & ~15, valid);
     }
 }
 
@@ -197,8 +149,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
     const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
     const int pair = blockIdx.x >> 1;
     const int w_step = gridDim.x >> 1;
-    const int w_begin = pair, w_end = list[w_step];
-    const int4* items = reinterpret_cast<const int4*>(list + kRangeInts);
+    const int w_begin = pair, w_end = list[0];
+    const int4* items = reinterpret_cast<const int4*>(list + kHeaderInts);
     const int kblocks = (Kdim + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
@@ -442,7 +394,7 @@ static int resident_pairs(Kern kern) {
         if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) return 0;
         const int by_sm = sm_count() / 2;
         n = n < by_sm ? n : by_sm;
-        cached[dev] = n < kMaxClusters ? n : kMaxClusters;
+        cached[dev] = n;
     }
     return cached[dev];
 }
@@ -475,7 +427,7 @@ static long long max_items(long long R, int E, int nf) {
 static int feat_tiles_up(const r3_shape* s) { return (s->F + tc::FEAT0 - 1) / tc::FEAT0; }
 static int feat_tiles_down(const r3_shape* s) { return (s->d + tc::FEAT1 - 1) / tc::FEAT1; }
 static size_t list_bytes(long long R, int E, int nf) {
-    return round_up(sizeof(int32_t) * tc::kRangeInts + 16 * (size_t)max_items(R, E, nf), 256);
+    return round_up(sizeof(int32_t) * tc::kHeaderInts + 16 * (size_t)max_items(R, E, nf), 256);
 }
 
 size_t tc_work_bytes(const r3_shape* s) {
@@ -507,7 +459,7 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int3
                                                 list_bytes(R, s->E, nf0));
     static TokenMapCache cache_xp, cache_h;
     if (phases & kPhaseUp) {
-        build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, pairs, list0, list1);
+        build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1);
         PairMaps m;
         if (!make_map_3d(&m.a0, w_gate, s->E, s->F, s->d, BMF / 2) ||
             !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2) ||

@@ -30,7 +30,8 @@ EXPORTS = [
     "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute", "r3_permute_static",
     "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_expert_up_swiglu",
     "r3_expert_down", "r3_combine",
-    "r3_combine_residual", "r3_combine_bwd_gates", "r3_replay_layer_workspace_bytes",
+    "r3_combine_residual", "r3_combine_bwd_gates", "r3_replay_finish",
+    "r3_replay_layer_workspace_bytes",
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
 ]
@@ -68,6 +69,7 @@ lib.r3_combine_residual.argtypes = [_SP, _P, _P, _P, _P, _P, _P]
 lib.r3_replay_blocks.argtypes = [_SP, ctypes.c_int32] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_stack.argtypes = [_SP, ctypes.c_int32] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
+lib.r3_replay_finish.argtypes = [_SP] + [_P] * 11
 lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_layer_host.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 for _n in EXPORTS:
@@ -336,6 +338,23 @@ def combine_bwd_gates(s: Shape, dy, o, row_of_slot, dgates=None, stream=None):
     _check(lib.r3_combine_bwd_gates(ctypes.byref(s), _ptr(dy), _ptr(o), _ptr(row_of_slot),
                                     _ptr(dgates), _stream(stream)))
     return dgates
+
+
+def replay_finish(s: Shape, logits, idx, o, row_of_slot, dy, *, residual=None, y=None, gates=None,
+                  dlogits=None, dev_status=None, stream=None):
+    """Replay gate + combine + gate gradient + router-logit gradient in one pass over `o`
+    (K <= 8).  Returns (y, gates, dlogits)."""
+    dev = _dev(o)
+    if y is None:
+        y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    if gates is None:
+        gates = torch.empty((s.T, s.K), dtype=torch.float32, device=dev)
+    if dlogits is None:
+        dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
+    _check(lib.r3_replay_finish(ctypes.byref(s), _ptr(logits), _ptr(idx), _ptr(o),
+                                _ptr(row_of_slot), _ptr(dy), _ptr(residual), _ptr(y), _ptr(gates),
+                                _ptr(dlogits), _ptr(dev_status), _stream(stream)))
+    return y, gates, dlogits
 
 
 def replay_layer_workspace_bytes(s: Shape) -> int:

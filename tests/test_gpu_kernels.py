@@ -135,6 +135,71 @@ def test_combine_and_dgates(r3, T, K, d, act, tol):
     assert torch.equal(y, y2)
 
 
+# ------------------------------------------------------------------ fused finish
+@pytest.mark.parametrize("T,E,K,d,act,tol,residual", [
+    (37, 8, 2, 128, torch.float32, TOL_F32, False),
+    (300, 128, 8, 2048, torch.bfloat16, TOL_BF16, False),
+    (129, 16, 3, 72, torch.bfloat16, TOL_BF16, True),
+    (513, 10, 8, 520, torch.float32, TOL_F32, True),
+    (1, 4, 1, 8, torch.bfloat16, TOL_BF16, False),
+])
+def test_replay_finish_matches_the_four_kernels_and_the_oracle(r3, T, E, K, d, act, tol, residual):
+    """Gate + combine + both gradients in one pass: bit-identical to the four separate calls, and
+    within tolerance of the oracle's Eq. replay_gate / replay_output / gradient."""
+    rng = np.random.default_rng(T + K)
+    idx_t = random_record(rng, T, E, K, torch.uint8)
+    idx_np = idx_t.to(torch.int64).numpy()
+    _, _, ros, _ = O.permutation(idx_np, E)
+    logits = (torch.randn(T, E) * 2).float()
+    o = torch.randn(T * K, d).to(act)
+    dy = torch.randn(T, d).to(act)
+    res = torch.randn(T, d).to(act) if residual else None
+    s = r3.make_shape(T, d, E, K, 8, act=act)
+    ros_c = torch.from_numpy(ros).cuda()
+    st = r3.new_status("cuda")
+    y, g, ds = r3.replay_finish(s, logits.cuda(), idx_t.cuda(), o.cuda(), ros_c, dy.cuda(),
+                                residual=None if res is None else res.cuda(), dev_status=st)
+    assert st.item() == 0
+    # the four kernels
+    g4 = r3.replay_gate_fwd(s, logits.cuda(), idx_t.cuda())
+    y4 = (r3.combine_residual(s, o.cuda(), ros_c, g4, res.cuda()) if residual
+          else r3.combine(s, o.cuda(), ros_c, g4))
+    dg4 = r3.combine_bwd_gates(s, dy.cuda(), o.cuda(), ros_c)
+    ds4 = r3.replay_gate_bwd(s, g4, dg4, idx_t.cuda())
+    assert torch.equal(g, g4) and torch.equal(y, y4) and torch.equal(ds, ds4)
+    # the oracle
+    g_ref = O.replay_gate(f64(logits), idx_np)
+    eo = f64(o)[ros.astype(np.int64)]
+    y_ref = np.einsum("tk,tkd->td", g_ref, eo) + (f64(res) if residual else 0.0)
+    ds_ref = O.replay_gate_bwd(g_ref, O.dgates(f64(dy), eo), idx_np, E)
+    assert rel_err(f64(g), g_ref) < TOL_F32
+    assert rel_err(f64(y), y_ref) < tol
+    assert rel_err(f64(ds), ds_ref) < max(tol, TOL_F32 * 10)
+
+
+def test_replay_finish_flags_bad_records_and_rejects_wide_k(r3):
+    T, E, K, d = 64, 16, 4, 64
+    rng = np.random.default_rng(5)
+    idx = random_record(rng, T, E, K, torch.uint8)
+    idx[3, 1] = idx[3, 0]                               # duplicate
+    _, _, ros, _ = O.permutation(random_record(rng, T, E, K, torch.int64).numpy(), E)
+    s = r3.make_shape(T, d, E, K, 8)
+    st = r3.new_status("cuda")
+    y, g, ds = r3.replay_finish(s, torch.randn(T, E).cuda(), idx.cuda(),
+                                torch.randn(T * K, d).bfloat16().cuda(),
+                                torch.from_numpy(ros).cuda(), torch.randn(T, d).bfloat16().cuda(),
+                                dev_status=st)
+    assert st.item() == r3.DEV_DUP_INDEX
+    assert torch.all(g[3] == 0) and torch.all(ds[3] == 0) and torch.all(y[3] == 0)
+    wide = r3.make_shape(T, d, E, 12, 8)
+    with pytest.raises(r3.R3Error) as ei:
+        r3.replay_finish(wide, torch.randn(T, E).cuda(), torch.zeros(T, 12, dtype=torch.uint8).cuda(),
+                         torch.randn(T * 12, d).bfloat16().cuda(),
+                         torch.zeros(T, 12, dtype=torch.int32).cuda(),
+                         torch.randn(T, d).bfloat16().cuda())
+    assert ei.value.code == 2
+
+
 # ------------------------------------------------------------------ capture: logits + TopKMask
 @pytest.mark.parametrize("act,rw", [(torch.float32, torch.float32), (torch.bfloat16, torch.float32),
                                     (torch.bfloat16, torch.bfloat16)])
