@@ -7,7 +7,11 @@
 // read every expert-output row twice and need four launches; here a team of threads owns a token,
 // gathers its K rows once, and keeps the same arithmetic and the same summation orders as those
 // kernels, so the results are bit-identical to theirs.  No atomics.
+#include <algorithm>
+
 #include "r3_common.cuh"
+#include "r3_internal.h"
+#include "r3_tc.cuh"
 
 namespace r3 {
 
@@ -179,6 +183,198 @@ replay_finish_kernel(const float* __restrict__ logits, const IdxT* __restrict__ 
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same computation with the token's rows staged in shared memory: one CTA of 4 warps per
+// token.  At its start the CTA asks for the token's K expert-output rows, its dy row and its
+// residual row with bulk asynchronous copies (one lane and one copy per row, completion counted on
+// an mbarrier); the data in flight lives in shared memory instead of registers, so six CTAs fit
+// on an SM and keep about 200 KB of copies per SM in flight while the first warp works out the
+// gates from the logits.  The four warps then split the columns.
+// y and the gates are bit-identical to the separate kernels (same per-element order); the gate
+// gradient is summed per lane over the columns, across the warp and then over the four warps,
+// a different (fixed) order than r3_combine_bwd_gates, so dlogits agrees with the separate
+// kernels to rounding.
+// ---------------------------------------------------------------------------------------------
+constexpr int kTokWarps = 4;
+constexpr int kTokThreads = kTokWarps * 32;
+constexpr int kTokHeader = 128;           // mbarrier, flags, gates, partial sums
+constexpr int kTokSmemLimit = 227 * 1024;
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes,
+                                          uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+template <typename ActT, typename IdxT>
+__global__ void __launch_bounds__(kTokThreads)
+replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __restrict__ idx,
+                            const ActT* __restrict__ o, const int32_t* __restrict__ row_of_slot,
+                            const ActT* __restrict__ dy, const ActT* __restrict__ residual,
+                            ActT* __restrict__ y, float* __restrict__ gates_out,
+                            float* __restrict__ dlogits, int E, int K, int d, int W,
+                            int32_t* dev_status) {
+    using V = Vec16<ActT>;
+    constexpr int N = V::N;
+    extern __shared__ __align__(128) uint8_t smem_tok[];
+    const uint32_t bar = tc::smem_u32(smem_tok);                       // 8 bytes
+    volatile int* flags = reinterpret_cast<volatile int*>(smem_tok + 8);   // [0] abort [1] ready
+    unsigned* have_s = reinterpret_cast<unsigned*>(smem_tok + 16);
+    float* g_s = reinterpret_cast<float*>(smem_tok + 32);               // [8]
+    const V* orow = reinterpret_cast<const V*>(smem_tok + kTokHeader + 128);
+    float* part2 = reinterpret_cast<float*>(smem_tok + kTokHeader);     // [kTokWarps][8] = 128 bytes
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t = blockIdx.x;
+    const int row_vecs = d / N;
+    const uint32_t row_bytes = (uint32_t)d * sizeof(ActT);
+
+    int my_e = -1;
+    float g = 0.f;
+    if (warp == 0) {
+        // ---- ask for the rows ---------------------------------------------------------------------
+        int32_t r = -1;
+        if (lane < K) r = row_of_slot[(size_t)t * K + lane];
+        if (lane == 0) {
+            tc::mbar_init(bar, 1);
+            flags[0] = 0;
+            tc::fence_barrier_init();
+        }
+        const unsigned have = __ballot_sync(0xffffffffu, r >= 0);
+        __syncwarp();
+        const uint32_t s_rows = tc::smem_u32(orow);
+        if (lane == 0) {
+            *have_s = have;
+            tc::mbar_expect_tx(bar, row_bytes * (uint32_t)(__popc(have) + 1 + (residual ? 1 : 0)));
+        }
+        __syncwarp();
+        if (lane < K) {
+            if (r >= 0)
+                bulk_load(s_rows + (uint32_t)lane * row_bytes, o + (size_t)r * d, row_bytes, bar);
+        } else if (lane == K) {
+            bulk_load(s_rows + (uint32_t)K * row_bytes, dy + (size_t)t * d, row_bytes, bar);
+        } else if (lane == K + 1) {
+            if (residual)
+                bulk_load(s_rows + (uint32_t)(K + 1) * row_bytes, residual + (size_t)t * d,
+                          row_bytes, bar);
+        }
+        // ---- replay gate while the copies fly: the first W lanes, one slot each -----------------
+        const IdxT* rec = idx + (size_t)t * K;
+        const float* lrow = logits + (size_t)t * E;
+        int bad = 0;
+        float s = -INFINITY;
+        if (lane < K) {
+            my_e = idx_to_int(rec[lane]);
+            if (my_e < 0 || my_e >= E) bad |= 1;
+            for (int j2 = 0; j2 < lane; ++j2)
+                if (idx_to_int(rec[j2]) == my_e) bad |= 2;
+            s = lrow[min(max(my_e, 0), E - 1)];
+        }
+        for (int ofs = W / 2; ofs > 0; ofs >>= 1) bad |= __shfl_xor_sync(0xffffffffu, bad, ofs, W);
+        if (bad && lane == 0)
+            report(dev_status, (bad & 1) ? R3_DEV_BAD_INDEX : R3_DEV_DUP_INDEX);
+        float m = s;
+        for (int ofs = W / 2; ofs > 0; ofs >>= 1)
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, ofs, W));
+        const float ex = lane < K ? expf(s - m) : 0.f;
+        float sum = ex;
+        for (int ofs = W / 2; ofs > 0; ofs >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, ofs, W);
+        const float inv = bad ? 0.f : 1.f / sum;
+        if (lane < K) {
+            g = ex * inv;
+            if (gates_out) gates_out[(size_t)t * K + lane] = g;
+        }
+        if (lane < kFusedMaxK) g_s[lane] = g;
+        // ---- one thread waits for the copies; the others sleep at the barrier below -----------
+        if (lane == 0) flags[1] = tc::mbar_wait(bar, 0u, flags, dev_status) ? 1 : 0;
+    }
+    __syncthreads();
+    const bool ready = flags[1] != 0;
+
+    // ---- combine and <dy, o_j> out of shared memory: the warps split the columns ------------------
+    float dacc[kFusedMaxK];
+#pragma unroll
+    for (int u = 0; u < kFusedMaxK; ++u) dacc[u] = 0.f;
+    if (ready) {
+        const unsigned have = *have_s;
+        float gj[kFusedMaxK];
+#pragma unroll
+        for (int u = 0; u < kFusedMaxK; ++u) gj[u] = g_s[u];
+        V* yv = reinterpret_cast<V*>(y) + (size_t)t * row_vecs;
+        for (int c = tid; c < row_vecs; c += kTokThreads) {
+            float gr[N];
+            orow[(size_t)K * row_vecs + c].unpack(gr);
+            float acc[N];
+#pragma unroll
+            for (int k2 = 0; k2 < N; ++k2) acc[k2] = 0.f;
+#pragma unroll
+            for (int u = 0; u < kFusedMaxK; ++u) {
+                if (have >> u & 1u) {
+                    float f[N];
+                    orow[(size_t)u * row_vecs + c].unpack(f);
+#pragma unroll
+                    for (int k2 = 0; k2 < N; ++k2) acc[k2] = fmaf(gj[u], f[k2], acc[k2]);
+#pragma unroll
+                    for (int k2 = 0; k2 < N; ++k2) dacc[u] = fmaf(gr[k2], f[k2], dacc[u]);
+                }
+            }
+            if (residual) {
+                float f[N];
+                orow[(size_t)(K + 1) * row_vecs + c].unpack(f);
+#pragma unroll
+                for (int k2 = 0; k2 < N; ++k2) acc[k2] += f[k2];
+            }
+            V out;
+            out.pack(acc);
+            yv[c] = out;
+        }
+    }
+    // ---- dg: across the warp, then the four warps in a fixed order -------------------------------
+#pragma unroll
+    for (int u = 0; u < kFusedMaxK; ++u) {
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) dacc[u] += __shfl_xor_sync(0xffffffffu, dacc[u], sft);
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int u = 0; u < kFusedMaxK; ++u) part2[warp * kFusedMaxK + u] = dacc[u];
+    }
+    __syncthreads();
+    if (warp == 0 && ready) {
+        float dg = 0.f;
+        if (lane < kFusedMaxK) {
+            for (int w2 = 0; w2 < kTokWarps; ++w2) dg += part2[w2 * kFusedMaxK + lane];
+        }
+        float cs = g * dg;                                        // lanes >= K hold g = 0
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) cs += __shfl_xor_sync(0xffffffffu, cs, sft);
+        const float val = g * (dg - cs);
+        float* out = dlogits + (size_t)t * E;
+        const int nchunk = (E + 3) >> 2;
+        for (int ch = lane; ch < ((nchunk + 31) & ~31); ch += 32) {
+            float q[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < K; ++j) {
+                const int ej = __shfl_sync(0xffffffffu, my_e, j);
+                const float vj = __shfl_sync(0xffffffffu, val, j);
+                if ((ej >> 2) == ch) q[ej & 3] = vj;
+            }
+            if (ch < nchunk) {
+                const int e0 = ch << 2;
+                if ((E & 3) == 0) {
+                    *reinterpret_cast<float4*>(out + e0) = make_float4(q[0], q[1], q[2], q[3]);
+                } else {
+                    for (int k2 = 0; k2 < 4 && e0 + k2 < E; ++k2) out[e0 + k2] = q[k2];
+                }
+            }
+        }
+    }
+    if (!ready) {
+        // the wait ran out: copies may still be in flight into this CTA's shared memory
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+}
+
 static int pick_team_fused(int row_vecs) {
     int tpt = 32;
     while (tpt < 256 && tpt < row_vecs) tpt <<= 1;
@@ -193,6 +389,21 @@ static void launch_finish(const r3_shape* s, const float* logits, const void* id
     const int T = s->T, K = s->K, d = s->d, E = s->E;
     int W = 1;
     while (W < K && W < 32) W <<= 1;
+    // staged kernel: one CTA per token, its K + 2 rows in shared memory (when they fit)
+    const size_t smem = kTokHeader + 128 + (size_t)(K + 1 + (residual ? 1 : 0)) * d * sizeof(ActT);
+    if (smem <= (size_t)kTokSmemLimit / 2) {
+        auto kern = replay_finish_staged_kernel<ActT, IdxT>;
+        static bool attr_set = false;          // one flag per instantiation
+        if (!attr_set) {
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
+            attr_set = true;
+        }
+        kern<<<T, kTokThreads, smem, cs>>>(
+            logits, static_cast<const IdxT*>(idx), static_cast<const ActT*>(o), row_of_slot,
+            static_cast<const ActT*>(dy), static_cast<const ActT*>(residual), static_cast<ActT*>(y),
+            gates_out, dlogits, E, K, d, W, dev_status);
+        return;
+    }
     const int tpt = pick_team_fused(d / Vec16<ActT>::N);
     const unsigned grid = (unsigned)((T + 256 / tpt - 1) / (256 / tpt));
 #define R3_FIN(TPT)                                                                              \

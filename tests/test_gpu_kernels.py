@@ -144,7 +144,8 @@ def test_combine_and_dgates(r3, T, K, d, act, tol):
     (1, 4, 1, 8, torch.bfloat16, TOL_BF16, False),
 ])
 def test_replay_finish_matches_the_four_kernels_and_the_oracle(r3, T, E, K, d, act, tol, residual):
-    """Gate + combine + both gradients in one pass: bit-identical to the four separate calls, and
+    """Gate + combine + both gradients in one pass: gates and y bit-identical to the separate
+    calls, dlogits equal to theirs up to the summation order of the gate gradient, and everything
     within tolerance of the oracle's Eq. replay_gate / replay_output / gradient."""
     rng = np.random.default_rng(T + K)
     idx_t = random_record(rng, T, E, K, torch.uint8)
@@ -166,7 +167,11 @@ def test_replay_finish_matches_the_four_kernels_and_the_oracle(r3, T, E, K, d, a
           else r3.combine(s, o.cuda(), ros_c, g4))
     dg4 = r3.combine_bwd_gates(s, dy.cuda(), o.cuda(), ros_c)
     ds4 = r3.replay_gate_bwd(s, g4, dg4, idx_t.cuda())
-    assert torch.equal(g, g4) and torch.equal(y, y4) and torch.equal(ds, ds4)
+    assert torch.equal(g, g4) and torch.equal(y, y4)
+    assert rel_err(f64(ds), f64(ds4)) < TOL_F32
+    y_b, g_b, ds_b = r3.replay_finish(s, logits.cuda(), idx_t.cuda(), o.cuda(), ros_c, dy.cuda(),
+                                      residual=None if res is None else res.cuda())
+    assert torch.equal(y, y_b) and torch.equal(g, g_b) and torch.equal(ds, ds_b)   # reproducible
     # the oracle
     g_ref = O.replay_gate(f64(logits), idx_np)
     eo = f64(o)[ros.astype(np.int64)]

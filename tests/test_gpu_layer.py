@@ -145,7 +145,10 @@ def run_big(r3, case, raw):
                                   dev_status=st)
     torch.cuda.synchronize()
     assert st.item() == 0
-    assert torch.equal(y, y2) and torch.equal(ds, ds2) and torch.equal(g, g2)
+    # the one-pass finish of the layer sums the gate gradient in another (fixed) order than
+    # r3_combine_bwd_gates: y and the gates agree bit for bit, dlogits to float32 rounding
+    assert torch.equal(y, y2) and torch.equal(g, g2)
+    assert (ds - ds2).abs().max().item() <= 1e-5 * ds.abs().max().item()
     return dict(y=y, ds=ds, g=g, logits=logits, counts=counts, offsets=offsets, ros=ros, sor=sor,
                 xp=xp)
 
