@@ -6,7 +6,8 @@
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
 
 A step is one pass of the whole path over one synthetic batch: training logits, replay gate,
-permute, grouped SwiGLU experts, combine, dgates, dlogits.  The default workload is the headline
+permute, grouped SwiGLU experts, combine, dgates, dlogits (the last four steps of the layer run as
+one kernel; the per-kernel table also times the separate entry points).  The default workload is the headline
 single bf16 layer (T=4096, d=2048, E=128, K=8, F=768).  One JSON line is printed by rank 0.
 """
 from __future__ import annotations
@@ -26,12 +27,12 @@ if ROOT not in sys.path:
 
 METRIC = "replayed-MoE-layer tokens/s (fwd+router bwd)"
 UNIT = "tokens/s"
-# kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, gate 1, permute 4,
-# tile list 1, expert GEMMs 2, combine 1, dgates 1, dlogits 1
-LAUNCHES_PER_STEP = 13
+# kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, permute 4,
+# GEMM work lists 1, expert GEMMs 2, finish (gate + combine + dgates + dlogits) 1
+LAUNCHES_PER_STEP = 10
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
-# from the ncu capture summarised in profiles/; None until captured.
-GEMM_UP_DRAM_TRAFFIC_BYTES = 993.5e6   # 947.5 MB read + 46.0 MB written
+# from the ncu capture summarised in profiles/grouped_gemm_pair_c2_layer_bf16.md.
+GEMM_UP_DRAM_TRAFFIC_BYTES = 991.4e6   # 943.6 MB read + 47.8 MB written
 
 
 def load_peaks():
@@ -310,13 +311,13 @@ def run_ours(args, w):
     # dominant kernel: the up-projection grouped GEMM (4 R d F of the 6 R d F expert FLOPs).
     # Its events bracket the call, which also holds the one-CTA tile-list kernel (a few us).
     achieved = flops["expert_up_swiglu"] / (seg_ms["expert_up_swiglu"] * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "grouped_gemm_tc_kernel<0> (gate/up + SwiGLU)",
+    roofline = {"bound": "tensor", "kernel": "grouped_gemm_pair_kernel<0> (gate/up + SwiGLU)",
                 "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": round(achieved / peaks["bf16_tflops"], 4),
                 "peak_kind": f"bf16 matmul burst, {peaks['source']}",
                 "frac_of_sustained": round(achieved / peaks["bf16_tflops_sustained"], 4),
                 "frac_of_nominal_2250": round(achieved / 2250.0, 4),
-                "traffic": GEMM_UP_DRAM_TRAFFIC_BYTES}
+                "traffic": GEMM_UP_DRAM_TRAFFIC_BYTES if wk.name == "c2_layer_bf16" else None}
 
     # ---- end to end through the host-buffer entry point -----------------------------------------
     xh, dyh, idxh = (t.cpu().pin_memory() for t in (x, dy, idx))

@@ -9,6 +9,7 @@
 // A pair whose index is out of range, or repeats an earlier slot of the same token, is dropped
 // (row_of_slot = -1) and reported through dev_status.
 #include "r3_common.cuh"
+#include "r3_tc.cuh"
 
 namespace r3 {
 
@@ -126,17 +127,29 @@ permute_rank_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ ch
     }
     __syncthreads();
     if (t < T) {
-        for (int j = 0; j < K; ++j) {
-            int e;
-            int32_t row = -1;
-            if (pair_ok(rec, j, E, e, nullptr)) {
-                const uint32_t* m = bits + e * kWords;
-                int rank = __popc(m[lt >> 5] & ((1u << (lt & 31)) - 1u));
-                for (int w = 0; w < (lt >> 5); ++w) rank += __popc(m[w]);
-                row = offsets[e] + chunk_base[(size_t)e * NB + blockIdx.x] + rank;
-                slot_of_row[row] = t * K + j;
+        // slots in batches of 8: the (independent) table reads of a batch are issued together
+        for (int j0 = 0; j0 < K; j0 += 8) {
+            int32_t row[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                int e;
+                row[u] = -1;
+                if (j < K && pair_ok(rec, j, E, e, nullptr)) {
+                    const uint32_t* m = bits + e * kWords;
+                    int rank = __popc(m[lt >> 5] & ((1u << (lt & 31)) - 1u));
+                    for (int w = 0; w < (lt >> 5); ++w) rank += __popc(m[w]);
+                    row[u] = offsets[e] + chunk_base[(size_t)e * NB + blockIdx.x] + rank;
+                }
             }
-            row_of_slot[(size_t)t * K + j] = row;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                if (j < K) {
+                    if (row[u] >= 0) slot_of_row[row[u]] = t * K + j;
+                    row_of_slot[(size_t)t * K + j] = row[u];
+                }
+            }
         }
     }
 }
@@ -168,6 +181,61 @@ permute_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ row
                 if (c < row_vecs) dst[c] = v[u];
             }
         }
+    }
+}
+
+
+// The same copy staged through shared memory with bulk asynchronous copies: a CTA of one warp
+// takes kRowTokens tokens; lane i brings token i's row in (one copy, completion counted on an
+// mbarrier) and, once it has landed, sends it to the token's K destination rows (one bulk store
+// each).  Nothing passes through registers, each copy is a whole row, and seven CTAs per SM keep
+// about 200 KB in flight.
+constexpr int kRowTokens = 8;
+
+__global__ void __launch_bounds__(32)
+permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_slot,
+                           uint8_t* __restrict__ xp, int T, int K, uint32_t row_bytes) {
+    extern __shared__ __align__(128) uint8_t smem_p[];
+    const uint32_t bar = tc::smem_u32(smem_p);
+    volatile int* flags = reinterpret_cast<volatile int*>(smem_p + 8);
+    const uint32_t rows0 = tc::smem_u32(smem_p + 128);
+    const int lane = threadIdx.x;
+    const int t0 = blockIdx.x * kRowTokens;
+    const int nt = min(kRowTokens, T - t0);
+    if (lane == 0) {
+        tc::mbar_init(bar, 1);
+        flags[0] = 0;
+        tc::fence_barrier_init();
+        tc::mbar_expect_tx(bar, row_bytes * (uint32_t)nt);
+    }
+    __syncwarp();
+    if (lane < nt)
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+            ::"r"(rows0 + (uint32_t)lane * row_bytes), "l"(x + (size_t)(t0 + lane) * row_bytes),
+              "r"(row_bytes), "r"(bar) : "memory");
+    int32_t r[8];
+    // destination rows of this lane's token (fetched while the copy flies); K > 8 goes in rounds
+    const bool ok = __all_sync(0xffffffffu, tc::mbar_wait(bar, 0u, flags, nullptr));
+    if (ok && lane < nt) {
+        const int32_t* rows = row_of_slot + (size_t)(t0 + lane) * K;
+        for (int j0 = 0; j0 < K; j0 += 8) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) r[u] = j0 + u < K ? rows[j0 + u] : -1;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (r[u] >= 0)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                                 ::"l"(xp + (size_t)r[u] * row_bytes),
+                                   "r"(rows0 + (uint32_t)lane * row_bytes), "r"(row_bytes)
+                                 : "memory");
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        // shared memory must outlive the stores that read it
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    }
+    if (!ok) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
     }
 }
 
@@ -213,7 +281,21 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
             static_cast<const IdxT*>(idx), chunk_counts, offsets, row_of_slot, slot_of_row,
             T, E, K, NB));
     if (x) {
-        const int row_vecs = (int)((size_t)shape->d * r3::act_bytes(shape) / 16);
+        const size_t row_bytes = (size_t)shape->d * r3::act_bytes(shape);
+        if (row_bytes * r3::kRowTokens <= 96 * 1024) {
+            const size_t smem = 128 + row_bytes * r3::kRowTokens;
+            static bool attr_set = false;
+            if (!attr_set) {
+                cudaFuncSetAttribute(r3::permute_rows_staged_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, 128 + 96 * 1024);
+                attr_set = true;
+            }
+            r3::permute_rows_staged_kernel<<<(T + r3::kRowTokens - 1) / r3::kRowTokens, 32, smem, cs>>>(
+                static_cast<const uint8_t*>(x), row_of_slot, static_cast<uint8_t*>(xp), T, K,
+                (uint32_t)row_bytes);
+            return r3::launch_status();
+        }
+        const int row_vecs = (int)(row_bytes / 16);
         const int wpb = 8;
         r3::permute_rows_kernel<16><<<(T + wpb - 1) / wpb, wpb * 32, 0, cs>>>(
             static_cast<const uint4*>(x), row_of_slot, static_cast<uint4*>(xp), T, K, row_vecs);
