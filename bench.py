@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 
 METRIC = "replayed-MoE-layer tokens/s (fwd+router bwd)"
 UNIT = "tokens/s"
-# kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, permute 4,
-# GEMM work lists 1, expert GEMMs 2, finish (gate + combine + dgates + dlogits) 1
+# kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, permute 4
+# (count, scan, rank), GEMM work lists 1, expert GEMMs 2, finish (gate + combine + dgates + dlogits) 1
 LAUNCHES_PER_STEP = 10
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
 # from the ncu capture summarised in profiles/grouped_gemm_pair_c2_layer_bf16.md.
@@ -240,7 +240,7 @@ def run_ours(args, w):
 
     # ---- per-kernel segments (same kernels through the per-step entry points, events between) --
     seg_names = ["logits", "gate_fwd", "permute", "expert_up_swiglu", "expert_down", "combine",
-                 "dgates", "gate_bwd", "finish_fused"]
+                 "dgates", "gate_bwd", "finish_fused", "permute_maps", "experts_gather"]
     logits = torch.empty((T, E), dtype=torch.float32, device=dev)
     dg = torch.empty((T, K), dtype=torch.float32, device=dev)
     pout = (torch.empty(E, dtype=torch.int32, device=dev),
@@ -278,6 +278,11 @@ def run_ours(args, w):
         r3.replay_finish(s, logits, idx, o, pout[2], dy, y=y, gates=gates, dlogits=dlogits,
                          dev_status=st)
         e[9].record()
+        # the layer's own dispatch: maps only, token rows gathered in place by the up projection
+        r3.permute(s, idx, None, out=pout[:4] + (None,), ws=pws, dev_status=st)
+        e[10].record()
+        r3.grouped_swiglu_gather(s, x, pout[3], pout[1], wg, wu, wd, o, ws=gws, dev_status=st)
+        e[11].record()
 
     for _ in range(3):
         seg_step(evs[0])
@@ -295,8 +300,10 @@ def run_ours(args, w):
         "dgates": T * (d * es + K * d * es + K * 4 + K * 4),
         "gate_bwd": T * (K * 9 + E * 4),
         "finish_fused": T * (K * d * es + 2 * d * es + K * 9 + K * 4 + E * 4),
+        "permute_maps": T * (K + K * 8),
     }
     flops = {"expert_up_swiglu": 4.0 * R * d * F, "expert_down": 2.0 * R * d * F,
+             "experts_gather": 6.0 * R * d * F,
              "logits": 2.0 * T * d * E}
     kernels = {}
     for n in seg_names:

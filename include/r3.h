@@ -21,6 +21,11 @@
  *    "host".  The library never allocates, frees or synchronises (except r3_replay_layer_host,
  *    which synchronises the stream before it returns); each call enqueues its kernels on
  *    `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream) and returns.
+ *    r3_replay_layer and the entry points built on it (_host, _blocks, _stack) also use one
+ *    internal non-blocking helper stream per device, created at the first such call on that
+ *    device and kept until the process exits: the router logits run there beside the
+ *    permutation.  The helper is forked from and joined back into `stream` with events, so the
+ *    call as a whole is ordered on `stream` exactly as if everything had been enqueued there.
  *  - Matrices are row-major and dense.  Weights are stored output-major: W_r [E, d],
  *    W_gate/W_up [E, F, d], W_down [E, d, F].
  *  - Activations and expert weights have dtype `act_dtype` (R3_F32 or R3_BF16); W_r has dtype
@@ -163,6 +168,21 @@ size_t r3_grouped_swiglu_workspace_bytes(const r3_shape* shape);
 r3_status r3_grouped_swiglu(const r3_shape* shape, const void* xp, const int32_t* offsets,
                             const void* w_gate, const void* w_up, const void* w_down, void* o,
                             void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* r3_grouped_swiglu without the permuted copy of the activations: the token operand of the up
+ * projection is read in place from x [T,d], row slot_of_row[r] / K for grouped row r (Eq.
+ * (replay_output): expert i sees exactly the tokens whose recorded mask has I_i = 1), so
+ * r3_permute can be called with x = xp = NULL and the R x d buffer never exists.  Results are
+ * bit-identical to r3_grouped_swiglu on xp[r] = x[slot_of_row[r] / K].  The rows arrive through
+ * four-row TMA gather copies, which on B200 run well below the rate of the tiled copies of the
+ * permuted form (measured: the up projection takes about 2.8x as long), so this form is for
+ * callers short of memory, not of time; r3_replay_layer uses the permuted copy.  bf16 only
+ * (R3_ERR_UNSUPPORTED for float32).  slot_of_row [R] and offsets [E+1] as written by r3_permute;
+ * workspace and dev_status as for r3_grouped_swiglu. */
+r3_status r3_grouped_swiglu_gather(const r3_shape* shape, const void* x, const int32_t* slot_of_row,
+                                   const int32_t* offsets, const void* w_gate, const void* w_up,
+                                   const void* w_down, void* o, void* workspace, size_t ws_bytes,
+                                   int32_t* dev_status, void* stream);
 
 /* The two halves of r3_grouped_swiglu as separate calls (same kernels, same workspace), so that a
  * caller can place other work, or timing events, between them:

@@ -1,9 +1,39 @@
 // The whole replayed layer as one enqueue: logits -> replay gate -> permute -> experts ->
 // combine -> dgates -> dlogits (Section 4.1, Eqs. replay_gate / replay_output and the
 // router-logit gradient), plus a variant whose per-step tensors live in host memory.
+#include <mutex>
+
 #include "r3_common.cuh"
 
 namespace r3 {
+
+// The router logits depend only on x and W_r, the permutation only on the record: the layer runs
+// the former on a helper stream beside the latter.  One non-blocking helper stream and two events
+// per device, created at the first call on that device and kept until the process exits; the
+// helper is forked from and joined back into the caller's stream with the events, so the call as
+// a whole is still ordered on the caller's stream (and can be captured with it).
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    int state = 0;                 // 0 = not tried, 1 = ready, -1 = unavailable
+};
+static SideStream* side_stream() {
+    static SideStream per_device[64];
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    SideStream& ss = per_device[dev];
+    if (ss.state == 0) {
+        const bool ok =
+            cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) == cudaSuccess;
+        ss.state = ok ? 1 : -1;
+        if (!ok) cudaGetLastError();
+    }
+    return ss.state == 1 ? &ss : nullptr;
+}
 
 struct LayerWs {
     float* logits;
@@ -71,22 +101,32 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
     const LayerWs w = carve(shape, workspace);
     float* gates = gates_out ? gates_out : w.gates;
     r3_status st;
-    // s_train = x W_r (only the logits are needed on the training side)
+    // s_train = x W_r (only the logits are needed on the training side, and only by the last
+    // kernel): on the helper stream, beside the permutation
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    SideStream* side = side_stream();
+    if (side && (cudaEventRecord(side->fork, cs) != cudaSuccess ||
+                 cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess))
+        return R3_ERR_CUDA;
     if ((st = r3_capture_topk_ws(shape, 1, x, w_router, nullptr, w.logits, w.router_ws,
-                                 w.router_bytes, stream)) != R3_OK)
+                                 w.router_bytes, side ? side->stream : cs)) != R3_OK)
         return st;
+    if (side && cudaEventRecord(side->join, side->stream) != cudaSuccess) return R3_ERR_CUDA;
     // K <= 8: gate, combine and both gradients in one pass over the expert outputs; wider records
     // take the four separate kernels (same results).
     const bool fused = shape->K <= 8;
-    if (!fused &&
-        (st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
-        return st;
+    if (!fused) {
+        if (side && cudaStreamWaitEvent(cs, side->join, 0) != cudaSuccess) return R3_ERR_CUDA;
+        if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
+            return st;
+    }
     if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
                          w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
         return st;
     if ((st = r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, w.swiglu_ws,
                                 w.swiglu_bytes, dev_status, stream)) != R3_OK)
         return st;
+    if (fused && side && cudaStreamWaitEvent(cs, side->join, 0) != cudaSuccess) return R3_ERR_CUDA;
     if (fused)
         return r3_replay_finish(shape, w.logits, idx, w.o, w.row_of_slot, dy, residual, y,
                                 gates_out, dlogits, dev_status, stream);

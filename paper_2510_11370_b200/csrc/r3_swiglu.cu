@@ -176,7 +176,8 @@ extern "C" size_t r3_grouped_swiglu_workspace_bytes(const r3_shape* shape) {
 
 namespace r3 {
 // Shared body of the three expert entry points.
-static r3_status run_experts(const r3_shape* shape, const void* xp, const int32_t* offsets,
+static r3_status run_experts(const r3_shape* shape, const void* xp, const void* x,
+                             const int32_t* slot_of_row, const int32_t* offsets,
                              const void* w_gate, const void* w_up, const void* w_down, void* o,
                              void* workspace, size_t ws_bytes, int32_t* dev_status, int phases,
                              void* stream) {
@@ -185,9 +186,13 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const int32_
     if (shape->E > 1024) return R3_ERR_UNSUPPORTED;
     if (shape->T == 0) return R3_OK;
     const bool up = phases & kPhaseUp, down = phases & kPhaseDown;
-    if ((up && (!xp || !offsets || !w_gate || !w_up)) || (down && (!w_down || !o)))
+    const bool gather = up && !xp;             // token rows read in place from x
+    if (gather && shape->act_dtype != R3_BF16) return R3_ERR_UNSUPPORTED;
+    if ((up && (!offsets || !w_gate || !w_up || (gather ? (!x || !slot_of_row) : !xp))) ||
+        (down && (!w_down || !o)))
         return R3_ERR_INVALID_ARG;
-    if ((up && (!aligned(xp, 16) || !aligned(w_gate, 16) || !aligned(w_up, 16))) ||
+    if ((up && (!aligned(xp, 16) || !aligned(x, 16) || !aligned(w_gate, 16) ||
+                !aligned(w_up, 16))) ||
         (down && (!aligned(o, 16) || !aligned(w_down, 16))))
         return R3_ERR_INVALID_ARG;
     if (!workspace || ws_bytes < r3_grouped_swiglu_workspace_bytes(shape) ||
@@ -197,7 +202,7 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const int32_
     void* h = workspace;
     int32_t* tiles = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + h_bytes(shape));
     if (shape->act_dtype == R3_BF16)
-        return launch_grouped_swiglu_tc(shape, xp, offsets, w_gate, w_up, w_down, h, o, tiles,
+        return launch_grouped_swiglu_tc(shape, xp, x, slot_of_row, offsets, w_gate, w_up, w_down, h, o, tiles,
                                         dev_status, phases, cs);
     if (up) {
         st = launch_build_tiles(offsets, shape->E, SBM, tiles, cs);
@@ -212,21 +217,31 @@ extern "C" r3_status r3_grouped_swiglu(const r3_shape* shape, const void* xp,
                                        const void* w_up, const void* w_down, void* o,
                                        void* workspace, size_t ws_bytes, int32_t* dev_status,
                                        void* stream) {
-    return r3::run_experts(shape, xp, offsets, w_gate, w_up, w_down, o, workspace, ws_bytes,
-                           dev_status, r3::kPhaseUp | r3::kPhaseDown, stream);
+    return r3::run_experts(shape, xp, nullptr, nullptr, offsets, w_gate, w_up, w_down, o, workspace,
+                           ws_bytes, dev_status, r3::kPhaseUp | r3::kPhaseDown, stream);
+}
+
+extern "C" r3_status r3_grouped_swiglu_gather(const r3_shape* shape, const void* x,
+                                              const int32_t* slot_of_row, const int32_t* offsets,
+                                              const void* w_gate, const void* w_up,
+                                              const void* w_down, void* o, void* workspace,
+                                              size_t ws_bytes, int32_t* dev_status, void* stream) {
+    if (!x || !slot_of_row) return R3_ERR_INVALID_ARG;
+    return r3::run_experts(shape, nullptr, x, slot_of_row, offsets, w_gate, w_up, w_down, o,
+                           workspace, ws_bytes, dev_status, r3::kPhaseUp | r3::kPhaseDown, stream);
 }
 
 extern "C" r3_status r3_expert_up_swiglu(const r3_shape* shape, const void* xp,
                                          const int32_t* offsets, const void* w_gate,
                                          const void* w_up, void* workspace, size_t ws_bytes,
                                          int32_t* dev_status, void* stream) {
-    return r3::run_experts(shape, xp, offsets, w_gate, w_up, nullptr, nullptr, workspace,
-                           ws_bytes, dev_status, r3::kPhaseUp, stream);
+    return r3::run_experts(shape, xp, nullptr, nullptr, offsets, w_gate, w_up, nullptr, nullptr,
+                           workspace, ws_bytes, dev_status, r3::kPhaseUp, stream);
 }
 
 extern "C" r3_status r3_expert_down(const r3_shape* shape, const void* w_down, void* o,
                                     void* workspace, size_t ws_bytes, int32_t* dev_status,
                                     void* stream) {
-    return r3::run_experts(shape, nullptr, nullptr, nullptr, nullptr, w_down, o, workspace,
-                           ws_bytes, dev_status, r3::kPhaseDown, stream);
+    return r3::run_experts(shape, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, w_down, o,
+                           workspace, ws_bytes, dev_status, r3::kPhaseDown, stream);
 }

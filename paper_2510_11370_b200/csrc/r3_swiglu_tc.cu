@@ -60,6 +60,7 @@ constexpr int FEAT1 = 2 * BMF;     // o features per item in MODE 1
 struct alignas(64) PairMaps {
     CUtensorMap a0, a1;
     CUtensorMap b[BNT / 16];
+    CUtensorMap g;                 // gather form: the un-permuted activations, box 64 x 1
 };
 
 // ---- work list -------------------------------------------------------------------------------
@@ -127,9 +128,14 @@ build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
 }
 
 // ---- the GEMM kernel --------------------------------------------------------------------------
-template <int MODE>
+// GATHER (up projection only): the token operand is read from the un-permuted activations
+// x [T, d], row slot_of_row[r] / K for grouped row r, with TMA gather4 copies (each lane of the
+// producer warp owns four rows of the CTA's half of the token tile and issues one copy per k
+// block), so the permuted copy of x never has to exist.
+template <int MODE, bool GATHER>
 __global__ void __launch_bounds__(THREADS, 1)
 grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* __restrict__ list,
+                         const int32_t* __restrict__ slot_of_row, int K,
                          __nv_bfloat16* __restrict__ out, int Kdim, int Nout,
                          int32_t* dev_status) {
     extern __shared__ uint8_t smem_raw[];
@@ -169,7 +175,64 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0) {
+    if (warp == 0 && GATHER) {
+        // ------------------------------ TMA producer, gather form (the whole warp) -------------
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        const int4 kNone = make_int4(0, 0, 0, 0);
+        // token (row of x) of rows 4*lane .. 4*lane+3 of this CTA's half of item `it`
+        auto load_tokens = [&](const int4& it, int* tok) {
+            const int half = it.z >> 1;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int in_half = 4 * lane + i, in_item = (int)rank * half + in_half;
+                tok[i] = (in_half < half && in_item < it.w) ? slot_of_row[it.y + in_item] / K : 0;
+            }
+        };
+        // item descriptors run two items ahead of the copies, token numbers one item ahead
+        int4 it_cur = w_begin < w_end ? items[w_begin] : kNone;
+        int4 it_nxt = w_begin + w_step < w_end ? items[w_begin + w_step] : kNone;
+        int cur[4], nxt[4];
+        load_tokens(it_cur, nxt);
+        for (int w = w_begin; ok && w < w_end; w += w_step) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
+            const int4 it = it_cur;
+            it_cur = it_nxt;
+            it_nxt = w + 2 * w_step < w_end ? items[w + 2 * w_step] : kNone;
+            load_tokens(it_cur, nxt);             // lands while this item's copies are issued
+            const int e = it.x & 0xffff, f = it.x >> 16, n = it.z, half = n >> 1;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                int free_ok = 1;
+                if (lane == 0)
+                    free_ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status) ? 1 : 0;
+                if (!__shfl_sync(0xffffffffu, free_ok, 0)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
+                if (lane == 0) {
+                    if (rank == 0)                      // bytes of both CTAs: 2 x (A + n/2 rows)
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(2 * A_BYTES + n * BK * 2));
+                    const int f0 = f * FEAT0 + (int)rank * (BMF / 2);
+                    tma_load_3d_pair(sa, &maps.a0, kb * BK, f0, e, lead_full);
+                    tma_load_3d_pair(sa + A_BYTES / 2, &maps.a1, kb * BK, f0, e, lead_full);
+                }
+                if (4 * lane < half)
+                    tma_gather4_pair(sb + (uint32_t)lane * 512u, &maps.g, kb * BK, cur[0], cur[1],
+                                     cur[2], cur[3], lead_full);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (lane == 0) {
+            for (int s = 0; ok && s < STAGES; ++s) {
+                ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 0) {
         // ------------------------------ TMA producer (each CTA loads its own halves) -----------
         if (lane == 0) {
             int stage = 0;
@@ -399,9 +462,10 @@ static int resident_pairs(Kern kern) {
     return cached[dev];
 }
 
-template <int MODE>
-static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* list, void* out,
-                             int Kdim, int Nout, int32_t* dev_status, cudaStream_t cs) {
+template <int MODE, bool GATHER>
+static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* list,
+                             const int32_t* slot_of_row, int K, void* out, int Kdim, int Nout,
+                             int32_t* dev_status, cudaStream_t cs) {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -414,7 +478,7 @@ static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* lis
     cfg.stream = cs;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<MODE>, maps, list,
+    return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<MODE, GATHER>, maps, list, slot_of_row, K,
                               static_cast<__nv_bfloat16*>(out), Kdim, Nout,
                               dev_status) == cudaSuccess ? R3_OK : R3_ERR_CUDA;
 }
@@ -435,7 +499,8 @@ size_t tc_work_bytes(const r3_shape* s) {
     return list_bytes(R, s->E, feat_tiles_up(s)) + list_bytes(R, s->E, feat_tiles_down(s));
 }
 
-r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int32_t* offsets,
+r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void* x,
+                                   const int32_t* slot_of_row, const int32_t* offsets,
                                    const void* w_gate, const void* w_up, const void* w_down,
                                    void* h, void* o, void* work, int32_t* dev_status, int phases,
                                    cudaStream_t cs) {
@@ -444,14 +509,16 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int3
     if (R == 0) return R3_OK;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<0>,
+        if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<0, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-            cudaFuncSetAttribute(grouped_gemm_pair_kernel<1>,
+            cudaFuncSetAttribute(grouped_gemm_pair_kernel<0, true>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return R3_ERR_CUDA;
         attr_set = true;
     }
-    const int pairs = resident_pairs(grouped_gemm_pair_kernel<0>);
+    const int pairs = resident_pairs(grouped_gemm_pair_kernel<0, false>);
     if (pairs <= 0) return R3_ERR_CUDA;
     const int nf0 = feat_tiles_up(s), nf1 = feat_tiles_down(s);
     int32_t* list0 = static_cast<int32_t*>(work);
@@ -462,10 +529,19 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int3
         build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1);
         PairMaps m;
         if (!make_map_3d(&m.a0, w_gate, s->E, s->F, s->d, BMF / 2) ||
-            !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2) ||
-            !token_maps(&cache_xp, xp, (uint64_t)R, (uint64_t)s->d, &m))
+            !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2))
             return R3_ERR_CUDA;
-        const r3_status st = launch_pair<0>(m, pairs, list0, h, s->d, s->F, dev_status, cs);
+        r3_status st;
+        if (xp) {
+            if (!token_maps(&cache_xp, xp, (uint64_t)R, (uint64_t)s->d, &m)) return R3_ERR_CUDA;
+            m.g = m.b[0];
+            st = launch_pair<0, false>(m, pairs, list0, nullptr, 0, h, s->d, s->F, dev_status, cs);
+        } else {
+            if (!make_map_2d(&m.g, x, (uint64_t)s->T, (uint64_t)s->d, 1)) return R3_ERR_CUDA;
+            for (int i = 0; i < BNT / 16; ++i) m.b[i] = m.g;
+            st = launch_pair<0, true>(m, pairs, list0, slot_of_row, s->K, h, s->d, s->F,
+                                      dev_status, cs);
+        }
         if (st != R3_OK) return st;
     }
     if (phases & kPhaseDown) {
@@ -474,7 +550,9 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const int3
             !token_maps(&cache_h, h, (uint64_t)R, (uint64_t)s->F, &m))
             return R3_ERR_CUDA;
         m.a1 = m.a0;
-        const r3_status st = launch_pair<1>(m, pairs, list1, o, s->F, s->d, dev_status, cs);
+        m.g = m.b[0];
+        const r3_status st = launch_pair<1, false>(m, pairs, list1, nullptr, 0, o, s->F, s->d,
+                                                   dev_status, cs);
         if (st != R3_OK) return st;
     }
     return launch_status();

@@ -28,7 +28,8 @@ EXPORTS = [
     "r3_status_string", "r3_capture_topk", "r3_capture_topk_batched",
     "r3_capture_topk_workspace_bytes", "r3_capture_topk_ws", "r3_replay_gate_fwd",
     "r3_replay_gate_bwd", "r3_permute_workspace_bytes", "r3_permute", "r3_permute_static",
-    "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_expert_up_swiglu",
+    "r3_grouped_swiglu_workspace_bytes", "r3_grouped_swiglu", "r3_grouped_swiglu_gather",
+    "r3_expert_up_swiglu",
     "r3_expert_down", "r3_combine",
     "r3_combine_residual", "r3_combine_bwd_gates", "r3_replay_finish",
     "r3_replay_layer_workspace_bytes",
@@ -62,6 +63,7 @@ lib.r3_replay_gate_bwd.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_permute.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_permute_static.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, _P]
 lib.r3_grouped_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
+lib.r3_grouped_swiglu_gather.argtypes = [_SP, _P, _P, _P, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_expert_up_swiglu.argtypes = [_SP, _P, _P, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_expert_down.argtypes = [_SP, _P, _P, _P, ctypes.c_size_t, _P, _P]
 lib.r3_combine.argtypes = [_SP, _P, _P, _P, _P, _P]
@@ -259,6 +261,20 @@ def grouped_swiglu(s: Shape, xp, offsets, w_gate, w_up, w_down, o=None, *, ws=No
     _check(lib.r3_grouped_swiglu(ctypes.byref(s), _ptr(xp), _ptr(offsets), _ptr(w_gate),
                                  _ptr(w_up), _ptr(w_down), _ptr(o), _ptr(ws), ws.numel(),
                                  _ptr(dev_status), _stream(stream)))
+    return o
+
+
+def grouped_swiglu_gather(s: Shape, x, slot_of_row, offsets, w_gate, w_up, w_down, o=None, *,
+                          ws=None, dev_status=None, stream=None):
+    """grouped_swiglu reading the token rows in place from x [T,d] through slot_of_row (bf16)."""
+    dev = _dev(x)
+    if o is None:
+        o = torch.empty((s.T * s.K, s.d), dtype=_act_dtype(s), device=dev)
+    if ws is None:
+        ws = workspace(grouped_swiglu_workspace_bytes(s), dev)
+    _check(lib.r3_grouped_swiglu_gather(ctypes.byref(s), _ptr(x), _ptr(slot_of_row), _ptr(offsets),
+                                        _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(o), _ptr(ws),
+                                        ws.numel(), _ptr(dev_status), _stream(stream)))
     return o
 
 

@@ -341,6 +341,14 @@ def run_swiglu_case(r3, T, d, E, K, F, act, tol, seed=0):
     o2 = r3.grouped_swiglu(s, xp.cuda(), torch.from_numpy(offsets).cuda(), wg.cuda(), wu.cuda(),
                            wd.cuda())
     assert torch.equal(o, o2)
+    if act == torch.bfloat16:
+        # the gather form reads the same rows in place from x: bit-identical
+        st2 = r3.new_status("cuda")
+        o3 = r3.grouped_swiglu_gather(s, x.cuda(), torch.from_numpy(sor.astype(np.int32)).cuda(),
+                                      torch.from_numpy(offsets).cuda(), wg.cuda(), wu.cuda(),
+                                      wd.cuda(), dev_status=st2)
+        assert st2.item() == 0
+        assert torch.equal(o, o3)
 
 
 @pytest.mark.parametrize("T,d,E,K,F", [(64, 128, 8, 2, 256), (300, 72, 5, 3, 40), (7, 8, 3, 1, 8)])
