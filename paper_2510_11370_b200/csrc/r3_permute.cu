@@ -8,7 +8,10 @@
 // chose the expert; the rank of a pair inside the chunk is the number of lower set bits.
 // A pair whose index is out of range, or repeats an earlier slot of the same token, is dropped
 // (row_of_slot = -1) and reported through dev_status.
+#include <cooperative_groups.h>
+
 #include "r3_common.cuh"
+#include "r3_internal.h"
 #include "r3_tc.cuh"
 
 namespace r3 {
@@ -154,6 +157,122 @@ permute_rank_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ ch
     }
 }
 
+// The three steps above as ONE cooperative launch (all chunk CTAs resident, two grid-wide
+// barriers): at a few thousand tokens the three separate launches cost more in launch and drain
+// time than in work.  Same arithmetic, same results; used whenever all the chunk CTAs fit on the
+// device at once.
+//   step 1  per-chunk counts -> chunk_counts[e][chunk]
+//   step 2  one warp per expert: exclusive scan along the chunks, total -> counts[e]
+//   step 3  every CTA scans counts[] into the expert offsets (shared memory), CTA 0 writes them
+//           out; then ranks and maps exactly as permute_rank_kernel
+template <typename IdxT>
+__global__ void __launch_bounds__(kChunk)
+permute_maps_coop_kernel(const IdxT* __restrict__ idx, int32_t* chunk_counts, int32_t* counts,
+                         int32_t* offsets, int32_t* __restrict__ row_of_slot,
+                         int32_t* __restrict__ slot_of_row, int T, int E, int K, int NB,
+                         int32_t* dev_status) {
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
+    extern __shared__ int32_t sm[];
+    int32_t* hist = sm;                                   // [E], later the expert offsets
+    uint32_t* bits = reinterpret_cast<uint32_t*>(sm + E); // [E][kWords]
+    __shared__ int32_t warp_sum[kChunk / 32];
+    const int lt = threadIdx.x, lane = lt & 31, warp = lt >> 5;
+    const int t = blockIdx.x * kChunk + lt;
+    const IdxT* rec = idx + (size_t)(t < T ? t : 0) * K;
+
+    // ---- step 1 -----------------------------------------------------------------------------
+    for (int e = lt; e < E; e += kChunk) hist[e] = 0;
+    for (int i = lt; i < E * kWords; i += kChunk) bits[i] = 0u;
+    __syncthreads();
+    if (t < T) {
+        for (int j = 0; j < K; ++j) {
+            int e;
+            if (pair_ok(rec, j, E, e, dev_status)) {
+                atomicAdd(&hist[e], 1);
+                atomicOr(&bits[e * kWords + (lt >> 5)], 1u << (lt & 31));
+            }
+        }
+    }
+    __syncthreads();
+    for (int e = lt; e < E; e += kChunk) chunk_counts[(size_t)e * NB + blockIdx.x] = hist[e];
+    grid.sync();
+
+    // ---- step 2 -----------------------------------------------------------------------------
+    const int warps_total = gridDim.x * (kChunk / 32);
+    for (int e = blockIdx.x * (kChunk / 32) + warp; e < E; e += warps_total) {
+        int32_t* row = chunk_counts + (size_t)e * NB;
+        int32_t carry = 0;
+        for (int b0 = 0; b0 < NB; b0 += 32) {
+            const int b = b0 + lane;
+            const int32_t v = b < NB ? row[b] : 0;
+            int32_t inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += n;
+            }
+            if (b < NB) row[b] = carry + inc - v;
+            carry += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        if (lane == 0) counts[e] = carry;
+    }
+    grid.sync();
+
+    // ---- step 3: offsets (each thread owns a run of experts), then ranks -----------------------
+    const int per = (E + kChunk - 1) / kChunk;
+    int32_t mine = 0;
+    for (int i = 0; i < per; ++i) {
+        const int e = lt * per + i;
+        if (e < E) mine += counts[e];
+    }
+    int32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_sum[warp] = inc;
+    __syncthreads();
+    int32_t run = inc - mine;
+    for (int w = 0; w < warp; ++w) run += warp_sum[w];
+    for (int i = 0; i < per; ++i) {
+        const int e = lt * per + i;
+        if (e < E) {
+            hist[e] = run;                                // exclusive offset of expert e
+            if (blockIdx.x == 0) offsets[e] = run;
+            run += counts[e];
+            if (blockIdx.x == 0 && e == E - 1) offsets[E] = run;
+        }
+    }
+    __syncthreads();
+    if (t < T) {
+        for (int j0 = 0; j0 < K; j0 += 8) {
+            int32_t row[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                int e;
+                row[u] = -1;
+                if (j < K && pair_ok(rec, j, E, e, nullptr)) {
+                    const uint32_t* m = bits + e * kWords;
+                    int rank = __popc(m[lt >> 5] & ((1u << (lt & 31)) - 1u));
+                    for (int w = 0; w < (lt >> 5); ++w) rank += __popc(m[w]);
+                    row[u] = hist[e] + chunk_counts[(size_t)e * NB + blockIdx.x] + rank;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                if (j < K) {
+                    if (row[u] >= 0) slot_of_row[row[u]] = t * K + j;
+                    row_of_slot[(size_t)t * K + j] = row[u];
+                }
+            }
+        }
+    }
+}
+
 // One warp per token: read x[t] once (16-byte pieces), write it to the token's K rows.
 template <int VEC_BYTES>
 __global__ void __launch_bounds__(256)
@@ -272,6 +391,30 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
     const int T = shape->T, E = shape->E, K = shape->K;
     const int NB = (T + r3::kChunk - 1) / r3::kChunk;
     int32_t* chunk_counts = static_cast<int32_t*>(workspace);
+    // one cooperative launch when all the chunk CTAs can be resident together
+    bool coop_done = false;
+    {
+        const size_t smem = (size_t)E * (1 + r3::kWords) * sizeof(int32_t);
+        int per_sm = 0;
+        cudaError_t qe = cudaErrorUnknown;
+        R3_DISPATCH_IDX(shape, IdxT, qe = cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+            &per_sm, r3::permute_maps_coop_kernel<IdxT>, r3::kChunk, smem));
+        if (qe == cudaSuccess && smem <= 48 * 1024 && (long long)per_sm * r3::sm_count() >= NB) {
+            int Tn = T, En = E, Kn = K, NBn = NB;
+            void* args[] = {(void*)&idx, (void*)&chunk_counts, (void*)&counts, (void*)&offsets,
+                            (void*)&row_of_slot, (void*)&slot_of_row, (void*)&Tn, (void*)&En,
+                            (void*)&Kn, (void*)&NBn, (void*)&dev_status};
+            cudaError_t le = cudaErrorUnknown;
+            R3_DISPATCH_IDX(shape, IdxT, le = cudaLaunchCooperativeKernel(
+                (const void*)r3::permute_maps_coop_kernel<IdxT>, dim3(NB), dim3(r3::kChunk), args,
+                smem, cs));
+            if (le != cudaSuccess) return R3_ERR_CUDA;
+            coop_done = true;
+        } else {
+            cudaGetLastError();
+        }
+    }
+    if (!coop_done) {
     R3_DISPATCH_IDX(shape, IdxT,
         r3::permute_count_kernel<IdxT><<<NB, r3::kChunk, E * sizeof(int32_t), cs>>>(
             static_cast<const IdxT*>(idx), chunk_counts, T, E, K, NB, dev_status));
@@ -280,6 +423,7 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
         r3::permute_rank_kernel<IdxT><<<NB, r3::kChunk, E * r3::kWords * sizeof(uint32_t), cs>>>(
             static_cast<const IdxT*>(idx), chunk_counts, offsets, row_of_slot, slot_of_row,
             T, E, K, NB));
+    }
     if (x) {
         const size_t row_bytes = (size_t)shape->d * r3::act_bytes(shape);
         if (row_bytes * r3::kRowTokens <= 96 * 1024) {
