@@ -14,7 +14,8 @@ namespace r3 {
 // a whole is still ordered on the caller's stream (and can be captured with it).
 struct SideStream {
     cudaStream_t stream = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr;
+    cudaStream_t copy = nullptr;   // host-buffer entry point: dy travels here beside the compute
+    cudaEvent_t fork = nullptr, join = nullptr, copy_fork = nullptr, copied = nullptr;
     int state = 0;                 // 0 = not tried, 1 = ready, -1 = unavailable
 };
 static SideStream* side_stream() {
@@ -27,6 +28,9 @@ static SideStream* side_stream() {
     if (ss.state == 0) {
         const bool ok =
             cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&ss.copy, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.copy_fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.copied, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) == cudaSuccess;
         ss.state = ok ? 1 : -1;
@@ -97,7 +101,7 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
                            const void* idx, const void* w_gate, const void* w_up,
                            const void* w_down, const void* dy, const void* residual, void* y,
                            float* dlogits, float* gates_out, void* workspace,
-                           int32_t* dev_status, void* stream) {
+                           int32_t* dev_status, void* stream, cudaEvent_t dy_ready = nullptr) {
     const LayerWs w = carve(shape, workspace);
     float* gates = gates_out ? gates_out : w.gates;
     r3_status st;
@@ -127,6 +131,8 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
                                 w.swiglu_bytes, dev_status, stream)) != R3_OK)
         return st;
     if (fused && side && cudaStreamWaitEvent(cs, side->join, 0) != cudaSuccess) return R3_ERR_CUDA;
+    // dy is first needed here (host-buffer entry point: it may still be on its way)
+    if (dy_ready && cudaStreamWaitEvent(cs, dy_ready, 0) != cudaSuccess) return R3_ERR_CUDA;
     if (fused)
         return r3_replay_finish(shape, w.logits, idx, w.o, w.row_of_slot, dy, residual, y,
                                 gates_out, dlogits, dev_status, stream);
@@ -284,13 +290,28 @@ extern "C" r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_h
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const r3::HostWs h = r3::carve_host(shape, workspace);
     const size_t T = shape->T, row = (size_t)shape->d * r3::act_bytes(shape);
+    if (!x_host || !w_router || !w_gate || !w_up || !w_down) return R3_ERR_INVALID_ARG;
     if (cudaMemcpyAsync(h.x, x_host, T * row, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
         cudaMemcpyAsync(h.idx, idx_host, T * shape->K * r3::idx_bytes(shape),
-                        cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-        cudaMemcpyAsync(h.dy, dy_host, T * row, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+                        cudaMemcpyHostToDevice, cs) != cudaSuccess)
         return R3_ERR_CUDA;
-    st = r3_replay_layer(shape, h.x, w_router, h.idx, w_gate, w_up, w_down, h.dy, h.y, h.dlogits,
-                         nullptr, h.inner, h.inner_bytes, dev_status, stream);
+    // x and the record are needed at once; dy only by the last kernel: it follows x over the
+    // link on a copy stream of its own while the layer computes
+    r3::SideStream* side = r3::side_stream();
+    cudaEvent_t dy_ready = nullptr;
+    if (side) {
+        if (cudaEventRecord(side->copy_fork, cs) != cudaSuccess ||
+            cudaStreamWaitEvent(side->copy, side->copy_fork, 0) != cudaSuccess ||
+            cudaMemcpyAsync(h.dy, dy_host, T * row, cudaMemcpyHostToDevice, side->copy) !=
+                cudaSuccess ||
+            cudaEventRecord(side->copied, side->copy) != cudaSuccess)
+            return R3_ERR_CUDA;
+        dy_ready = side->copied;
+    } else if (cudaMemcpyAsync(h.dy, dy_host, T * row, cudaMemcpyHostToDevice, cs) != cudaSuccess) {
+        return R3_ERR_CUDA;
+    }
+    st = r3::run_layer(shape, h.x, w_router, h.idx, w_gate, w_up, w_down, h.dy, nullptr, h.y,
+                       h.dlogits, nullptr, h.inner, dev_status, stream, dy_ready);
     if (st != R3_OK) return st;
     if (cudaMemcpyAsync(y_host, h.y, T * row, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
         cudaMemcpyAsync(dlogits_host, h.dlogits, T * shape->E * 4, cudaMemcpyDeviceToHost, cs) !=
