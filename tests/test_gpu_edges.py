@@ -1,0 +1,134 @@
+"""Degenerate and boundary cases of the replayed layer on the GPU, each against the oracle:
+no tokens, one token, K = 1 (gate 1, zero router gradient), K = E (every expert), all tokens on
+one expert (127 empty experts, one expert spanning many token tiles), records wider than a byte
+(int16, E > 256), token counts that straddle the 256-token chunks of the dispatch, and a
+token count beyond what the one-launch dispatch can keep resident (three-launch path)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import r3_oracle as O
+from paper_2510_11370_b200 import synth
+from tests.helpers import Case, f32, f64, random_record, rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 1e-5
+
+
+@pytest.fixture(scope="module")
+def r3():
+    from paper_2510_11370_b200 import r3 as mod
+    return mod
+
+
+def layer_against_oracle(r3, case, tol, idx=None):
+    if idx is not None:
+        case.idx = idx
+    s = r3.shape_of(case.w)
+    c = case.cuda()
+    st = r3.new_status("cuda")
+    y, ds, g = r3.replay_layer(s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"], c["w_down"],
+                               c["dy"], dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    ref = case.oracle_layer()
+    assert rel_err(f64(g), ref["g"]) < 1e-5
+    assert rel_err(f64(y), ref["y"]) < tol
+    denom = np.abs(ref["ds"]).max()
+    if denom > 0:
+        assert rel_err(f64(ds), ref["ds"]) < tol
+    else:
+        assert float(ds.abs().max()) == 0.0
+    return y, ds, g
+
+
+def test_no_tokens_is_ok_and_launches_nothing(r3):
+    s = r3.make_shape(0, 64, 8, 2, 64)
+    e = lambda *sh, dt=torch.bfloat16: torch.empty(sh, dtype=dt, device="cuda")
+    ws = r3.workspace(4096, "cuda")
+    y, ds, g = r3.replay_layer(s, e(0, 64), e(8, 64, dt=torch.float32), e(0, 2, dt=torch.uint8),
+                               e(8, 64, 64), e(8, 64, 64), e(8, 64, 64), e(0, 64), ws=ws)
+    assert y.shape == (0, 64) and ds.shape == (0, 8)
+    counts, offsets, ros, sor, _ = r3.permute(s, e(0, 2, dt=torch.uint8))
+    torch.cuda.synchronize()
+    assert counts.sum().item() == 0 and offsets.abs().sum().item() == 0
+
+
+@pytest.mark.parametrize("act,tol", [("f32", TOL_F32), ("bf16", TOL_BF16)])
+def test_one_token(r3, act, tol):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="one", T=1, d=128, E=16, K=4, F=64,
+                     act=act)
+    layer_against_oracle(r3, Case(w), tol)
+
+
+def test_k1_gate_is_one_and_router_gradient_is_zero(r3):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="k1", T=300, d=256, E=16, K=1, F=128)
+    y, ds, g = layer_against_oracle(r3, Case(w), TOL_BF16)
+    assert torch.all(g == 1.0) and torch.all(ds == 0.0)
+
+
+def test_k_equals_e_uses_every_expert(r3):
+    w = synth.scaled(synth.WORKLOADS["c1_tiny_fp32"], name="kE", T=130, d=64, E=8, K=8, F=64,
+                     record="noise", sigma=0.5)
+    case = Case(w)
+    y, ds, g = layer_against_oracle(r3, case, TOL_F32)
+    # K = M: the replay gate is the full softmax of the training logits
+    full = torch.softmax(torch.from_numpy(case.s), dim=1).numpy()
+    picked = np.take_along_axis(full, case.idx_np(), axis=1)
+    assert rel_err(f64(g), picked) < 1e-5
+
+
+def test_every_token_on_the_same_experts(r3):
+    """K experts take all T tokens (T rows each, several 256-row token tiles), the others none."""
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="hot", T=700, d=256, E=32, K=2, F=128)
+    case = Case(w)
+    idx = torch.tensor([[5, 17]], dtype=torch.uint8).repeat(w.T, 1)
+    y, ds, g = layer_against_oracle(r3, case, TOL_BF16, idx=idx)
+    s = r3.shape_of(w)
+    counts, offsets, _, _, _ = r3.permute(s, idx.cuda())
+    c = counts.cpu().numpy()
+    assert c[5] == w.T and c[17] == w.T and c.sum() == 2 * w.T
+
+
+@pytest.mark.parametrize("act,tol", [("f32", TOL_F32), ("bf16", TOL_BF16)])
+def test_int16_record_with_more_than_256_experts(r3, act, tol):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="wide", T=200, d=64, E=300, K=3, F=64,
+                     act=act, sigma=0.2)
+    assert w.idx_dtype == torch.int16
+    layer_against_oracle(r3, Case(w), tol)
+
+
+@pytest.mark.parametrize("T", [255, 256, 257, 513])
+def test_dispatch_across_chunk_boundaries_is_bit_exact(r3, T):
+    E, K = 24, 5
+    idx = random_record(np.random.default_rng(T), T, E, K, torch.uint8)
+    s = r3.make_shape(T, 8, E, K, 8)
+    counts, offsets, ros, sor, _ = r3.permute(s, idx.cuda())
+    rc, ro, rr, rs = O.permutation(idx.to(torch.int64).numpy(), E)
+    assert np.array_equal(counts.cpu().numpy(), rc) and np.array_equal(offsets.cpu().numpy(), ro)
+    assert np.array_equal(ros.cpu().numpy(), rr) and np.array_equal(sor.cpu().numpy(), rs)
+
+
+def test_dispatch_of_more_chunks_than_fit_on_the_device_at_once(r3):
+    """T / 256 chunk CTAs beyond the resident limit take the three-launch dispatch; the maps are
+    checked against their defining properties (the oracle's stable sort at this size takes long)."""
+    T, E, K = 400_000, 8, 2
+    rng = np.random.default_rng(11)
+    first = rng.integers(0, E, size=T)
+    second = (first + rng.integers(1, E, size=T)) % E
+    idx_np = np.stack([first, second], axis=1)
+    idx = torch.from_numpy(idx_np.astype(np.uint8))
+    s = r3.make_shape(T, 8, E, K, 8)
+    counts, offsets, ros, sor, _ = r3.permute(s, idx.cuda())
+    counts, offsets, ros, sor = (t.cpu().numpy() for t in (counts, offsets, ros, sor))
+    assert np.array_equal(counts, np.bincount(idx_np.reshape(-1), minlength=E))
+    assert np.array_equal(offsets, np.concatenate([[0], np.cumsum(counts)]))
+    flat = ros.reshape(-1)
+    assert np.array_equal(np.sort(flat), np.arange(T * K))              # a permutation
+    assert np.array_equal(sor[flat], np.arange(T * K))                  # and its inverse
+    expert_of_row = idx_np.reshape(-1)[sor]
+    assert np.all(np.diff(expert_of_row) >= 0)                          # grouped by expert
+    same = np.diff(expert_of_row) == 0
+    assert np.all(np.diff(sor // K)[same] > 0)                          # stable within an expert
