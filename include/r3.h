@@ -278,6 +278,40 @@ r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host, const 
                                float* dlogits_host, void* workspace, size_t ws_bytes,
                                int32_t* dev_status, void* stream);
 
+/* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */
+
+/* Eq. (kl), the k3 estimate of KL(pi_train || pi_infer), and Eq. (etdf), the Extreme Token
+ * Distribution Function, over n response tokens:
+ *   *kl_out       = (1/n) sum_t [ r_t - 1 - log r_t ],   r_t = p_train[t] / p_infer[t]   (float64)
+ *   counts_out[i] = #{ t : max(r_t, 1/r_t) > taus[i] }   (so F(taus[i]) = counts_out[i] / n)
+ * p_train, p_infer [n] float32 probabilities of the sampled tokens (positive); taus [n_tau]
+ * float32 (device), n_tau <= 16; kl_out [1] float64 and counts_out [n_tau] int64 (device).
+ * Each k3 term is formed in float32 by a cancellation-free expression of (p_train - p_infer) /
+ * p_infer (relative error below 1e-5, typically 1e-7) and the terms are summed in float64 in a
+ * fixed order (reproducible); the threshold decision is taken on float32 ratios.  workspace: r3_prob_discrepancy_workspace_bytes(n). */
+size_t r3_prob_discrepancy_workspace_bytes(int64_t n);
+r3_status r3_prob_discrepancy(const float* p_train, const float* p_infer, int64_t n,
+                              const float* taus, int32_t n_tau, double* kl_out,
+                              int64_t* counts_out, void* workspace, size_t ws_bytes, void* stream);
+
+/* Section 3.2, router-level and token-level comparison of two routing records rec_a, rec_b
+ * [L, T, K] (shape->T, K, E, idx_type; K <= 32; each (layer, token) holds K distinct experts, in
+ * any slot order):
+ *   diff[l,t]        = K - |{rec_a[l,t,.]} & {rec_b[l,t,.]}|   differing expert choices of a router
+ *   hist[v]          = number of routers (l,t) with diff = v                 [K+1] int64
+ *   token_choices[t] = sum_l diff[l,t]                                       [T]   int32
+ *   token_routers[t] = number of layers l with diff[l,t] > 0                 [T]   int32
+ * diff_out [L,T] uint8 may be NULL.  All outputs are exact integers. */
+r3_status r3_record_diff(const r3_shape* shape, int32_t L, const void* rec_a, const void* rec_b,
+                         uint8_t* diff_out, int32_t* token_choices, int32_t* token_routers,
+                         int64_t* hist, void* stream);
+
+/* Section 3.2, sequence-level comparison: seq_sum[s] = sum of token_routers over the tokens
+ * [cu_seqlens[s], cu_seqlens[s+1]) of sequence s; the paper's mean difference per token of a
+ * sequence is seq_sum[s] / length.  cu_seqlens [S+1] int32 (device), seq_sum [S] int64. */
+r3_status r3_sequence_diff(const int32_t* token_routers, const int32_t* cu_seqlens, int32_t S,
+                           int64_t* seq_sum, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

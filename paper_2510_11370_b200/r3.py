@@ -35,6 +35,8 @@ EXPORTS = [
     "r3_replay_layer_workspace_bytes",
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
+    "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
+    "r3_sequence_diff",
 ]
 
 
@@ -74,6 +76,12 @@ lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_finish.argtypes = [_SP] + [_P] * 11
 lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_layer_host.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
+lib.r3_prob_discrepancy_workspace_bytes.restype = ctypes.c_size_t
+lib.r3_prob_discrepancy_workspace_bytes.argtypes = [ctypes.c_int64]
+lib.r3_prob_discrepancy.argtypes = [_P, _P, ctypes.c_int64, _P, ctypes.c_int32, _P, _P, _P,
+                                    ctypes.c_size_t, _P]
+lib.r3_record_diff.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, _P]
+lib.r3_sequence_diff.argtypes = [_P, _P, ctypes.c_int32, _P, _P]
 for _n in EXPORTS:
     if _n not in ("r3_status_string",) and not _n.endswith("_bytes"):
         getattr(lib, _n).restype = ctypes.c_int
@@ -409,3 +417,45 @@ def replay_layer_host(s: Shape, x_host, w_router, idx_host, w_gate, w_up, w_down
                                     _ptr(dlogits_host, True), _ptr(ws), ws.numel(),
                                     _ptr(dev_status), _stream(stream)))
     return y_host, dlogits_host
+
+
+# ---------------------------------------------------------------------------------------------
+def prob_discrepancy(p_train, p_infer, taus, *, kl=None, counts=None, ws=None, stream=None):
+    """k3 KL estimate (Eq. kl) and extreme-token counts (Eq. etdf) of two float32 probability
+    arrays.  `taus`: a list or a float32 device tensor.  Returns (kl [1] float64, counts [n_tau]
+    int64); F(tau) = counts / n."""
+    dev = _dev(p_train)
+    n = p_train.numel()
+    if not (isinstance(taus, torch.Tensor) and taus.is_cuda and taus.dtype == torch.float32):
+        taus = torch.as_tensor(taus, dtype=torch.float32, device=dev).contiguous()
+    if kl is None:
+        kl = torch.empty(1, dtype=torch.float64, device=dev)
+    if counts is None:
+        counts = torch.empty(taus.numel(), dtype=torch.int64, device=dev)
+    if ws is None:
+        ws = workspace(lib.r3_prob_discrepancy_workspace_bytes(n), dev)
+    _check(lib.r3_prob_discrepancy(_ptr(p_train), _ptr(p_infer), n, _ptr(taus), taus.numel(),
+                                   _ptr(kl), _ptr(counts), _ptr(ws), ws.numel(), _stream(stream)))
+    return kl, counts
+
+
+def record_diff(s: Shape, L: int, rec_a, rec_b, *, want_diff=True, stream=None):
+    """Differing expert choices between two records [L,T,K].  Returns (diff [L,T] uint8 or None,
+    token_choices [T], token_routers [T], hist [K+1] int64)."""
+    dev = _dev(rec_a)
+    diff = torch.empty((L, s.T), dtype=torch.uint8, device=dev) if want_diff else None
+    choices = torch.empty(s.T, dtype=torch.int32, device=dev)
+    routers = torch.empty(s.T, dtype=torch.int32, device=dev)
+    hist = torch.empty(s.K + 1, dtype=torch.int64, device=dev)
+    _check(lib.r3_record_diff(ctypes.byref(s), L, _ptr(rec_a), _ptr(rec_b), _ptr(diff),
+                              _ptr(choices), _ptr(routers), _ptr(hist), _stream(stream)))
+    return diff, choices, routers, hist
+
+
+def sequence_diff(token_routers, cu_seqlens, *, stream=None):
+    """Per-sequence sums of token_routers over [cu_seqlens[s], cu_seqlens[s+1])."""
+    S = cu_seqlens.numel() - 1
+    out = torch.empty(S, dtype=torch.int64, device=_dev(token_routers))
+    _check(lib.r3_sequence_diff(_ptr(token_routers), _ptr(cu_seqlens), S, _ptr(out),
+                                _stream(stream)))
+    return out
