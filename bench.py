@@ -426,6 +426,17 @@ def run_diag(args):
     ms_p = timed(lambda: r3.prob_discrepancy(pt, pi, taus_d, kl=kl_o, counts=cnt_o, ws=ws))
     ms_r = timed(lambda: r3.record_diff(s, L, a, b, want_diff=False))
     kl, counts = r3.prob_discrepancy(pt, pi, taus, ws=ws)
+    # record store (Section 4.2): packed record of 4 sequences x 65536 tokens out of 16-token pages
+    PT, Bq, Ts = 16, 4, 4 * 65536
+    n_store_pages = Ts // PT
+    page_bytes = r3.record_page_bytes(s, L, PT)
+    pages = torch.randint(0, 128, (n_store_pages * page_bytes,), dtype=torch.uint8, device=dev)
+    bt = torch.randperm(n_store_pages, generator=g, device=dev).to(torch.int32).reshape(Bq, -1).contiguous()
+    cu = torch.arange(Bq + 1, dtype=torch.int32, device=dev) * (Ts // Bq)
+    out_rec = torch.empty((L, Ts, K), dtype=torch.uint8, device=dev)
+    ms_g = timed(lambda: r3.record_gather(s, L, PT, pages, bt, cu, Ts, out=out_rec))
+    pos0 = torch.zeros(Bq, dtype=torch.int32, device=dev)
+    ms_a = timed(lambda: r3.record_append(s, L, PT, pages, bt, pos0, cu, out_rec))
     t0 = time.perf_counter()
     m = 2_000_000
     ref_kl = D.kl_k3(pt[:m].cpu().numpy(), pi[:m].cpu().numpy())
@@ -441,7 +452,11 @@ def run_diag(args):
         "kernels": {
             "prob_discrepancy": {"ms": round(ms_p, 5), "hbm_gbs": round(8 * n / ms_p / 1e6, 1)},
             "record_diff": {"ms": round(ms_r, 5),
-                            "hbm_gbs": round(2 * L * T * K / ms_r / 1e6, 1)}},
+                            "hbm_gbs": round(2 * L * T * K / ms_r / 1e6, 1)},
+            "record_gather": {"ms": round(ms_g, 5), "hbm_gbs": round(2 * L * Ts * K / ms_g / 1e6, 1),
+                              "frac_of_measured_hbm": round(2 * L * Ts * K / ms_g / 1e6 / peaks["hbm_gbs"], 3)},
+            "record_append": {"ms": round(ms_a, 5), "hbm_gbs": round(2 * L * Ts * K / ms_a / 1e6, 1),
+                              "frac_of_measured_hbm": round(2 * L * Ts * K / ms_a / 1e6 / peaks["hbm_gbs"], 3)}},
         "kl_k3": kl.item(), "F_tau": [c / n for c in counts.cpu().tolist()],
         "cpu_baseline": {"value": m / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
                          "sample": f"first {m} tokens, kl_k3 + extreme_counts in numpy",

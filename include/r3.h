@@ -60,7 +60,8 @@ typedef enum {
     R3_ERR_UNSUPPORTED = 2,   /* a legal shape this build has no kernel for */
     R3_ERR_WORKSPACE = 3,     /* workspace missing, too small or misaligned */
     R3_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
-    R3_ERR_SCRATCH_LIMIT = 5  /* the problem needs more than the library's fixed on-device scratch */
+    R3_ERR_SCRATCH_LIMIT = 5, /* the problem needs more than the library's fixed on-device scratch */
+    R3_ERR_OUT_OF_PAGES = 6   /* r3_pagepool_alloc: fewer free pages than asked for */
 } r3_status;
 
 enum { R3_F32 = 0, R3_BF16 = 1 };
@@ -311,6 +312,53 @@ r3_status r3_record_diff(const r3_shape* shape, int32_t L, const void* rec_a, co
  * sequence is seq_sum[s] / length.  cu_seqlens [S+1] int32 (device), seq_sum [S] int64. */
 r3_status r3_sequence_diff(const int32_t* token_routers, const int32_t* cu_seqlens, int32_t S,
                            int64_t* seq_sum, void* stream);
+
+/* ---- routing-record store (Section 4.2: router masks cached with the prefix KV cache) --------- */
+
+/* Records are kept in pages of `page_tokens` tokens, laid out [page][layer][token in page][slot]
+ * (r3_record_page_bytes per page) in a device buffer `pages` of n_pages pages owned by the
+ * caller.  A sequence is the list of its page numbers: row b of block_table [B, max_pages] int32
+ * (device).  Two sequences that share a prefix list the same pages for it, which is how cached
+ * masks are reused without recomputation (Section 4.2).  shape gives K and idx_type.
+ *
+ * r3_record_append (inference side): rec_new [L, N, K] holds the records of N new tokens, packed
+ * sequence after sequence (cu_new [B+1]); the tokens of sequence b go to positions seq_pos0[b],
+ * seq_pos0[b]+1, ... of that sequence.  Multi-turn use appends again to the same sequence.
+ * r3_record_gather (training side): out [L, T, K] receives the records of positions 0 ..
+ * len_b - 1 of every sequence, packed in the order of cu_seqlens [B+1] - the record that
+ * r3_replay_layer / r3_replay_blocks take.
+ * Both copy bytes (bit-exact).  dev_status (optional): R3_DEV_BAD_INDEX when a position has no
+ * page (table entry < 0, >= n_pages, or beyond max_pages); that record is skipped. */
+size_t r3_record_page_bytes(const r3_shape* shape, int32_t L, int32_t page_tokens);
+r3_status r3_record_append(const r3_shape* shape, int32_t L, int32_t page_tokens, int32_t n_pages,
+                           void* pages, const int32_t* block_table, int32_t max_pages,
+                           const int32_t* seq_pos0, const int32_t* cu_new, int32_t B,
+                           const void* rec_new, int32_t N, int32_t* dev_status, void* stream);
+r3_status r3_record_gather(const r3_shape* shape, int32_t L, int32_t page_tokens, int32_t n_pages,
+                           const void* pages, const int32_t* block_table, int32_t max_pages,
+                           const int32_t* cu_seqlens, int32_t B, void* out, int32_t T,
+                           int32_t* dev_status, void* stream);
+
+/* Host-side bookkeeping of the pages (no device work; all pointers are HOST pointers; the pool
+ * allocates host memory only, freed by r3_pagepool_destroy).  Not thread-safe.
+ *   match   : the pages of the longest already stored whole-page prefix of token_ids (use counts
+ *             go up); returns how many pages matched - their records need not be produced again
+ *   alloc   : n unused pages (use count 1), R3_ERR_OUT_OF_PAGES if fewer are free
+ *   publish : makes every full page of a sequence (token_ids = the n_tokens ids whose records the
+ *             table's pages hold) findable by later match calls; a prefix is indexed once
+ *   release : use counts go down; a page nobody uses leaves the index and becomes free
+ * A page is identified by a chained 64-bit hash of all token ids up to its end, and a match also
+ * compares the page's own ids: distinct prefixes are confused only on a hash collision. */
+typedef struct r3_pagepool r3_pagepool;
+r3_pagepool* r3_pagepool_create(int32_t n_pages, int32_t page_tokens);
+void r3_pagepool_destroy(r3_pagepool* pool);
+int32_t r3_pagepool_free_pages(const r3_pagepool* pool);
+int32_t r3_pagepool_match(r3_pagepool* pool, const int32_t* token_ids, int32_t n_tokens,
+                          int32_t* pages_out, int32_t max_pages);
+r3_status r3_pagepool_alloc(r3_pagepool* pool, int32_t n, int32_t* pages_out);
+r3_status r3_pagepool_publish(r3_pagepool* pool, const int32_t* token_ids, int32_t n_tokens,
+                              const int32_t* table, int32_t n_table);
+r3_status r3_pagepool_release(r3_pagepool* pool, const int32_t* table, int32_t n);
 
 #ifdef __cplusplus
 }

@@ -327,6 +327,7 @@ extern "C" const char* r3_status_string(r3_status s) {
         case R3_ERR_UNSUPPORTED: return "R3_ERR_UNSUPPORTED: no kernel for this shape";
         case R3_ERR_WORKSPACE: return "R3_ERR_WORKSPACE: workspace missing, too small or misaligned";
         case R3_ERR_CUDA: return "R3_ERR_CUDA: a CUDA call failed";
+        case R3_ERR_OUT_OF_PAGES: return "R3_ERR_OUT_OF_PAGES: not enough free record pages";
         case R3_ERR_SCRATCH_LIMIT:
             return "R3_ERR_SCRATCH_LIMIT: E * ceil(T/256) exceeds the 262144 counters of the "
                    "library's fixed scratch; use r3_permute with a caller workspace";

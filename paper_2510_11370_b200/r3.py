@@ -36,7 +36,9 @@ EXPORTS = [
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
-    "r3_sequence_diff",
+    "r3_sequence_diff", "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
+    "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
+    "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
 ]
 
 
@@ -82,8 +84,23 @@ lib.r3_prob_discrepancy.argtypes = [_P, _P, ctypes.c_int64, _P, ctypes.c_int32, 
                                     ctypes.c_size_t, _P]
 lib.r3_record_diff.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, _P]
 lib.r3_sequence_diff.argtypes = [_P, _P, ctypes.c_int32, _P, _P]
+_I32 = ctypes.c_int32
+lib.r3_record_page_bytes.restype = ctypes.c_size_t
+lib.r3_record_page_bytes.argtypes = [_SP, _I32, _I32]
+lib.r3_record_append.argtypes = [_SP, _I32, _I32, _I32, _P, _P, _I32, _P, _P, _I32, _P, _I32, _P, _P]
+lib.r3_record_gather.argtypes = [_SP, _I32, _I32, _I32, _P, _P, _I32, _P, _I32, _P, _I32, _P, _P]
+lib.r3_pagepool_create.restype = ctypes.c_void_p
+lib.r3_pagepool_create.argtypes = [_I32, _I32]
+lib.r3_pagepool_destroy.restype = None
+lib.r3_pagepool_destroy.argtypes = [_P]
+lib.r3_pagepool_free_pages.argtypes = [_P]
+lib.r3_pagepool_match.argtypes = [_P, _P, _I32, _P, _I32]
+lib.r3_pagepool_alloc.argtypes = [_P, _I32, _P]
+lib.r3_pagepool_publish.argtypes = [_P, _P, _I32, _P, _I32]
+lib.r3_pagepool_release.argtypes = [_P, _P, _I32]
+_NOT_STATUS = ("r3_status_string", "r3_pagepool_create", "r3_pagepool_destroy")
 for _n in EXPORTS:
-    if _n not in ("r3_status_string",) and not _n.endswith("_bytes"):
+    if _n not in _NOT_STATUS and not _n.endswith("_bytes"):
         getattr(lib, _n).restype = ctypes.c_int
 
 
@@ -459,3 +476,73 @@ def sequence_diff(token_routers, cu_seqlens, *, stream=None):
     _check(lib.r3_sequence_diff(_ptr(token_routers), _ptr(cu_seqlens), S, _ptr(out),
                                 _stream(stream)))
     return out
+
+
+# ---------------------------------------------------------------------------------------------
+def record_page_bytes(s: Shape, L: int, page_tokens: int) -> int:
+    return lib.r3_record_page_bytes(ctypes.byref(s), L, page_tokens)
+
+
+def record_append(s: Shape, L: int, page_tokens: int, pages, block_table, seq_pos0, cu_new,
+                  rec_new, *, dev_status=None, stream=None):
+    """Writes rec_new [L, N, K] (N new tokens, packed by cu_new) into the pages of their sequences."""
+    n_pages = pages.numel() // record_page_bytes(s, L, page_tokens)
+    B, max_pages = block_table.shape
+    _check(lib.r3_record_append(ctypes.byref(s), L, page_tokens, n_pages, _ptr(pages),
+                                _ptr(block_table), max_pages, _ptr(seq_pos0), _ptr(cu_new), B,
+                                _ptr(rec_new), rec_new.shape[1], _ptr(dev_status), _stream(stream)))
+
+
+def record_gather(s: Shape, L: int, page_tokens: int, pages, block_table, cu_seqlens, T: int, *,
+                  out=None, dev_status=None, stream=None):
+    """The packed record [L, T, K] of a variable-length batch, assembled from the pages."""
+    n_pages = pages.numel() // record_page_bytes(s, L, page_tokens)
+    B, max_pages = block_table.shape
+    if out is None:
+        out = torch.empty((L, T, s.K), dtype=_idx_dtype(s), device=_dev(pages))
+    _check(lib.r3_record_gather(ctypes.byref(s), L, page_tokens, n_pages, _ptr(pages),
+                                _ptr(block_table), max_pages, _ptr(cu_seqlens), B, _ptr(out), T,
+                                _ptr(dev_status), _stream(stream)))
+    return out
+
+
+class PagePool:
+    """Host-side page bookkeeping of the record store (r3_pagepool_*): lists in, lists out."""
+
+    def __init__(self, n_pages: int, page_tokens: int):
+        self.page_tokens = page_tokens
+        self._h = lib.r3_pagepool_create(n_pages, page_tokens)
+        if not self._h:
+            raise ValueError("r3_pagepool_create failed")
+
+    def close(self):
+        if self._h:
+            lib.r3_pagepool_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    @staticmethod
+    def _arr(v):
+        return (ctypes.c_int32 * max(len(v), 1))(*v)
+
+    def free_pages(self) -> int:
+        return lib.r3_pagepool_free_pages(self._h)
+
+    def match(self, token_ids) -> list:
+        cap = len(token_ids) // self.page_tokens
+        out = (ctypes.c_int32 * max(cap, 1))()
+        n = lib.r3_pagepool_match(self._h, self._arr(token_ids), len(token_ids), out, cap)
+        return list(out[:n])
+
+    def alloc(self, n: int) -> list:
+        out = (ctypes.c_int32 * max(n, 1))()
+        _check(lib.r3_pagepool_alloc(self._h, n, out))
+        return list(out[:n])
+
+    def publish(self, token_ids, table) -> None:
+        _check(lib.r3_pagepool_publish(self._h, self._arr(token_ids), len(token_ids),
+                                       self._arr(table), len(table)))
+
+    def release(self, table) -> None:
+        _check(lib.r3_pagepool_release(self._h, self._arr(table), len(table)))
