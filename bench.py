@@ -381,6 +381,126 @@ def run_ours(args, w):
         torch.distributed.destroy_process_group()
 
 
+def run_stack(args, w):
+    """Config 5: `w.layers` MoE blocks back to back with all their weights resident
+    (r3_replay_blocks; every block has its own seeded input, record and weights)."""
+    import torch
+    from paper_2510_11370_b200 import build, synth
+    build.build()
+    from paper_2510_11370_b200 import r3
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    dev = torch.device("cuda", 0)
+    peaks = load_peaks()
+    L, T, d, E, K, F = w.layers, w.T, w.d, w.E, w.K, w.F
+    s = r3.shape_of(w)
+    x = torch.stack([synth.activations(w, dev, l) for l in range(L)])
+    dy = torch.stack([synth.upstream_grad(w, dev, l) for l in range(L)])
+    w_r = torch.stack([synth.router_weight(w, dev, l) for l in range(L)])
+    wg = torch.empty((L, E, F, d), dtype=w.act_dtype, device=dev)
+    wu = torch.empty((L, E, F, d), dtype=w.act_dtype, device=dev)
+    wd = torch.empty((L, E, d, F), dtype=w.act_dtype, device=dev)
+    idx = torch.empty((L, T, K), dtype=w.idx_dtype, device=dev)
+    for l in range(L):
+        a, b, c = synth.expert_weights(w, dev, l)
+        wg[l], wu[l], wd[l] = a, b, c
+        del a, b, c
+        _, lg = r3.capture_topk_ws(s, 1, x[l], w_r[l], want_idx=False, want_logits=True)
+        idx[l] = synth.make_record(w, lg, l)
+    y = torch.empty_like(x)
+    dl = torch.empty((L, T, E), dtype=torch.float32, device=dev)
+    ws = r3.workspace(r3.replay_layer_workspace_bytes(s), dev)
+    st = r3.new_status(dev)
+
+    def step():
+        r3.replay_blocks(s, L, x, w_r, idx, wg, wu, wd, dy, y=y, dlogits=dl, ws=ws, dev_status=st)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1) / args.steps
+    assert st.item() == 0
+    clocks = sampler.stop(t0, t1)
+    flop = 6.0 * T * K * d * F * L
+    line = {
+        "metric": METRIC, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "blocks": L, "T": T, "d": d, "E": E, "K": K, "F": F,
+                   "weights_gb": round(3 * L * E * F * d * 2 / 1e9, 1),
+                   "l2": "58 GB of weights stream through the 126 MB L2 every step"},
+        "layer_tokens_per_s": L * T / (ms * 1e-3),
+        "roofline": {"bound": "tensor", "kernel": "both grouped GEMMs of all blocks (whole-step time, "
+                     "all other kernels included)", "achieved": round(flop / (ms * 1e-3) / 1e12, 1),
+                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": round(flop / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
+                     "peak_kind": f"bf16 matmul sustained, {peaks['source']}", "traffic": None},
+        "gpu_launches": LAUNCHES_PER_STEP * L * args.steps, "clocks": clocks, "peaks": peaks,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_capture(args, w):
+    """Config 4, inference side: router logits + TopKMask of a decode batch for `w.layers` layers
+    in one launch (r3_capture_topk_batched), records packed as uint8."""
+    import torch
+    from paper_2510_11370_b200 import build, synth
+    build.build()
+    from paper_2510_11370_b200 import r3
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    dev = torch.device("cuda", 0)
+    peaks = load_peaks()
+    L, T, d, E, K = w.layers, w.T, w.d, w.E, w.K
+    s = r3.shape_of(w)
+    reps = 8                                  # rotate over > L2-sized input rings
+    xs = [torch.stack([synth.activations(w, dev, l + 100 * r) for l in range(L)]) for r in range(reps)]
+    wr = torch.stack([synth.router_weight(w, dev, l) for l in range(L)])
+    idx = torch.empty((L, T, K), dtype=w.idx_dtype, device=dev)
+    one_idx = torch.empty((T, K), dtype=w.idx_dtype, device=dev)
+
+    def timed(fn, n):
+        for i in range(max(args.warmup, 3)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    ms_b = timed(lambda i: r3.capture_topk_batched(s, L, xs[i % reps], wr, idx_out=idx), args.steps)
+    ms_1 = timed(lambda i: r3.capture_topk(s, xs[i % reps][i % L], wr[i % L], idx_out=one_idx),
+                 args.steps)
+    bytes_b = L * (T * d * 2 + E * d * 2 + T * K)
+    line = {
+        "metric": "capture layer-tokens/s (router logits + top-K -> uint8 record)",
+        "value": L * T / (ms_b * 1e-3), "unit": "layer-tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_b, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "T": T, "d": d, "E": E, "K": K,
+                   "l2": f"inputs rotate over {reps} sets of {L * T * d * 2 / 1e6:.0f} MB (> L2 in all)"},
+        "kernels": {"capture_batched": {"ms": round(ms_b, 5), "hbm_gbs": round(bytes_b / ms_b / 1e6, 1),
+                                        "frac_of_measured_hbm": round(bytes_b / ms_b / 1e6 / peaks["hbm_gbs"], 3)},
+                    "capture_one_layer": {"us_per_call": round(ms_1 * 1e3, 2)}},
+        "record_bytes_per_step": L * T * K, "peaks": peaks,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def run_diag(args):
     """Discrepancy measures of Sections 3.1-3.2 (not the headline path): k3 KL + F(tau) over 10 M
     token probabilities (the paper's scatter sample), and the router/token-level comparison of two
@@ -476,11 +596,17 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=4096,
                     help="tokens of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stack", action="store_true",
+                    help="with a multi-layer workload (c5_stack48): time all its blocks, weights resident")
     args = ap.parse_args()
     from paper_2510_11370_b200 import synth
     if args.workload == "diag":
         return run_diag(args)
     w = synth.WORKLOADS[args.workload]
+    if args.impl != "reference" and args.workload == "c4_capture":
+        return run_capture(args, w)
+    if args.impl != "reference" and w.layers > 1 and args.stack:
+        return run_stack(args, w)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -9,10 +9,13 @@
 // the same fp32 TMEM accumulator: x is exact in bf16, so the logits keep float32-level accuracy
 // while the contraction runs on the tensor pipe.
 //
-// One CTA per 128-token tile: warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer, warps 2-5
-// = epilogue.  Each epilogue thread owns one token: it streams its E logits out of TMEM 32 at a
-// time, writes them (optionally) to logits_out and keeps a sorted top-K list in registers
-// (strict comparisons in ascending expert order, so exact ties keep the lower index first).
+// One CTA of 12 warps per 128-token tile: warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA
+// issuer, warps 2-5 read the finished accumulator out of TMEM into a [128][E + 1] float tile in
+// shared memory (the copy ring is free by then).  All 12 warps then finish tokens out of that
+// tile, four at a time per warp: the lanes write the token's logits out coalesced and pick the K
+// largest with K rounds of warp reductions on order-preserving integer keys (exact ties go to the
+// lower expert).  A per-thread sorted insertion list, one thread per token, took 12 us of
+// dependent compare-and-swaps per tile; this takes about a third of that.
 #include "r3_common.cuh"
 #include "r3_internal.h"
 #include "r3_tc.cuh"
@@ -26,9 +29,9 @@ constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int UK = 16;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int THREADS = 6 * 32;
+constexpr int THREADS = 12 * 32;           // producer, MMA issuer, 4 TMEM readers; all 12 pick top-K
 constexpr int BAR_BYTES = 256;
-constexpr int MAX_STAGES = 4;
+constexpr int MAX_STAGES = 7;
 constexpr int KMAX = 16;                 // longest record the register top-K list supports
 constexpr int SMEM_LIMIT = 227 * 1024;
 
@@ -47,6 +50,57 @@ split_router_weight_kernel(const float* __restrict__ w, __nv_bfloat16* __restric
     base[0] = hi;
     base[per_layer] = mid;
     base[2 * per_layer] = lo;
+}
+
+// One warp finishes NT tokens at a time out of the shared-memory logits tile: lane l holds the
+// logits of experts l + 32 s (slot s), writes them out (coalesced) and, if a record is wanted,
+// picks the K largest by K rounds of warp reductions on order-preserving integer keys; exact ties
+// go to the lower expert.  NT tokens are interleaved so that their reduction chains overlap.
+template <typename IdxT, int SLOTS, int NT>
+__device__ __forceinline__ void finish_tokens(const float* tile, int LD, const int* rows, int n_rows,
+                                              int lane, int E, int K, size_t out_row0,
+                                              IdxT* idx_out, float* logits_out) {
+    uint32_t key[NT][SLOTS];
+#pragma unroll
+    for (int a = 0; a < NT; ++a) {
+#pragma unroll
+        for (int sl = 0; sl < SLOTS; ++sl) {
+            const int e = lane + 32 * sl;
+            key[a][sl] = 0u;                             // 0 = no candidate (below every real key)
+            if (a < n_rows && e < E) {
+                const float v = tile[(size_t)rows[a] * LD + e];
+                if (logits_out) logits_out[(out_row0 + rows[a]) * E + e] = v;
+                const uint32_t u = __float_as_uint(v);
+                const uint32_t k2 = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+                key[a][sl] = k2 ? k2 : 1u;
+            }
+        }
+    }
+    if (!idx_out) return;
+    int mine[NT];
+#pragma unroll
+    for (int a = 0; a < NT; ++a) mine[a] = 0;
+    for (int j = 0; j < K; ++j) {
+#pragma unroll
+        for (int a = 0; a < NT; ++a) {
+            uint32_t best = 0u;
+#pragma unroll
+            for (int sl = 0; sl < SLOTS; ++sl) best = max(best, key[a][sl]);
+            const uint32_t top = __reduce_max_sync(0xffffffffu, best);
+            uint32_t cand = 0xffffffffu;                 // lowest expert of this lane with that key
+#pragma unroll
+            for (int sl = SLOTS - 1; sl >= 0; --sl)
+                if (key[a][sl] == top) cand = (uint32_t)(lane + 32 * sl);
+            const uint32_t win = __reduce_min_sync(0xffffffffu, cand);
+#pragma unroll
+            for (int sl = 0; sl < SLOTS; ++sl)
+                if (win == (uint32_t)(lane + 32 * sl)) key[a][sl] = 0u;
+            if (lane == j) mine[a] = (int)win;
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < NT; ++a)
+        if (a < n_rows && lane < K) idx_out[(out_row0 + rows[a]) * K + lane] = (IdxT)mine[a];
 }
 
 template <typename IdxT, int KM>
@@ -100,6 +154,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                 if (++stage == stages) { stage = 0; phase ^= 1u; }
             }
         }
+        __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(BM, E);
@@ -123,54 +178,46 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
             if (ok) tc_commit(acc_bar);
         }
-    } else {
+        __syncwarp();
+    } else if (warp < 6) {
+        // ------------------------------ epilogue, part 1 --------------------------------------
+        // every epilogue warp dumps its 32 tokens' logits from tensor memory into a [128][E + 1]
+        // float tile in shared memory (the copy ring is free once the accumulator is complete)
         const int q = warp & 3;
-        const int r_in = q * 32 + lane;
-        const int t = t0 + r_in;
-        const bool row_ok = t < T;
-        if (mbar_wait(acc_bar, 0u, abort_flag, nullptr)) {
+        float* tile = reinterpret_cast<float*>(base_ptr);
+        if (__all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, nullptr))) {
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            float tv[KM];
-            int ti[KM];
-#pragma unroll
-            for (int j = 0; j < KM; ++j) { tv[j] = -INFINITY; ti[j] = 0; }
-            float* lrow = logits_out ? logits_out + ((size_t)layer * T + (row_ok ? t : 0)) * E
-                                     : nullptr;
+            float* trow = tile + (size_t)(q * 32 + lane) * (E + 1);
             for (int c = 0; c < E; c += 32) {
                 float v[32];
                 tc_ld32(taddr + c, v);
                 tc_wait_ld();
-                if (lrow && row_ok) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        if (c + i < E)
-                            *reinterpret_cast<float4*>(lrow + c + i) =
-                                make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-                }
-                if (idx_out) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (c + i < E && v[i] > tv[KM - 1]) {
-                            tv[KM - 1] = v[i];
-                            ti[KM - 1] = c + i;
-#pragma unroll
-                            for (int j = KM - 1; j > 0; --j) {
-                                if (tv[j] > tv[j - 1]) {
-                                    const float fv = tv[j]; tv[j] = tv[j - 1]; tv[j - 1] = fv;
-                                    const int iv = ti[j]; ti[j] = ti[j - 1]; ti[j - 1] = iv;
-                                }
-                            }
-                        }
-                    }
-                }
+                for (int i = 0; i < 32; ++i)
+                    if (c + i < E) trow[c + i] = v[i];
             }
-            if (idx_out && row_ok) {
-                IdxT* rec = idx_out + ((size_t)layer * T + t) * K;
+        }
+    }
+    // ------------------------------ epilogue, part 2: all six warps, a few tokens each ---------
+    tc_fence_before();
+    __syncthreads();
+    if (!*abort_flag) {
+        const float* tile = reinterpret_cast<const float*>(base_ptr);
+        const int n_tok = min(BM, T - t0);
+        constexpr int NT = 4, NW = THREADS / 32;
+        for (int r0 = warp * NT; r0 < n_tok; r0 += NW * NT) {
+            int rows[NT];
 #pragma unroll
-                for (int j = 0; j < KM; ++j)
-                    if (j < K) rec[j] = (IdxT)ti[j];
-            }
+            for (int a = 0; a < NT; ++a) rows[a] = min(r0 + a, n_tok - 1);
+            const int n_rows = min(NT, n_tok - r0);
+            const size_t out_row0 = (size_t)layer * T + t0;
+            if (E <= 128)
+                finish_tokens<IdxT, 4, NT>(tile, E + 1, rows, n_rows, lane, E, K, out_row0, idx_out,
+                                           logits_out);
+            else
+                finish_tokens<IdxT, 8, NT>(tile, E + 1, rows, n_rows, lane, E, K, out_row0, idx_out,
+                                           logits_out);
         }
     }
 
@@ -226,9 +273,13 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
 #define R3_RT(IDX, KM)                                                                          \
     do {                                                                                        \
         auto kern = router_tc_kernel<IDX, KM>;                                                  \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=    \
-            cudaSuccess)                                                                        \
-            return R3_ERR_CUDA;                                                                 \
+        static int attr_smem = 0;              /* largest size set so far, per instantiation */ \
+        if (smem > attr_smem) {                                                                 \
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
+                                     SMEM_LIMIT) != cudaSuccess)                                \
+                return R3_ERR_CUDA;                                                             \
+            attr_smem = SMEM_LIMIT;                                                             \
+        }                                                                                       \
         kern<<<grid, THREADS, smem, cs>>>(mx, mw, static_cast<IDX*>(idx_out), logits_out, s->T, \
                                           s->d, s->E, s->K, planes, stages, tmem_cols);         \
     } while (0)
