@@ -298,3 +298,50 @@ def replay_stack_tokens(x_rows, layers, dy_rows, store=None):
         if store is not None:
             x = _f64(store(x))
     return x, dss
+
+
+# ----------------------------------------------------------------------------------------------
+# Update-stage backward to the layer input and the router weight (Section 4.1, purpose (b):
+# the mask I_infer is a constant, everything else is differentiated)
+# ----------------------------------------------------------------------------------------------
+def dsilu(z: np.ndarray) -> np.ndarray:
+    """d silu / dz = sigma(z) (1 + z (1 - sigma(z)))."""
+    sg = 1.0 / (1.0 + np.exp(-z))
+    return sg * (1.0 + z * (1.0 - sg))
+
+
+def swiglu_expert_bwd_input(x, do, w_gate_i, w_up_i, w_down_i) -> np.ndarray:
+    """dL/dx for o = E_i(x) given dL/do, by the chain rule through
+    a = W_gate x, b = W_up x, h = silu(a) b, o = W_down h."""
+    x, do = _f64(x), _f64(do)
+    wg, wu, wd = _f64(w_gate_i), _f64(w_up_i), _f64(w_down_i)
+    a, b = x @ wg.T, x @ wu.T
+    dh = do @ wd                                   # [n, F]
+    da = dh * b * dsilu(a)
+    db = dh * silu(a)
+    return da @ wg + db @ wu
+
+
+def layer_bwd_input(x, w_r, idx_infer, w_gate, w_up, w_down, dy):
+    """Gradients of  L = <dy, y_replay(x)>  (any loss whose gradient at y is dy) with the recorded
+    mask held constant:
+        dx   [T, d]  = sum_j g_j dE_{e_j}/dx^T dy   (expert path)  +  ds W_r   (router path)
+        dW_r [E, d]  = ds^T x
+        ds   [T, E]  as replay_gate_bwd.
+    Returns a dict with dx, dw_r, ds, dx_expert, dx_router."""
+    x, dy, w_r = _f64(x), _f64(dy), _f64(w_r)
+    idx = np.asarray(idx_infer, dtype=np.int64)
+    T, K = idx.shape
+    E = w_r.shape[0]
+    f = layer_fwd_bwd(x, w_r, idx, w_gate, w_up, w_down, dy)
+    dx_e = np.zeros_like(x)
+    for i in range(E):
+        tt, jj = np.nonzero(idx == i)
+        if tt.size == 0:
+            continue
+        do = f["g"][tt, jj][:, None] * dy[tt]      # dL/d(E_i(x_t)) = g_{t,j} dy_t
+        contrib = swiglu_expert_bwd_input(x[tt], do, w_gate[i], w_up[i], w_down[i])
+        np.add.at(dx_e, tt, contrib)
+    dx_r = f["ds"] @ w_r
+    return dict(dx=dx_e + dx_r, dw_r=f["ds"].T @ x, ds=f["ds"], dx_expert=dx_e, dx_router=dx_r,
+                y=f["y"], g=f["g"])

@@ -389,3 +389,77 @@ def test_pins_catch_planted_mistakes(monkeypatch):
     # gates from other logits change the output
     other = O.replay_output(x, s + rng(1).standard_normal(s.shape), idx, wg, wu, wd)[0]
     assert not np.allclose(good, other)
+
+
+# ---------------------------------------------------------------------------------------------
+# Update-stage backward to the layer input and the router weight
+# ---------------------------------------------------------------------------------------------
+def _tiny_layer(seed, T=5, d=6, E=4, K=2, F=5):
+    rng = np.random.default_rng(seed)
+    x = rng.normal(size=(T, d))
+    w_r = rng.normal(size=(E, d)) * 0.5
+    wg = rng.normal(size=(E, F, d)) * 0.4
+    wu = rng.normal(size=(E, F, d)) * 0.4
+    wd = rng.normal(size=(E, d, F)) * 0.4
+    dy = rng.normal(size=(T, d))
+    idx = np.stack([rng.permutation(E)[:K] for _ in range(T)])
+    return x, w_r, idx, wg, wu, wd, dy
+
+
+def _loss(x, w_r, idx, wg, wu, wd, dy):
+    s = O.router_logits(x, w_r)
+    y, _, _ = O.replay_output(x, s, idx, wg, wu, wd)
+    return float(np.sum(dy * y))
+
+
+def test_dsilu_is_the_derivative_of_silu():
+    z = np.linspace(-6, 6, 41)
+    h = 1e-6
+    assert np.allclose(O.dsilu(z), (O.silu(z + h) - O.silu(z - h)) / (2 * h), atol=1e-8)
+
+
+def test_input_gradient_matches_central_differences():
+    x, w_r, idx, wg, wu, wd, dy = _tiny_layer(0)
+    got = O.layer_bwd_input(x, w_r, idx, wg, wu, wd, dy)
+    h = 1e-6
+    num = np.zeros_like(x)
+    for t in range(x.shape[0]):
+        for c in range(x.shape[1]):
+            xp, xm = x.copy(), x.copy()
+            xp[t, c] += h
+            xm[t, c] -= h
+            num[t, c] = (_loss(xp, w_r, idx, wg, wu, wd, dy) - _loss(xm, w_r, idx, wg, wu, wd, dy)) / (2 * h)
+    assert np.abs(got["dx"] - num).max() / np.abs(num).max() < 1e-7
+    assert np.allclose(got["dx"], got["dx_expert"] + got["dx_router"])
+
+
+def test_router_weight_gradient_matches_central_differences():
+    x, w_r, idx, wg, wu, wd, dy = _tiny_layer(1)
+    got = O.layer_bwd_input(x, w_r, idx, wg, wu, wd, dy)
+    h = 1e-6
+    num = np.zeros_like(w_r)
+    for e in range(w_r.shape[0]):
+        for c in range(w_r.shape[1]):
+            wp, wm = w_r.copy(), w_r.copy()
+            wp[e, c] += h
+            wm[e, c] -= h
+            num[e, c] = (_loss(x, wp, idx, wg, wu, wd, dy) - _loss(x, wm, idx, wg, wu, wd, dy)) / (2 * h)
+    assert np.abs(got["dw_r"] - num).max() / np.abs(num).max() < 1e-7
+
+
+def test_input_gradient_special_cases():
+    x, w_r, idx, wg, wu, wd, dy = _tiny_layer(2, K=1)
+    got = O.layer_bwd_input(x, w_r, idx, wg, wu, wd, dy)
+    assert np.all(got["dx_router"] == 0) and np.all(got["dw_r"] == 0)   # K = 1: the gate is 1
+    # and the expert path is then the gradient of one SwiGLU MLP per token (torch autograd, float64)
+    xt = torch.tensor(x, requires_grad=True)
+    out = torch.zeros(())
+    for t in range(x.shape[0]):
+        e = int(idx[t, 0])
+        hmid = torch.nn.functional.silu(xt[t] @ torch.tensor(wg[e]).T) * (xt[t] @ torch.tensor(wu[e]).T)
+        out = out + (torch.tensor(dy[t]) * (hmid @ torch.tensor(wd[e]).T)).sum()
+    out.backward()
+    assert np.allclose(got["dx"], xt.grad.numpy(), atol=1e-12)
+    # zero upstream gradient -> zero gradients
+    z = O.layer_bwd_input(x, w_r, idx, wg, wu, wd, np.zeros_like(dy))
+    assert np.all(z["dx"] == 0) and np.all(z["dw_r"] == 0)
