@@ -279,6 +279,24 @@ r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host, const 
                                float* dlogits_host, void* workspace, size_t ws_bytes,
                                int32_t* dev_status, void* stream);
 
+/* ---- Update-stage backward to the layer input (Section 4.1, purpose (b)) ------------------------ */
+
+/* Input gradient of the expert networks on the grouped rows.  With a = xp W_gate,e^T,
+ * b = xp W_up,e^T (the forward's pre-activations), h = silu(a) * b, o = h W_down,e^T and a
+ * gradient dout = dL/do:
+ *   dh  = dout W_down,e ;  da = dh * b * silu'(a) ;  db = dh * silu(a) ;
+ *   dxp = da W_gate,e + db W_up,e                                   (= dL/dxp)
+ * dout, dxp [R,d]; pre_gate, pre_up [R,F] (as stored by the forward, bf16); weights as in
+ * r3_grouped_swiglu (read transposed in place, no transposed copy is made).  bf16 only
+ * (R3_ERR_UNSUPPORTED for float32).  dh, da, db are rounded to bf16 once each.
+ * workspace: r3_grouped_swiglu_bwd_workspace_bytes(shape). */
+size_t r3_grouped_swiglu_bwd_workspace_bytes(const r3_shape* shape);
+r3_status r3_grouped_swiglu_bwd_input(const r3_shape* shape, const void* dout, const void* pre_gate,
+                                      const void* pre_up, const int32_t* offsets,
+                                      const void* w_gate, const void* w_up, const void* w_down,
+                                      void* dxp, void* workspace, size_t ws_bytes,
+                                      int32_t* dev_status, void* stream);
+
 /* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */
 
 /* Eq. (kl), the k3 estimate of KL(pi_train || pi_infer), and Eq. (etdf), the Extreme Token

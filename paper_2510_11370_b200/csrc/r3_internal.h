@@ -40,6 +40,15 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const 
                                    void* h, void* o, void* work, int32_t* dev_status, int phases,
                                    cudaStream_t stream);
 
+// Input gradient of the grouped SwiGLU experts on the tensor cores (bf16): dout [R,d] -> dxp [R,d]
+// with the forward's pre-activations pre_gate, pre_up [R,F].  `work`: tc_bwd_work_bytes().
+size_t tc_bwd_work_bytes(const r3_shape* shape);
+r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* shape, const void* dout, const void* pre_gate,
+                                       const void* pre_up, const int32_t* offsets,
+                                       const void* w_gate, const void* w_up, const void* w_down,
+                                       void* dxp, void* work, int32_t* dev_status,
+                                       cudaStream_t stream);
+
 // Router logits + top-K on the tensor cores (bf16 activations, E a multiple of 16 up to 256,
 // K <= 16).  float32 router weights need router_tc_workspace_bytes() of scratch for their three
 // bf16 planes; bf16 router weights need none.

@@ -2,6 +2,12 @@
 //
 //   MODE 0:  h[r, f]  = silu(xp[r] . W_gate,e[f]) * (xp[r] . W_up,e[f])      (K = d, out = F)
 //   MODE 1:  o[r, c]  = h[r] . W_down,e[c]                                    (K = F, out = d)
+// and the two input-gradient GEMMs of the Update stage, whose weight operand is read TRANSPOSED
+// (MN-major shared-memory tiles straight from the forward layout, no transposed copy):
+//   MODE 2:  dh[r, f] = sum_c do[r, c] W_down,e[c, f]                         (K = d, out = F)
+//   MODE 3:  dxp[r, c] = sum_f da[r, f] W_gate,e[f, c] + db[r, f] W_up,e[f, c] (K = 2F, out = d;
+//            k blocks alternate between (W_gate, da) and (W_up, db); da, db = planes 0, 1 of one
+//            [2, R, F] array)
 //
 // Orientation.  The WEIGHT rows are the M side of the MMA and the TOKEN rows are the N side, so
 // the accumulator holds out^T: tensor-memory lane = output feature, column = token.  M is fixed
@@ -157,7 +163,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
     const int w_step = gridDim.x >> 1;
     const int w_begin = pair, w_end = list[0];
     const int4* items = reinterpret_cast<const int4*>(list + kHeaderInts);
-    const int kblocks = (Kdim + BK - 1) / BK;
+    // MODE 3 walks the k blocks of both weight matrices alternately
+    const int kblocks = (MODE == 3 ? 2 : 1) * ((Kdim + BK - 1) / BK);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -255,11 +262,23 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
                         const int f0 = f * FEAT0 + (int)rank * (BMF / 2);
                         tma_load_3d_pair(sa, &maps.a0, kb * BK, f0, e, lead_full);
                         tma_load_3d_pair(sa + A_BYTES / 2, &maps.a1, kb * BK, f0, e, lead_full);
-                    } else {
+                    } else if (MODE == 1) {
                         tma_load_3d_pair(sa, &maps.a0, kb * BK, f * FEAT1 + (int)rank * BMF, e,
                                          lead_full);
+                    } else {
+                        // transposed weights: two boxes of 64 output features x 64 k rows
+                        const int which = MODE == 3 ? (kb & 1) : 0;
+                        const int kk = MODE == 3 ? (kb >> 1) : kb;
+                        const CUtensorMap* amap = which ? &maps.a1 : &maps.a0;
+                        const int m0 = f * FEAT1 + (int)rank * BMF;
+                        tma_load_3d_pair(sa, amap, m0, kk * BK, e, lead_full);
+                        tma_load_3d_pair(sa + A_BYTES / 2, amap, m0 + 64, kk * BK, e, lead_full);
                     }
-                    tma_load_2d_pair(sb, bmap, kb * BK, it.y + (int)rank * half, lead_full);
+                    if (MODE == 3)
+                        tma_load_3d_pair(sb, bmap, (kb >> 1) * BK, it.y + (int)rank * half, kb & 1,
+                                         lead_full);
+                    else
+                        tma_load_2d_pair(sb, bmap, kb * BK, it.y + (int)rank * half, lead_full);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -278,7 +297,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
             bool ok = true;
             for (int w = w_begin; ok && w < w_end; w += w_step) {
                 const int n = items[w].z;
-                const uint32_t idesc = instr_desc_bf16(2 * BMF, n);
+                const uint32_t idesc = instr_desc_bf16(2 * BMF, n) | (MODE >= 2 ? kInstrDescAMajorMN : 0u);
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNT);
@@ -289,12 +308,16 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
                     }
                     tc_fence_after();
                     const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sb);
+                    const uint64_t da = MODE >= 2 ? smem_desc_mn_sw128(sa, A_BYTES / 2)
+                                                  : smem_desc_sw128(sa);
+                    const uint64_t db = smem_desc_sw128(sb);
+                    // per MMA (16 along k): K-major tiles move 32 bytes inside the swizzled row,
+                    // the MN-major tile moves two groups of 8 k rows = 2048 bytes
+                    constexpr uint64_t a_step = MODE >= 2 ? (2048 >> 4) : 2;
 #pragma unroll
                     for (int kk = 0; kk < BK / UK; ++kk) {
-                        // 16 bf16 = 32 bytes further along k inside the swizzled row
-                        tc_mma_bf16_pair(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
-                                         idesc, (kb | kk) != 0 ? 1u : 0u);
+                        tc_mma_bf16_pair(d_tmem, da + a_step * kk, db + (uint64_t)(kk * 2), idesc,
+                                         (kb | kk) != 0 ? 1u : 0u);
                     }
                     tc_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -483,6 +506,33 @@ static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* lis
                               dev_status) == cudaSuccess ? R3_OK : R3_ERR_CUDA;
 }
 
+// Backward of h = silu(a) * b:  da = dh * b * silu'(a),  db = dh * silu(a), written as planes 0
+// and 1 of dab [2, R, F].  16-byte vectors; F is a multiple of 8.
+__global__ void __launch_bounds__(256)
+swiglu_bwd_kernel(const uint4* __restrict__ dh, const uint4* __restrict__ a,
+                  const uint4* __restrict__ b, uint4* __restrict__ dab, long long n_vec) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_vec) return;
+    const uint4 vd = dh[i], va = a[i], vb = b[i];
+    uint4 oa, ob;
+    const __nv_bfloat162* pd = reinterpret_cast<const __nv_bfloat162*>(&vd);
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&va);
+    const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&vb);
+    __nv_bfloat162* qa = reinterpret_cast<__nv_bfloat162*>(&oa);
+    __nv_bfloat162* qb = reinterpret_cast<__nv_bfloat162*>(&ob);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 fd = __bfloat1622float2(pd[k]), fa = __bfloat1622float2(pa[k]),
+                     fb = __bfloat1622float2(pb[k]);
+        const float s0 = 1.f / (1.f + __expf(-fa.x)), s1 = 1.f / (1.f + __expf(-fa.y));
+        qa[k] = __floats2bfloat162_rn(fd.x * fb.x * s0 * (1.f + fa.x * (1.f - s0)),
+                                      fd.y * fb.y * s1 * (1.f + fa.y * (1.f - s1)));
+        qb[k] = __floats2bfloat162_rn(fd.x * fa.x * s0, fd.y * fa.y * s1);
+    }
+    dab[i] = oa;
+    dab[n_vec + i] = ob;
+}
+
 }  // namespace tc
 
 static long long max_items(long long R, int E, int nf) {
@@ -555,6 +605,74 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
                                                    dev_status, cs);
         if (st != R3_OK) return st;
     }
+    return launch_status();
+}
+
+// ---- input gradient of the expert networks (Update stage) ------------------------------------
+size_t tc_bwd_work_bytes(const r3_shape* s) {
+    const long long R = (long long)s->T * s->K;
+    const int nf_h = (s->F + tc::FEAT1 - 1) / tc::FEAT1;
+    return round_up((size_t)R * s->F * 2, 256) + round_up(2 * (size_t)R * s->F * 2, 256) +
+           list_bytes(R, s->E, nf_h) + list_bytes(R, s->E, feat_tiles_down(s));
+}
+
+r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, const void* pre_gate,
+                                       const void* pre_up, const int32_t* offsets,
+                                       const void* w_gate, const void* w_up, const void* w_down,
+                                       void* dxp, void* work, int32_t* dev_status,
+                                       cudaStream_t cs) {
+    using namespace tc;
+    const long long R = (long long)s->T * s->K;
+    if (R == 0) return R3_OK;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<2, false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(grouped_gemm_pair_kernel<3, false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+            return R3_ERR_CUDA;
+        attr_set = true;
+    }
+    const int pairs = resident_pairs(grouped_gemm_pair_kernel<2, false>);
+    if (pairs <= 0) return R3_ERR_CUDA;
+    const int nf_h = (s->F + FEAT1 - 1) / FEAT1, nf_x = feat_tiles_down(s);
+    char* w = static_cast<char*>(work);
+    void* dh = w;
+    w += round_up((size_t)R * s->F * 2, 256);
+    void* dab = w;
+    w += round_up(2 * (size_t)R * s->F * 2, 256);
+    int32_t* list_h = reinterpret_cast<int32_t*>(w);
+    int32_t* list_x = reinterpret_cast<int32_t*>(w + list_bytes(R, s->E, nf_h));
+    build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf_h, nf_x, list_h, list_x);
+
+    // dh = dout W_down   (weights transposed: contraction over d)
+    static TokenMapCache cache_do;
+    PairMaps m;
+    if (!make_map_3d(&m.a0, w_down, s->E, s->d, s->F, BK) ||
+        !token_maps(&cache_do, dout, (uint64_t)R, (uint64_t)s->d, &m))
+        return R3_ERR_CUDA;
+    m.a1 = m.a0;
+    m.g = m.b[0];
+    r3_status st = launch_pair<2, false>(m, pairs, list_h, nullptr, 0, dh, s->d, s->F, dev_status, cs);
+    if (st != R3_OK) return st;
+
+    // through the SwiGLU
+    const long long n_vec = R * s->F / 8;
+    swiglu_bwd_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, cs>>>(
+        static_cast<const uint4*>(dh), static_cast<const uint4*>(pre_gate),
+        static_cast<const uint4*>(pre_up), static_cast<uint4*>(dab), n_vec);
+
+    // dxp = da W_gate + db W_up   (weights transposed: contraction over F, both matrices)
+    PairMaps m2;
+    if (!make_map_3d(&m2.a0, w_gate, s->E, s->F, s->d, BK) ||
+        !make_map_3d(&m2.a1, w_up, s->E, s->F, s->d, BK))
+        return R3_ERR_CUDA;
+    for (int i = 0; i < BNT / 16; ++i)
+        if (!make_map_3d(&m2.b[i], dab, 2, (uint64_t)R, (uint64_t)s->F, 8u * (i + 1)))
+            return R3_ERR_CUDA;
+    m2.g = m2.b[0];
+    st = launch_pair<3, false>(m2, pairs, list_x, nullptr, 0, dxp, s->F, s->d, dev_status, cs);
+    if (st != R3_OK) return st;
     return launch_status();
 }
 

@@ -188,11 +188,20 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
            (1ull << 46) | (2ull << 61);
 }
+// The same for an MN-major bf16 operand (rows of the tile run along k, 64 consecutive elements
+// of the M / N dimension are one 128-byte row, as TMA writes a box of 64 elements x k rows with the
+// 128-byte swizzle): leading byte offset = distance between successive 64-element blocks of the
+// M / N dimension, stride byte offset 1024 = distance between successive groups of 8 k rows.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t block_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(block_bytes >> 4) << 16) |
+           ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
 // Instruction descriptor of tcgen05.mma kind::f16: D = f32, A = B = bf16, both K-major.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);
 }
+constexpr uint32_t kInstrDescAMajorMN = 1u << 15;      // A is MN-major (B stays K-major)
 
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem_addr, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"

@@ -36,7 +36,8 @@ EXPORTS = [
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
-    "r3_sequence_diff", "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
+    "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
+    "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
     "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
 ]
@@ -52,7 +53,9 @@ _P = ctypes.c_void_p
 _SP = ctypes.POINTER(Shape)
 lib.r3_status_string.restype = ctypes.c_char_p
 lib.r3_status_string.argtypes = [ctypes.c_int]
+lib.r3_grouped_swiglu_bwd_input.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, _P, _P]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
+           "r3_grouped_swiglu_bwd_workspace_bytes",
            "r3_replay_stack_workspace_bytes",
            "r3_replay_layer_workspace_bytes", "r3_replay_layer_host_workspace_bytes"):
     getattr(lib, _n).restype = ctypes.c_size_t
@@ -546,3 +549,18 @@ class PagePool:
 
     def release(self, table) -> None:
         _check(lib.r3_pagepool_release(self._h, self._arr(table), len(table)))
+
+
+def grouped_swiglu_bwd_input(s: Shape, dout, pre_gate, pre_up, offsets, w_gate, w_up, w_down,
+                             dxp=None, *, ws=None, dev_status=None, stream=None):
+    """Input gradient of the grouped SwiGLU experts: dout [R,d] -> dxp [R,d] (bf16)."""
+    dev = _dev(dout)
+    if dxp is None:
+        dxp = torch.empty((s.T * s.K, s.d), dtype=_act_dtype(s), device=dev)
+    if ws is None:
+        ws = workspace(lib.r3_grouped_swiglu_bwd_workspace_bytes(ctypes.byref(s)), dev)
+    _check(lib.r3_grouped_swiglu_bwd_input(ctypes.byref(s), _ptr(dout), _ptr(pre_gate),
+                                           _ptr(pre_up), _ptr(offsets), _ptr(w_gate), _ptr(w_up),
+                                           _ptr(w_down), _ptr(dxp), _ptr(ws), ws.numel(),
+                                           _ptr(dev_status), _stream(stream)))
+    return dxp
