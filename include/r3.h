@@ -297,6 +297,51 @@ r3_status r3_grouped_swiglu_bwd_input(const r3_shape* shape, const void* dout, c
                                       void* dxp, void* workspace, size_t ws_bytes,
                                       int32_t* dev_status, void* stream);
 
+/* r3_grouped_swiglu that also keeps what its backward needs: besides o it stores the
+ * pre-activations pre_gate = xp W_gate,e^T and pre_up = xp W_up,e^T ([R,F] each, rounded to bf16
+ * from the float32 accumulator; h is formed from the unrounded values, so o is bit-identical to
+ * r3_grouped_swiglu's).  bf16 only (R3_ERR_UNSUPPORTED for float32).  Same workspace. */
+r3_status r3_grouped_swiglu_train(const r3_shape* shape, const void* xp, const int32_t* offsets,
+                                  const void* w_gate, const void* w_up, const void* w_down,
+                                  void* o, void* pre_gate, void* pre_up, void* workspace,
+                                  size_t ws_bytes, int32_t* dev_status, void* stream);
+
+/* Gradient of the expert outputs under Eq. (replay_output), y_t = sum_j g[t,j] o[row(t,j)]:
+ *   dout[row_of_slot[t,j], :] = gates[t,j] * dy[t, :]
+ * dy [T,d], gates [T,K] float32, row_of_slot [T,K], dout [R,d] (every row written once; slots
+ * with row_of_slot < 0 are skipped).  No workspace. */
+r3_status r3_scale_rows(const r3_shape* shape, const void* dy, const float* gates,
+                        const int32_t* row_of_slot, void* dout, void* stream);
+
+/* Last step of the backward to the layer input.  The input x_t reaches the loss through its K
+ * experts and through the training logits s = x W_r^T that feed the replay gate (the recorded
+ * mask is a constant, Section 4.1):
+ *   dx[t,:]        = sum_j dxp[row_of_slot[t,j], :] + sum_j dlogits[t, e_j] * W_r[e_j, :]
+ *   dw_router[e,:] = sum over tokens t whose record holds e of dlogits[t,e] * x[t,:]
+ * (dlogits is zero outside the record, so these are the full products dlogits W_r and
+ * dlogits^T x.)  dxp [R,d], dlogits [T,E] float32, idx [T,K], x [T,d], w_router [E,d]
+ * (router_w_dtype), dx [T,d], dw_router [E,d] float32; row_of_slot / slot_of_row / offsets from
+ * r3_permute.  Sums run in float32 in slot order and in ascending token order: reproducible.  An
+ * expert that appears twice in a token's record contributes its term twice to dx, as the
+ * gradient of the gate does.  No workspace. */
+r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp, const int32_t* row_of_slot,
+                               const int32_t* slot_of_row, const int32_t* offsets,
+                               const float* dlogits, const void* idx, const void* x,
+                               const void* w_router, void* dx, float* dw_router, void* stream);
+
+/* r3_replay_layer followed by its backward to the layer input and to the router weight, one
+ * enqueue: y, dlogits as in r3_replay_layer, then dout = g dy, the expert input gradient
+ * (r3_grouped_swiglu_bwd_input) and r3_input_grad_finish.  dx [T,d], dw_router [E,d] float32.
+ * The gradients with respect to the expert weights are not computed.  bf16 only
+ * (R3_ERR_UNSUPPORTED for float32; r3_replay_layer_train_workspace_bytes returns 0 then).
+ * workspace: r3_replay_layer_train_workspace_bytes(shape), 256-byte aligned. */
+size_t r3_replay_layer_train_workspace_bytes(const r3_shape* shape);
+r3_status r3_replay_layer_train(const r3_shape* shape, const void* x, const void* w_router,
+                                const void* idx, const void* w_gate, const void* w_up,
+                                const void* w_down, const void* dy, void* y, float* dlogits,
+                                void* dx, float* dw_router, void* workspace, size_t ws_bytes,
+                                int32_t* dev_status, void* stream);
+
 /* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */
 
 /* Eq. (kl), the k3 estimate of KL(pi_train || pi_infer), and Eq. (etdf), the Extreme Token

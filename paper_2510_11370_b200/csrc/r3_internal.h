@@ -32,13 +32,15 @@ r3_status launch_build_tiles(const int32_t* offsets, int E, int BM, int32_t* til
 size_t tc_work_bytes(const r3_shape* shape);
 // phases: bit 0 = gate/up projections + SwiGLU (xp -> h), bit 1 = down projection (h -> o).
 enum { kPhaseUp = 1, kPhaseDown = 2 };
+// pre_gate / pre_up (optional, [R,F] bf16): the up phase also stores xp W_gate^T and xp W_up^T.
 // Token operand of the up projection: either the permuted rows `xp` [R, d], or (xp == nullptr) the
 // un-permuted activations `x` [T, d] gathered in place through `slot_of_row` [R].
 r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const void* x,
                                    const int32_t* slot_of_row, const int32_t* offsets,
                                    const void* w_gate, const void* w_up, const void* w_down,
                                    void* h, void* o, void* work, int32_t* dev_status, int phases,
-                                   cudaStream_t stream);
+                                   cudaStream_t stream, void* pre_gate = nullptr,
+                                   void* pre_up = nullptr);
 
 // Input gradient of the grouped SwiGLU experts on the tensor cores (bf16): dout [R,d] -> dxp [R,d]
 // with the forward's pre-activations pre_gate, pre_up [R,F].  `work`: tc_bwd_work_bytes().

@@ -101,7 +101,8 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
                            const void* idx, const void* w_gate, const void* w_up,
                            const void* w_down, const void* dy, const void* residual, void* y,
                            float* dlogits, float* gates_out, void* workspace,
-                           int32_t* dev_status, void* stream, cudaEvent_t dy_ready = nullptr) {
+                           int32_t* dev_status, void* stream, cudaEvent_t dy_ready = nullptr,
+                           void* pre_gate = nullptr, void* pre_up = nullptr) {
     const LayerWs w = carve(shape, workspace);
     float* gates = gates_out ? gates_out : w.gates;
     r3_status st;
@@ -127,9 +128,12 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
     if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
                          w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
         return st;
-    if ((st = r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, w.swiglu_ws,
-                                w.swiglu_bytes, dev_status, stream)) != R3_OK)
-        return st;
+    st = pre_gate ? r3_grouped_swiglu_train(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
+                                            pre_gate, pre_up, w.swiglu_ws, w.swiglu_bytes,
+                                            dev_status, stream)
+                  : r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
+                                      w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
+    if (st != R3_OK) return st;
     if (fused && side && cudaStreamWaitEvent(cs, side->join, 0) != cudaSuccess) return R3_ERR_CUDA;
     // dy is first needed here (host-buffer entry point: it may still be on its way)
     if (dy_ready && cudaStreamWaitEvent(cs, dy_ready, 0) != cudaSuccess) return R3_ERR_CUDA;
@@ -159,6 +163,73 @@ extern "C" r3_status r3_replay_layer(const r3_shape* shape, const void* x, const
         return R3_ERR_WORKSPACE;
     return r3::run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y, dlogits,
                          gates_out, workspace, dev_status, stream);
+}
+
+// ---- forward plus the backward to the layer input and the router weight ------------------------
+namespace r3 {
+struct TrainWs {
+    void* inner; size_t inner_bytes;
+    float* gates; void* pre_gate; void* pre_up; void* dxp; void* bwd_ws; size_t bwd_bytes;
+    size_t total;
+};
+static TrainWs carve_train(const r3_shape* s, void* base) {
+    TrainWs t;
+    size_t off = 0;
+    char* b = static_cast<char*>(base);
+    auto take = [&](size_t bytes) {
+        void* p = b ? b + off : nullptr;
+        off += round_up(bytes ? bytes : 1, 256);
+        return p;
+    };
+    const size_t R = (size_t)s->T * s->K;
+    t.inner_bytes = r3_replay_layer_workspace_bytes(s);
+    t.inner = take(t.inner_bytes);
+    t.gates = static_cast<float*>(take(R * 4));
+    t.pre_gate = take(R * s->F * act_bytes(s));
+    t.pre_up = take(R * s->F * act_bytes(s));
+    t.dxp = take(R * s->d * act_bytes(s));
+    t.bwd_bytes = r3_grouped_swiglu_bwd_workspace_bytes(s);
+    t.bwd_ws = take(t.bwd_bytes);
+    t.total = off;
+    return t;
+}
+}  // namespace r3
+
+extern "C" size_t r3_replay_layer_train_workspace_bytes(const r3_shape* shape) {
+    if (r3::check_shape(shape) != R3_OK || shape->act_dtype != R3_BF16) return 0;
+    return r3::carve_train(shape, nullptr).total;
+}
+
+extern "C" r3_status r3_replay_layer_train(const r3_shape* shape, const void* x,
+                                           const void* w_router, const void* idx,
+                                           const void* w_gate, const void* w_up,
+                                           const void* w_down, const void* dy, void* y,
+                                           float* dlogits, void* dx, float* dw_router,
+                                           void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                           void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->act_dtype != R3_BF16) return R3_ERR_UNSUPPORTED;
+    if (shape->T == 0) return R3_OK;
+    if (!x || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !y || !dlogits || !dx ||
+        !dw_router)
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_layer_train_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    const r3::TrainWs t = r3::carve_train(shape, workspace);
+    const r3::LayerWs w = r3::carve(shape, t.inner);
+    st = r3::run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y, dlogits,
+                       t.gates, t.inner, dev_status, stream, nullptr, t.pre_gate, t.pre_up);
+    if (st != R3_OK) return st;
+    // the expert outputs are no longer needed: their buffer takes dout = g dy
+    if ((st = r3_scale_rows(shape, dy, t.gates, w.row_of_slot, w.o, stream)) != R3_OK) return st;
+    if ((st = r3_grouped_swiglu_bwd_input(shape, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
+                                          w_up, w_down, t.dxp, t.bwd_ws, t.bwd_bytes, dev_status,
+                                          stream)) != R3_OK)
+        return st;
+    return r3_input_grad_finish(shape, t.dxp, w.row_of_slot, w.slot_of_row, w.offsets, dlogits,
+                                idx, x, w_router, dx, dw_router, stream);
 }
 
 // ---- a stack of L replayed MoE blocks with residual connections ------------------------------

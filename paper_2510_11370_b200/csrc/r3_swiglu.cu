@@ -180,14 +180,17 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const void* 
                              const int32_t* slot_of_row, const int32_t* offsets,
                              const void* w_gate, const void* w_up, const void* w_down, void* o,
                              void* workspace, size_t ws_bytes, int32_t* dev_status, int phases,
-                             void* stream) {
+                             void* stream, void* pre_gate = nullptr, void* pre_up = nullptr) {
     r3_status st = check_shape(shape);
     if (st != R3_OK) return st;
     if (shape->E > 1024) return R3_ERR_UNSUPPORTED;
     if (shape->T == 0) return R3_OK;
     const bool up = phases & kPhaseUp, down = phases & kPhaseDown;
     const bool gather = up && !xp;             // token rows read in place from x
-    if (gather && shape->act_dtype != R3_BF16) return R3_ERR_UNSUPPORTED;
+    if ((gather || pre_gate || pre_up) && shape->act_dtype != R3_BF16) return R3_ERR_UNSUPPORTED;
+    if ((pre_gate != nullptr) != (pre_up != nullptr) || !aligned(pre_gate, 16) ||
+        !aligned(pre_up, 16))
+        return R3_ERR_INVALID_ARG;
     if ((up && (!offsets || !w_gate || !w_up || (gather ? (!x || !slot_of_row) : !xp))) ||
         (down && (!w_down || !o)))
         return R3_ERR_INVALID_ARG;
@@ -202,8 +205,8 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const void* 
     void* h = workspace;
     int32_t* tiles = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + h_bytes(shape));
     if (shape->act_dtype == R3_BF16)
-        return launch_grouped_swiglu_tc(shape, xp, x, slot_of_row, offsets, w_gate, w_up, w_down, h, o, tiles,
-                                        dev_status, phases, cs);
+        return launch_grouped_swiglu_tc(shape, xp, x, slot_of_row, offsets, w_gate, w_up, w_down,
+                                        h, o, tiles, dev_status, phases, cs, pre_gate, pre_up);
     if (up) {
         st = launch_build_tiles(offsets, shape->E, SBM, tiles, cs);
         if (st != R3_OK) return st;
@@ -219,6 +222,17 @@ extern "C" r3_status r3_grouped_swiglu(const r3_shape* shape, const void* xp,
                                        void* stream) {
     return r3::run_experts(shape, xp, nullptr, nullptr, offsets, w_gate, w_up, w_down, o, workspace,
                            ws_bytes, dev_status, r3::kPhaseUp | r3::kPhaseDown, stream);
+}
+
+extern "C" r3_status r3_grouped_swiglu_train(const r3_shape* shape, const void* xp,
+                                             const int32_t* offsets, const void* w_gate,
+                                             const void* w_up, const void* w_down, void* o,
+                                             void* pre_gate, void* pre_up, void* workspace,
+                                             size_t ws_bytes, int32_t* dev_status, void* stream) {
+    if (shape && shape->T > 0 && (!pre_gate || !pre_up)) return R3_ERR_INVALID_ARG;
+    return r3::run_experts(shape, xp, nullptr, nullptr, offsets, w_gate, w_up, w_down, o, workspace,
+                           ws_bytes, dev_status, r3::kPhaseUp | r3::kPhaseDown, stream, pre_gate,
+                           pre_up);
 }
 
 extern "C" r3_status r3_grouped_swiglu_gather(const r3_shape* shape, const void* x,

@@ -56,7 +56,7 @@ constexpr int B_BYTES = (BNT / 2) * BK * 2;      // up to 16 KB of tokens per CT
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_WARPS = 4;
 constexpr int THREADS = (2 + EPI_WARPS) * 32;
-constexpr int EPI_BYTES = 20 * 1024;             // transpose / exchange buffers of the epilogue
+constexpr int EPI_BYTES = 28 * 1024;             // transpose / exchange buffers of the epilogue
 constexpr int BAR_BYTES = 256;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + 1024;  // + alignment
 constexpr int FEAT0 = BMF;         // h features per item in MODE 0 (64 per CTA, gate + up rows)
@@ -142,7 +142,8 @@ template <int MODE, bool GATHER>
 __global__ void __launch_bounds__(THREADS, 1)
 grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* __restrict__ list,
                          const int32_t* __restrict__ slot_of_row, int K,
-                         __nv_bfloat16* __restrict__ out, int Kdim, int Nout,
+                         __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ pre_gate,
+                         __nv_bfloat16* __restrict__ pre_up, int Kdim, int Nout,
                          int32_t* dev_status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -353,6 +354,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
                 const bool gate = q < 2;
                 float* xpair = reinterpret_cast<float*>(epi_ptr + p * 8192);      // 2 x [2][16][32]
                 __nv_bfloat16* hb = reinterpret_cast<__nv_bfloat16*>(epi_ptr + 16384 + q * 1024);
+                // training: the pre-activations are kept for the backward pass
+                __nv_bfloat16* gb = reinterpret_cast<__nv_bfloat16*>(epi_ptr + 20480 + q * 2048);
+                __nv_bfloat16* ub = gb + 512;
+                const bool keep = pre_gate != nullptr;
                 const int feat = f * FEAT0 + (int)rank * (BMF / 2) + p * 32 + (lane & 3) * 8;
                 const int own = gate ? 0 : 16;        // first of the 16 tokens this warp finishes
 #pragma unroll 1
@@ -377,15 +382,28 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
                         const float g = gate ? v[i] : other;
                         const float u = gate ? other : v[16 + i];
                         hb[i * 32 + lane] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+                        if (keep) {
+                            gb[i * 32 + lane] = __float2bfloat16_rn(g);
+                            ub[i * 32 + lane] = __float2bfloat16_rn(u);
+                        }
                     }
                     __syncwarp();
 #pragma unroll
                     for (int rr = 0; rr < 2; ++rr) {
                         const int tl = (lane >> 2) + 8 * rr;
-                        const uint4 val = *reinterpret_cast<const uint4*>(hb + tl * 32 + (lane & 3) * 8);
                         const int tok = c + own + tl;
-                        if (alive && tok < valid && feat + 8 <= Nout)
-                            *reinterpret_cast<uint4*>(out + (size_t)(row0 + tok) * Nout + feat) = val;
+                        if (alive && tok < valid && feat + 8 <= Nout) {
+                            const size_t at = (size_t)(row0 + tok) * Nout + feat;
+                            const int in_tile = tl * 32 + (lane & 3) * 8;
+                            *reinterpret_cast<uint4*>(out + at) =
+                                *reinterpret_cast<const uint4*>(hb + in_tile);
+                            if (keep) {
+                                *reinterpret_cast<uint4*>(pre_gate + at) =
+                                    *reinterpret_cast<const uint4*>(gb + in_tile);
+                                *reinterpret_cast<uint4*>(pre_up + at) =
+                                    *reinterpret_cast<const uint4*>(ub + in_tile);
+                            }
+                        }
                     }
                     __syncwarp();
                 }
@@ -488,7 +506,8 @@ static int resident_pairs(Kern kern) {
 template <int MODE, bool GATHER>
 static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* list,
                              const int32_t* slot_of_row, int K, void* out, int Kdim, int Nout,
-                             int32_t* dev_status, cudaStream_t cs) {
+                             int32_t* dev_status, cudaStream_t cs, void* pre_gate = nullptr,
+                             void* pre_up = nullptr) {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -502,7 +521,8 @@ static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* lis
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<MODE, GATHER>, maps, list, slot_of_row, K,
-                              static_cast<__nv_bfloat16*>(out), Kdim, Nout,
+                              static_cast<__nv_bfloat16*>(out), static_cast<__nv_bfloat16*>(pre_gate),
+                              static_cast<__nv_bfloat16*>(pre_up), Kdim, Nout,
                               dev_status) == cudaSuccess ? R3_OK : R3_ERR_CUDA;
 }
 
@@ -553,7 +573,7 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
                                    const int32_t* slot_of_row, const int32_t* offsets,
                                    const void* w_gate, const void* w_up, const void* w_down,
                                    void* h, void* o, void* work, int32_t* dev_status, int phases,
-                                   cudaStream_t cs) {
+                                   cudaStream_t cs, void* pre_gate, void* pre_up) {
     using namespace tc;
     const long long R = (long long)s->T * s->K;
     if (R == 0) return R3_OK;
@@ -585,12 +605,13 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
         if (xp) {
             if (!token_maps(&cache_xp, xp, (uint64_t)R, (uint64_t)s->d, &m)) return R3_ERR_CUDA;
             m.g = m.b[0];
-            st = launch_pair<0, false>(m, pairs, list0, nullptr, 0, h, s->d, s->F, dev_status, cs);
+            st = launch_pair<0, false>(m, pairs, list0, nullptr, 0, h, s->d, s->F, dev_status, cs,
+                                       pre_gate, pre_up);
         } else {
             if (!make_map_2d(&m.g, x, (uint64_t)s->T, (uint64_t)s->d, 1)) return R3_ERR_CUDA;
             for (int i = 0; i < BNT / 16; ++i) m.b[i] = m.g;
             st = launch_pair<0, true>(m, pairs, list0, slot_of_row, s->K, h, s->d, s->F,
-                                      dev_status, cs);
+                                      dev_status, cs, pre_gate, pre_up);
         }
         if (st != R3_OK) return st;
     }

@@ -37,6 +37,8 @@ EXPORTS = [
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
     "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
+    "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
+    "r3_replay_layer_train_workspace_bytes", "r3_replay_layer_train",
     "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
     "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
@@ -54,8 +56,12 @@ _SP = ctypes.POINTER(Shape)
 lib.r3_status_string.restype = ctypes.c_char_p
 lib.r3_status_string.argtypes = [ctypes.c_int]
 lib.r3_grouped_swiglu_bwd_input.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, _P, _P]
+lib.r3_grouped_swiglu_train.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, _P, _P]
+lib.r3_scale_rows.argtypes = [_SP] + [_P] * 5
+lib.r3_input_grad_finish.argtypes = [_SP] + [_P] * 11
+lib.r3_replay_layer_train.argtypes = [_SP] + [_P] * 12 + [ctypes.c_size_t, _P, _P]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
-           "r3_grouped_swiglu_bwd_workspace_bytes",
+           "r3_grouped_swiglu_bwd_workspace_bytes", "r3_replay_layer_train_workspace_bytes",
            "r3_replay_stack_workspace_bytes",
            "r3_replay_layer_workspace_bytes", "r3_replay_layer_host_workspace_bytes"):
     getattr(lib, _n).restype = ctypes.c_size_t
@@ -549,6 +555,62 @@ class PagePool:
 
     def release(self, table) -> None:
         _check(lib.r3_pagepool_release(self._h, self._arr(table), len(table)))
+
+
+def grouped_swiglu_train(s: Shape, xp, offsets, w_gate, w_up, w_down, *, ws=None, dev_status=None,
+                         stream=None):
+    """Grouped experts that also return the pre-activations: (o [R,d], pre_gate, pre_up [R,F])."""
+    dev = _dev(xp)
+    R = s.T * s.K
+    o = torch.empty((R, s.d), dtype=_act_dtype(s), device=dev)
+    pre_gate = torch.empty((R, s.F), dtype=_act_dtype(s), device=dev)
+    pre_up = torch.empty((R, s.F), dtype=_act_dtype(s), device=dev)
+    if ws is None:
+        ws = workspace(lib.r3_grouped_swiglu_workspace_bytes(ctypes.byref(s)), dev)
+    _check(lib.r3_grouped_swiglu_train(ctypes.byref(s), _ptr(xp), _ptr(offsets), _ptr(w_gate),
+                                       _ptr(w_up), _ptr(w_down), _ptr(o), _ptr(pre_gate),
+                                       _ptr(pre_up), _ptr(ws), ws.numel(), _ptr(dev_status),
+                                       _stream(stream)))
+    return o, pre_gate, pre_up
+
+
+def scale_rows(s: Shape, dy, gates, row_of_slot, dout=None, *, stream=None):
+    """dout[row_of_slot[t,j]] = gates[t,j] * dy[t]."""
+    if dout is None:
+        dout = torch.empty((s.T * s.K, s.d), dtype=_act_dtype(s), device=_dev(dy))
+    _check(lib.r3_scale_rows(ctypes.byref(s), _ptr(dy), _ptr(gates), _ptr(row_of_slot),
+                             _ptr(dout), _stream(stream)))
+    return dout
+
+
+def input_grad_finish(s: Shape, dxp, row_of_slot, slot_of_row, offsets, dlogits, idx, x, w_router,
+                      *, stream=None):
+    """(dx [T,d], dw_router [E,d] float32) from the expert input gradient and dlogits."""
+    dev = _dev(dxp)
+    dx = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    dw_r = torch.empty((s.E, s.d), dtype=torch.float32, device=dev)
+    _check(lib.r3_input_grad_finish(ctypes.byref(s), _ptr(dxp), _ptr(row_of_slot),
+                                    _ptr(slot_of_row), _ptr(offsets), _ptr(dlogits), _ptr(idx),
+                                    _ptr(x), _ptr(w_router), _ptr(dx), _ptr(dw_r),
+                                    _stream(stream)))
+    return dx, dw_r
+
+
+def replay_layer_train(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, ws=None,
+                       dev_status=None, stream=None):
+    """Forward and backward-to-input of one replayed layer: (y, dlogits, dx, dw_router)."""
+    dev = _dev(x)
+    y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
+    dx = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    dw_r = torch.empty((s.E, s.d), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(lib.r3_replay_layer_train_workspace_bytes(ctypes.byref(s)), dev)
+    _check(lib.r3_replay_layer_train(ctypes.byref(s), _ptr(x), _ptr(w_router), _ptr(idx),
+                                     _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(dy), _ptr(y),
+                                     _ptr(dlogits), _ptr(dx), _ptr(dw_r), _ptr(ws), ws.numel(),
+                                     _ptr(dev_status), _stream(stream)))
+    return y, dlogits, dx, dw_r
 
 
 def grouped_swiglu_bwd_input(s: Shape, dout, pre_gate, pre_up, offsets, w_gate, w_up, w_down,
