@@ -345,3 +345,39 @@ def layer_bwd_input(x, w_r, idx_infer, w_gate, w_up, w_down, dy):
     dx_r = f["ds"] @ w_r
     return dict(dx=dx_e + dx_r, dw_r=f["ds"].T @ x, ds=f["ds"], dx_expert=dx_e, dx_router=dx_r,
                 y=f["y"], g=f["g"])
+
+
+# ----------------------------------------------------------------------------------------------
+# Update-stage backward to the expert weights (Section 4.1, purpose (b): with the mask replayed,
+# the experts that receive a gradient are exactly those the rollout activated)
+# ----------------------------------------------------------------------------------------------
+def swiglu_expert_bwd_weights(x, do, w_gate_i, w_up_i, w_down_i):
+    """(dW_gate_i [F,d], dW_up_i [F,d], dW_down_i [d,F]) for o = E_i(x) given dL/do over the n
+    tokens routed to expert i:  a = W_gate x, b = W_up x, h = silu(a) b, o = W_down h, so
+        dW_down = do^T h,  dh = do W_down,  da = dh b silu'(a),  db = dh silu(a),
+        dW_gate = da^T x,  dW_up = db^T x."""
+    x, do = _f64(x), _f64(do)
+    wg, wu, wd = _f64(w_gate_i), _f64(w_up_i), _f64(w_down_i)
+    a, b = x @ wg.T, x @ wu.T
+    h = silu(a) * b
+    dh = do @ wd
+    da = dh * b * dsilu(a)
+    db = dh * silu(a)
+    return da.T @ x, db.T @ x, do.T @ h
+
+
+def layer_bwd_weights(x, w_r, idx_infer, w_gate, w_up, w_down, dy, experts=None):
+    """Expert-weight gradients of L = <dy, y_replay(x)> with the recorded mask held constant.
+    Expert i sees the tokens whose record holds i, each with dL/do = g_{t,j} dy_t; an expert that
+    no record names gets a zero gradient.  `experts` limits the work to those expert ids.
+    Returns {i: (dW_gate_i, dW_up_i, dW_down_i)}."""
+    x, dy, w_r = _f64(x), _f64(dy), _f64(w_r)
+    idx = np.asarray(idx_infer, dtype=np.int64)
+    E = w_r.shape[0]
+    g = replay_gate(router_logits(x, w_r), idx)
+    out = {}
+    for i in (range(E) if experts is None else experts):
+        tt, jj = np.nonzero(idx == i)
+        do = g[tt, jj][:, None] * dy[tt]
+        out[int(i)] = swiglu_expert_bwd_weights(x[tt], do, w_gate[i], w_up[i], w_down[i])
+    return out

@@ -463,3 +463,58 @@ def test_input_gradient_special_cases():
     # zero upstream gradient -> zero gradients
     z = O.layer_bwd_input(x, w_r, idx, wg, wu, wd, np.zeros_like(dy))
     assert np.all(z["dx"] == 0) and np.all(z["dw_r"] == 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# Update-stage backward to the expert weights
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("which", [0, 1, 2])
+def test_expert_weight_gradients_match_central_differences(which):
+    x, w_r, idx, wg, wu, wd, dy = _tiny_layer(10 + which, T=6, d=4, E=3, K=2, F=3)
+    got = O.layer_bwd_weights(x, w_r, idx, wg, wu, wd, dy)
+    ws = [wg, wu, wd]
+    target = ws[which]
+    h = 1e-6
+    num = np.zeros_like(target)
+    for pos in np.ndindex(*target.shape):
+        keep = target[pos]
+        target[pos] = keep + h
+        up = _loss(x, w_r, idx, *ws, dy)
+        target[pos] = keep - h
+        dn = _loss(x, w_r, idx, *ws, dy)
+        target[pos] = keep
+        num[pos] = (up - dn) / (2 * h)
+    mine = np.stack([got[e][which] for e in range(wg.shape[0])])
+    assert np.abs(mine - num).max() / np.abs(num).max() < 1e-7
+
+
+def test_expert_weight_gradients_autograd_second_opinion_and_special_cases():
+    x, w_r, idx, wg, wu, wd, dy = _tiny_layer(20, T=7, d=5, E=4, K=2, F=3)
+    idx[idx == 3] = 0                      # expert 3 is never recorded ...
+    idx[:, 1] = np.where(idx[:, 0] == idx[:, 1], 1 + idx[:, 0] % 2, idx[:, 1])
+    idx[idx == 3] = 2
+    assert not np.any(idx == 3) and np.all(idx[:, 0] != idx[:, 1])
+    got = O.layer_bwd_weights(x, w_r, idx, wg, wu, wd, dy)
+    for m in got[3]:
+        assert np.all(m == 0)              # ... so its weights get no gradient
+    # torch autograd through the dense printed form (gate = masked softmax, constant mask)
+    tw = [torch.tensor(w, requires_grad=True) for w in (wg, wu, wd)]
+    xt = torch.tensor(x)
+    s = xt @ torch.tensor(w_r).T
+    mask = torch.zeros_like(s)
+    mask.scatter_(1, torch.tensor(idx), 1.0)
+    e = mask * torch.exp(s)
+    gate = e / e.sum(dim=1, keepdim=True)
+    y = torch.zeros_like(xt)
+    for i in range(wg.shape[0]):
+        o = (torch.nn.functional.silu(xt @ tw[0][i].T) * (xt @ tw[1][i].T)) @ tw[2][i].T
+        y = y + gate[:, i:i + 1] * o
+    (torch.tensor(dy) * y).sum().backward()
+    for i in range(wg.shape[0]):
+        for which in range(3):
+            assert np.allclose(got[i][which], tw[which].grad[i].numpy(), atol=1e-12)
+    # restricting the experts changes nothing for those computed; zero dy gives zero
+    part = O.layer_bwd_weights(x, w_r, idx, wg, wu, wd, dy, experts=[1])
+    assert list(part) == [1] and all(np.array_equal(a, b) for a, b in zip(part[1], got[1]))
+    z = O.layer_bwd_weights(x, w_r, idx, wg, wu, wd, np.zeros_like(dy))
+    assert all(np.all(m == 0) for i in z for m in z[i])
