@@ -297,6 +297,20 @@ r3_status r3_grouped_swiglu_bwd_input(const r3_shape* shape, const void* dout, c
                                       void* dxp, void* workspace, size_t ws_bytes,
                                       int32_t* dev_status, void* stream);
 
+/* The whole backward of the grouped experts: dxp as r3_grouped_swiglu_bwd_input, and the
+ * gradients of the expert weights, for each expert e over its rows [offsets[e], offsets[e+1]):
+ *   dW_down[e] = dout_e^T h_e     dW_gate[e] = da_e^T xp_e     dW_up[e] = db_e^T xp_e
+ * xp [R,d] are the permuted rows the forward saw.  dw_gate, dw_up [E,F,d] and dw_down [E,d,F] are
+ * float32 and are OVERWRITTEN (an expert without rows gets zeros); products of bf16 operands
+ * (h, da, db rounded to bf16 once each) accumulate in float32 in a fixed order.  bf16 only.
+ * workspace: r3_grouped_swiglu_bwd_workspace_bytes(shape). */
+r3_status r3_grouped_swiglu_bwd(const r3_shape* shape, const void* xp, const void* dout,
+                                const void* pre_gate, const void* pre_up, const int32_t* offsets,
+                                const void* w_gate, const void* w_up, const void* w_down,
+                                void* dxp, float* dw_gate, float* dw_up, float* dw_down,
+                                void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                void* stream);
+
 /* r3_grouped_swiglu that also keeps what its backward needs: besides o it stores the
  * pre-activations pre_gate = xp W_gate,e^T and pre_up = xp W_up,e^T ([R,F] each, rounded to bf16
  * from the float32 accumulator; h is formed from the unrounded values, so o is bit-identical to
@@ -331,15 +345,17 @@ r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp, const int
 
 /* r3_replay_layer followed by its backward to the layer input and to the router weight, one
  * enqueue: y, dlogits as in r3_replay_layer, then dout = g dy, the expert input gradient
- * (r3_grouped_swiglu_bwd_input) and r3_input_grad_finish.  dx [T,d], dw_router [E,d] float32.
- * The gradients with respect to the expert weights are not computed.  bf16 only
+ * (r3_grouped_swiglu_bwd) and r3_input_grad_finish.  dx [T,d], dw_router [E,d] float32.
+ * dw_gate, dw_up [E,F,d], dw_down [E,d,F] float32 receive the expert-weight gradients
+ * (overwritten); pass all three null to skip them.  bf16 only
  * (R3_ERR_UNSUPPORTED for float32; r3_replay_layer_train_workspace_bytes returns 0 then).
  * workspace: r3_replay_layer_train_workspace_bytes(shape), 256-byte aligned. */
 size_t r3_replay_layer_train_workspace_bytes(const r3_shape* shape);
 r3_status r3_replay_layer_train(const r3_shape* shape, const void* x, const void* w_router,
                                 const void* idx, const void* w_gate, const void* w_up,
                                 const void* w_down, const void* dy, void* y, float* dlogits,
-                                void* dx, float* dw_router, void* workspace, size_t ws_bytes,
+                                void* dx, float* dw_router, float* dw_gate, float* dw_up,
+                                float* dw_down, void* workspace, size_t ws_bytes,
                                 int32_t* dev_status, void* stream);
 
 /* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */

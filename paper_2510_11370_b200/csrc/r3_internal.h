@@ -44,12 +44,20 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* shape, const void* xp, const 
 
 // Input gradient of the grouped SwiGLU experts on the tensor cores (bf16): dout [R,d] -> dxp [R,d]
 // with the forward's pre-activations pre_gate, pre_up [R,F].  `work`: tc_bwd_work_bytes().
+// With dw_gate non-null (then xp, dw_up, dw_down too) the expert-weight gradients follow.
 size_t tc_bwd_work_bytes(const r3_shape* shape);
 r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* shape, const void* dout, const void* pre_gate,
                                        const void* pre_up, const int32_t* offsets,
                                        const void* w_gate, const void* w_up, const void* w_down,
                                        void* dxp, void* work, int32_t* dev_status,
-                                       cudaStream_t stream);
+                                       cudaStream_t stream, const void* xp = nullptr,
+                                       float* dw_gate = nullptr, float* dw_up = nullptr,
+                                       float* dw_down = nullptr);
+// dW_down[e] = dout_e^T h_e, dW_gate[e] = da_e^T xp_e, dW_up[e] = db_e^T xp_e (float32 [E,d,F],
+// [E,F,d], [E,F,d]); all operands bf16, [R, .] row-major.
+r3_status launch_wgrad_tc(const r3_shape* shape, const void* xp, const void* dout, const void* h,
+                          const void* da, const void* db, const int32_t* offsets, float* dw_gate,
+                          float* dw_up, float* dw_down, int32_t* dev_status, cudaStream_t stream);
 
 // Router logits + top-K on the tensor cores (bf16 activations, E a multiple of 16 up to 256,
 // K <= 16).  float32 router weights need router_tc_workspace_bytes() of scratch for their three

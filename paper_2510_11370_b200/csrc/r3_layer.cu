@@ -205,6 +205,7 @@ extern "C" r3_status r3_replay_layer_train(const r3_shape* shape, const void* x,
                                            const void* w_gate, const void* w_up,
                                            const void* w_down, const void* dy, void* y,
                                            float* dlogits, void* dx, float* dw_router,
+                                           float* dw_gate, float* dw_up, float* dw_down,
                                            void* workspace, size_t ws_bytes, int32_t* dev_status,
                                            void* stream) {
     r3_status st = r3::check_shape(shape);
@@ -214,6 +215,8 @@ extern "C" r3_status r3_replay_layer_train(const r3_shape* shape, const void* x,
     if (!x || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !y || !dlogits || !dx ||
         !dw_router)
         return R3_ERR_INVALID_ARG;
+    const bool weights = dw_gate || dw_up || dw_down;
+    if (weights && (!dw_gate || !dw_up || !dw_down)) return R3_ERR_INVALID_ARG;
     if (!workspace || !r3::aligned(workspace, 256) ||
         ws_bytes < r3_replay_layer_train_workspace_bytes(shape))
         return R3_ERR_WORKSPACE;
@@ -224,10 +227,13 @@ extern "C" r3_status r3_replay_layer_train(const r3_shape* shape, const void* x,
     if (st != R3_OK) return st;
     // the expert outputs are no longer needed: their buffer takes dout = g dy
     if ((st = r3_scale_rows(shape, dy, t.gates, w.row_of_slot, w.o, stream)) != R3_OK) return st;
-    if ((st = r3_grouped_swiglu_bwd_input(shape, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
-                                          w_up, w_down, t.dxp, t.bwd_ws, t.bwd_bytes, dev_status,
-                                          stream)) != R3_OK)
-        return st;
+    st = weights ? r3_grouped_swiglu_bwd(shape, w.xp, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
+                                         w_up, w_down, t.dxp, dw_gate, dw_up, dw_down, t.bwd_ws,
+                                         t.bwd_bytes, dev_status, stream)
+                 : r3_grouped_swiglu_bwd_input(shape, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
+                                               w_up, w_down, t.dxp, t.bwd_ws, t.bwd_bytes,
+                                               dev_status, stream);
+    if (st != R3_OK) return st;
     return r3_input_grad_finish(shape, t.dxp, w.row_of_slot, w.slot_of_row, w.offsets, dlogits,
                                 idx, x, w_router, dx, dw_router, stream);
 }

@@ -288,3 +288,31 @@ extern "C" r3_status r3_grouped_swiglu_bwd_input(const r3_shape* shape, const vo
                                             w_down, dxp, workspace, dev_status,
                                             static_cast<cudaStream_t>(stream));
 }
+
+extern "C" r3_status r3_grouped_swiglu_bwd(const r3_shape* shape, const void* xp, const void* dout,
+                                           const void* pre_gate, const void* pre_up,
+                                           const int32_t* offsets, const void* w_gate,
+                                           const void* w_up, const void* w_down, void* dxp,
+                                           float* dw_gate, float* dw_up, float* dw_down,
+                                           void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                           void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->act_dtype != R3_BF16 || shape->E > 1024) return R3_ERR_UNSUPPORTED;
+    if (shape->T == 0) return R3_OK;
+    if (!xp || !dout || !pre_gate || !pre_up || !offsets || !w_gate || !w_up || !w_down || !dxp ||
+        !dw_gate || !dw_up || !dw_down)
+        return R3_ERR_INVALID_ARG;
+    if (!r3::aligned(xp, 16) || !r3::aligned(dout, 16) || !r3::aligned(pre_gate, 16) ||
+        !r3::aligned(pre_up, 16) || !r3::aligned(dxp, 16) || !r3::aligned(w_gate, 16) ||
+        !r3::aligned(w_up, 16) || !r3::aligned(w_down, 16) || !r3::aligned(dw_gate, 16) ||
+        !r3::aligned(dw_up, 16) || !r3::aligned(dw_down, 16))
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_grouped_swiglu_bwd_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    return r3::launch_grouped_swiglu_bwd_tc(shape, dout, pre_gate, pre_up, offsets, w_gate, w_up,
+                                            w_down, dxp, workspace, dev_status,
+                                            static_cast<cudaStream_t>(stream), xp, dw_gate, dw_up,
+                                            dw_down);
+}

@@ -527,14 +527,17 @@ static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* lis
 }
 
 // Backward of h = silu(a) * b:  da = dh * b * silu'(a),  db = dh * silu(a), written as planes 0
-// and 1 of dab [2, R, F].  16-byte vectors; F is a multiple of 8.
+// and 1 of dab [2, R, F].  16-byte vectors; F is a multiple of 8.  With `h` non-null the forward's
+// h = silu(a) * b is formed again (the weight gradient of the down projection needs it).
 __global__ void __launch_bounds__(256)
 swiglu_bwd_kernel(const uint4* __restrict__ dh, const uint4* __restrict__ a,
-                  const uint4* __restrict__ b, uint4* __restrict__ dab, long long n_vec) {
+                  const uint4* __restrict__ b, uint4* __restrict__ dab, uint4* __restrict__ h,
+                  long long n_vec) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_vec) return;
     const uint4 vd = dh[i], va = a[i], vb = b[i];
-    uint4 oa, ob;
+    uint4 oa, ob, oh;
+    __nv_bfloat162* qh = reinterpret_cast<__nv_bfloat162*>(&oh);
     const __nv_bfloat162* pd = reinterpret_cast<const __nv_bfloat162*>(&vd);
     const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&va);
     const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&vb);
@@ -548,9 +551,11 @@ swiglu_bwd_kernel(const uint4* __restrict__ dh, const uint4* __restrict__ a,
         qa[k] = __floats2bfloat162_rn(fd.x * fb.x * s0 * (1.f + fa.x * (1.f - s0)),
                                       fd.y * fb.y * s1 * (1.f + fa.y * (1.f - s1)));
         qb[k] = __floats2bfloat162_rn(fd.x * fa.x * s0, fd.y * fa.y * s1);
+        qh[k] = __floats2bfloat162_rn(fa.x * s0 * fb.x, fa.y * s1 * fb.y);
     }
     dab[i] = oa;
     dab[n_vec + i] = ob;
+    if (h) h[i] = oh;
 }
 
 }  // namespace tc
@@ -633,7 +638,7 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
 size_t tc_bwd_work_bytes(const r3_shape* s) {
     const long long R = (long long)s->T * s->K;
     const int nf_h = (s->F + tc::FEAT1 - 1) / tc::FEAT1;
-    return round_up((size_t)R * s->F * 2, 256) + round_up(2 * (size_t)R * s->F * 2, 256) +
+    return 2 * round_up((size_t)R * s->F * 2, 256) + round_up(2 * (size_t)R * s->F * 2, 256) +
            list_bytes(R, s->E, nf_h) + list_bytes(R, s->E, feat_tiles_down(s));
 }
 
@@ -641,7 +646,8 @@ r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, cons
                                        const void* pre_up, const int32_t* offsets,
                                        const void* w_gate, const void* w_up, const void* w_down,
                                        void* dxp, void* work, int32_t* dev_status,
-                                       cudaStream_t cs) {
+                                       cudaStream_t cs, const void* xp, float* dw_gate,
+                                       float* dw_up, float* dw_down) {
     using namespace tc;
     const long long R = (long long)s->T * s->K;
     if (R == 0) return R3_OK;
@@ -662,6 +668,9 @@ r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, cons
     w += round_up((size_t)R * s->F * 2, 256);
     void* dab = w;
     w += round_up(2 * (size_t)R * s->F * 2, 256);
+    void* h = w;
+    w += round_up((size_t)R * s->F * 2, 256);
+    const bool weights = dw_gate != nullptr;
     int32_t* list_h = reinterpret_cast<int32_t*>(w);
     int32_t* list_x = reinterpret_cast<int32_t*>(w + list_bytes(R, s->E, nf_h));
     build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf_h, nf_x, list_h, list_x);
@@ -681,7 +690,8 @@ r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, cons
     const long long n_vec = R * s->F / 8;
     swiglu_bwd_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, cs>>>(
         static_cast<const uint4*>(dh), static_cast<const uint4*>(pre_gate),
-        static_cast<const uint4*>(pre_up), static_cast<uint4*>(dab), n_vec);
+        static_cast<const uint4*>(pre_up), static_cast<uint4*>(dab),
+        weights ? static_cast<uint4*>(h) : nullptr, n_vec);
 
     // dxp = da W_gate + db W_up   (weights transposed: contraction over F, both matrices)
     PairMaps m2;
@@ -694,6 +704,11 @@ r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, cons
     m2.g = m2.b[0];
     st = launch_pair<3, false>(m2, pairs, list_x, nullptr, 0, dxp, s->F, s->d, dev_status, cs);
     if (st != R3_OK) return st;
+    if (weights) {
+        const char* db = static_cast<const char*>(dab) + (size_t)R * s->F * 2;
+        return launch_wgrad_tc(s, xp, dout, h, dab, db, offsets, dw_gate, dw_up, dw_down,
+                               dev_status, cs);
+    }
     return launch_status();
 }
 

@@ -1,0 +1,308 @@
+// Expert-weight gradients of the grouped SwiGLU experts on the tensor cores (bf16 operands, float32
+// result).  For expert e with grouped rows [offsets[e], offsets[e+1]):
+//   dW_down[e] [d,F] = dout_e^T h_e      dW_gate[e] [F,d] = da_e^T xp_e      dW_up[e] [F,d] = db_e^T xp_e
+// Every product contracts over the expert's token rows, so both operands are read "MN-major": a
+// TMA box of 64 consecutive columns x 64 token rows lands as 64 swizzled 128-byte rows, and the
+// tcgen05 descriptors walk the rows as the k dimension.  One CTA per SM (cta_group::1), tiles of
+// 128 x 256 outputs, float32 accumulators in tensor memory (two stages, so a tile's epilogue runs
+// under the next tile's MMAs), items (problem, expert, n tile, m tile) dealt round-robin.
+//
+// The token count of an expert is ragged.  Rows of the last 64-row block that belong to the next
+// expert must not contribute: whole 16-row MMA steps beyond the expert's end are not issued, and
+// inside the last partial step the surplus rows are overwritten with zeros in shared memory (both
+// operands) before the MMA reads them.
+#include "r3_tc.cuh"
+#include "r3_internal.h"
+
+namespace r3 {
+namespace wg {
+
+using namespace tc;
+
+constexpr int WM = 128;                 // output rows per tile (MMA M)
+constexpr int WN = 256;                 // output columns per tile (MMA N)
+constexpr int WK = 64;                  // token rows per pipeline stage
+constexpr int UK = 16;                  // token rows per MMA
+constexpr int STAGES = 4;
+constexpr int ACC_STAGES = 2;
+constexpr int BOX_BYTES = 64 * WK * 2;  // one TMA box: 64 columns x 64 rows of bf16
+constexpr int A_BYTES = (WM / 64) * BOX_BYTES;
+constexpr int B_BYTES = (WN / 64) * BOX_BYTES;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 48 KB
+constexpr int EPI_WARPS = 4;
+constexpr int EPI_BYTES = EPI_WARPS * 32 * 32 * 4;      // a 32 x 32 float block per warp
+constexpr int THREADS = 32 * (2 + EPI_WARPS);
+constexpr int TMEM_COLS = ACC_STAGES * WN;              // 512
+constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 256;
+constexpr uint32_t kInstrDescBothMN = (1u << 15) | (1u << 16);
+constexpr int MAX_PROBLEMS = 3;
+
+struct Problem {
+    CUtensorMap a;      // [R, M] bf16, box 64 x 64
+    CUtensorMap b;      // [R, N] bf16, box 64 x 64
+    float* out;         // [E, M, N]
+    int M, N;
+    int mt, nt;         // tiles along M and N
+    int item0;          // first item of this problem
+};
+struct Params {
+    Problem p[MAX_PROBLEMS];
+    int n_problems;
+    int total_items;
+};
+
+struct Item {
+    int q, e, m0, n0;
+};
+__device__ __forceinline__ Item decode(const Params& P, int i) {
+    int q = 0;
+#pragma unroll
+    for (int k = 1; k < MAX_PROBLEMS; ++k)
+        if (k < P.n_problems && i >= P.p[k].item0) q = k;
+    const int local = i - P.p[q].item0;
+    const int per_e = P.p[q].mt * P.p[q].nt;
+    const int e = local / per_e, rem = local - e * per_e;
+    const int n = rem / P.p[q].mt, m = rem - n * P.p[q].mt;
+    return Item{q, e, m * WM, n * WN};
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offsets,
+             int32_t* dev_status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t* epi_ptr = base_ptr + STAGES * STAGE_BYTES;
+    const uint32_t bar0 = base + STAGES * STAGE_BYTES + EPI_BYTES;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + ACC_STAGES + a); };
+    uint8_t* misc = epi_ptr + EPI_BYTES + 128;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int w_begin = blockIdx.x, w_step = gridDim.x, w_end = P.total_items;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), EPI_WARPS);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer -------------------------------------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int w = w_begin; ok && w < w_end; w += w_step) {
+                const Item it = decode(P, w);
+                const CUtensorMap* amap = &P.p[it.q].a;
+                const CUtensorMap* bmap = &P.p[it.q].b;
+                const int lo = offsets[it.e], hi = offsets[it.e + 1];
+                for (int row = lo; row < hi; row += WK) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(full_bar(stage), (uint32_t)STAGE_BYTES);
+#pragma unroll
+                    for (int bx = 0; bx < WM / 64; ++bx)
+                        tma_load_2d(sa + bx * BOX_BYTES, amap, it.m0 + 64 * bx, row,
+                                    full_bar(stage));
+#pragma unroll
+                    for (int bx = 0; bx < WN / 64; ++bx)
+                        tma_load_2d(sb + bx * BOX_BYTES, bmap, it.n0 + 64 * bx, row,
+                                    full_bar(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            // every stage's release has landed before this CTA may leave
+            for (int s = 0; ok && s < STAGES; ++s) {
+                ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer (whole warp: it also clears ragged rows) -----
+        int stage = 0, acc = 0;
+        uint32_t phase = 0, acc_phase = 0;
+        bool ok = true;
+        constexpr uint32_t idesc = instr_desc_bf16(WM, WN) | kInstrDescBothMN;
+        for (int w = w_begin; ok && w < w_end; w += w_step) {
+            const Item it = decode(P, w);
+            const int lo = offsets[it.e], hi = offsets[it.e + 1];
+            int go = 1;
+            if (lane == 0)
+                go = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status) ? 1 : 0;
+            if (!__shfl_sync(0xffffffffu, go, 0)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * WN);
+            for (int row = lo; row < hi; row += WK) {
+                if (lane == 0)
+                    go = mbar_wait(full_bar(stage), phase, abort_flag, dev_status) ? 1 : 0;
+                if (!__shfl_sync(0xffffffffu, go, 0)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                const int valid = min(WK, hi - row);
+                const int ksteps = (valid + UK - 1) / UK;
+                if (valid < ksteps * UK) {
+                    // rows valid .. ksteps*16-1 of all six boxes: 8 x 16 bytes per row and box
+                    uint8_t* tile = base_ptr + stage * STAGE_BYTES;
+                    const int n_rows = ksteps * UK - valid;
+                    const int n_vec = n_rows * (STAGE_BYTES / BOX_BYTES) * 8;
+                    for (int v = lane; v < n_vec; v += 32) {
+                        const int piece = v & 7, rb = v >> 3;
+                        const int r = valid + rb % n_rows, bx = rb / n_rows;
+                        *reinterpret_cast<uint4*>(tile + bx * BOX_BYTES + r * 128 + piece * 16) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    const uint64_t da = smem_desc_mn_sw128(sa, BOX_BYTES);
+                    const uint64_t db = smem_desc_mn_sw128(sb, BOX_BYTES);
+                    for (int kk = 0; kk < ksteps; ++kk)
+                        tc_mma_bf16(d_tmem, da + (uint64_t)(kk * (2048 >> 4)),
+                                    db + (uint64_t)(kk * (2048 >> 4)), idesc,
+                                    (row != lo || kk != 0) ? 1u : 0u);
+                    tc_commit(empty_bar(stage));
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (lane == 0) tc_commit(tfull_bar(acc));
+            __syncwarp();
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+    } else {
+        // ------------------------------ epilogue: TMEM -> float32 rows --------------------------
+        const int q = warp & 3;                       // TMEM lane quadrant this warp may read
+        float4* tbuf = reinterpret_cast<float4*>(epi_ptr + (warp - 2) * 4096);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool alive = true;
+        for (int w = w_begin; w < w_end; w += w_step) {
+            const Item it = decode(P, w);
+            const int M = P.p[it.q].M, N = P.p[it.q].N;
+            float* out = P.p[it.q].out + (size_t)it.e * M * N;
+            const bool empty = offsets[it.e + 1] == offsets[it.e];   // no MMA ran: gradient 0
+            if (alive) {
+                const bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status);
+                alive = __all_sync(0xffffffffu, ok);
+            }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * WN);
+#pragma unroll 1
+            for (int c = 0; c < WN && alive; c += 32) {
+                if (it.n0 + c >= N) break;
+                float v[32];
+                if (!empty) {
+                    tc_ld32(taddr + c, v);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0.f;
+                }
+                // the lane's row goes to shared memory in 16-byte pieces, piece j at slot
+                // j ^ (row & 7): conflict-free both for these stores and for the row reads below
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    tbuf[lane * 8 + (j ^ (lane & 7))] =
+                        make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                __syncwarp();
+#pragma unroll
+                for (int rr = 0; rr < 8; ++rr) {
+                    const int r = rr * 4 + (lane >> 3), j = lane & 7;
+                    const float4 val = tbuf[r * 8 + (j ^ (r & 7))];
+                    const int m = it.m0 + q * 32 + r, n = it.n0 + c + 4 * j;
+                    if (m < M && n + 4 <= N)
+                        *reinterpret_cast<float4*>(out + (size_t)m * N + n) = val;
+                }
+                __syncwarp();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && alive) mbar_arrive(tempty_bar(acc));
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ------------------------------ teardown ---------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // copies may still be in flight into this CTA's shared memory: give them time to land
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace wg
+
+// bf16 matrix [rows, cols] as an MN-major operand: boxes of 64 columns x 64 rows.
+static bool operand_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols) {
+    return tc::make_map_2d(m, ptr, rows, cols, wg::WK);
+}
+
+r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, const void* h,
+                          const void* da, const void* db, const int32_t* offsets, float* dw_gate,
+                          float* dw_up, float* dw_down, int32_t* dev_status, cudaStream_t cs) {
+    using namespace wg;
+    const uint64_t R = (uint64_t)s->T * s->K;
+    if (R == 0) return R3_OK;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SMEM_BYTES) != cudaSuccess)
+            return R3_ERR_CUDA;
+        attr_set = true;
+    }
+    Params P;
+    const void* a_ptr[3] = {dout, da, db};
+    const void* b_ptr[3] = {h, xp, xp};
+    float* out[3] = {dw_down, dw_gate, dw_up};
+    const int Ms[3] = {s->d, s->F, s->F}, Ns[3] = {s->F, s->d, s->d};
+    int items = 0;
+    for (int q = 0; q < 3; ++q) {
+        Problem& p = P.p[q];
+        if (!operand_map(&p.a, a_ptr[q], R, (uint64_t)Ms[q]) ||
+            !operand_map(&p.b, b_ptr[q], R, (uint64_t)Ns[q]))
+            return R3_ERR_CUDA;
+        p.out = out[q];
+        p.M = Ms[q];
+        p.N = Ns[q];
+        p.mt = (Ms[q] + WM - 1) / WM;
+        p.nt = (Ns[q] + WN - 1) / WN;
+        p.item0 = items;
+        items += s->E * p.mt * p.nt;
+    }
+    P.n_problems = 3;
+    P.total_items = items;
+    const int grid = items < sm_count() ? items : sm_count();
+    wgrad_kernel<<<grid, THREADS, SMEM_BYTES, cs>>>(P, offsets, dev_status);
+    return launch_status();
+}
+
+}  // namespace r3

@@ -37,7 +37,7 @@ EXPORTS = [
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
     "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
-    "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
+    "r3_grouped_swiglu_bwd", "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
     "r3_replay_layer_train_workspace_bytes", "r3_replay_layer_train",
     "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
@@ -59,7 +59,8 @@ lib.r3_grouped_swiglu_bwd_input.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, 
 lib.r3_grouped_swiglu_train.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, _P, _P]
 lib.r3_scale_rows.argtypes = [_SP] + [_P] * 5
 lib.r3_input_grad_finish.argtypes = [_SP] + [_P] * 11
-lib.r3_replay_layer_train.argtypes = [_SP] + [_P] * 12 + [ctypes.c_size_t, _P, _P]
+lib.r3_replay_layer_train.argtypes = [_SP] + [_P] * 15 + [ctypes.c_size_t, _P, _P]
+lib.r3_grouped_swiglu_bwd.argtypes = [_SP] + [_P] * 13 + [ctypes.c_size_t, _P, _P]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
            "r3_grouped_swiglu_bwd_workspace_bytes", "r3_replay_layer_train_workspace_bytes",
            "r3_replay_stack_workspace_bytes",
@@ -596,9 +597,29 @@ def input_grad_finish(s: Shape, dxp, row_of_slot, slot_of_row, offsets, dlogits,
     return dx, dw_r
 
 
+def grouped_swiglu_bwd(s: Shape, xp, dout, pre_gate, pre_up, offsets, w_gate, w_up, w_down, *,
+                       ws=None, dev_status=None, stream=None):
+    """Backward of the grouped experts: (dxp [R,d], dw_gate, dw_up [E,F,d], dw_down [E,d,F])."""
+    dev = _dev(dout)
+    dxp = torch.empty((s.T * s.K, s.d), dtype=_act_dtype(s), device=dev)
+    dw_gate = torch.empty((s.E, s.F, s.d), dtype=torch.float32, device=dev)
+    dw_up = torch.empty((s.E, s.F, s.d), dtype=torch.float32, device=dev)
+    dw_down = torch.empty((s.E, s.d, s.F), dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = workspace(lib.r3_grouped_swiglu_bwd_workspace_bytes(ctypes.byref(s)), dev)
+    _check(lib.r3_grouped_swiglu_bwd(ctypes.byref(s), _ptr(xp), _ptr(dout), _ptr(pre_gate),
+                                     _ptr(pre_up), _ptr(offsets), _ptr(w_gate), _ptr(w_up),
+                                     _ptr(w_down), _ptr(dxp), _ptr(dw_gate), _ptr(dw_up),
+                                     _ptr(dw_down), _ptr(ws), ws.numel(), _ptr(dev_status),
+                                     _stream(stream)))
+    return dxp, dw_gate, dw_up, dw_down
+
+
 def replay_layer_train(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, ws=None,
-                       dev_status=None, stream=None):
-    """Forward and backward-to-input of one replayed layer: (y, dlogits, dx, dw_router)."""
+                       dev_status=None, stream=None, expert_grads=False, dw_experts=None):
+    """Forward and backward of one replayed layer: (y, dlogits, dx, dw_router), and with
+    expert_grads also (dw_gate, dw_up, dw_down) appended (float32; `dw_experts` may supply the
+    three output tensors)."""
     dev = _dev(x)
     y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
     dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
@@ -606,10 +627,19 @@ def replay_layer_train(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, 
     dw_r = torch.empty((s.E, s.d), dtype=torch.float32, device=dev)
     if ws is None:
         ws = workspace(lib.r3_replay_layer_train_workspace_bytes(ctypes.byref(s)), dev)
+    dws = (None, None, None)
+    if expert_grads:
+        dws = dw_experts or (
+            torch.empty((s.E, s.F, s.d), dtype=torch.float32, device=dev),
+            torch.empty((s.E, s.F, s.d), dtype=torch.float32, device=dev),
+            torch.empty((s.E, s.d, s.F), dtype=torch.float32, device=dev))
     _check(lib.r3_replay_layer_train(ctypes.byref(s), _ptr(x), _ptr(w_router), _ptr(idx),
                                      _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(dy), _ptr(y),
-                                     _ptr(dlogits), _ptr(dx), _ptr(dw_r), _ptr(ws), ws.numel(),
+                                     _ptr(dlogits), _ptr(dx), _ptr(dw_r), _ptr(dws[0]),
+                                     _ptr(dws[1]), _ptr(dws[2]), _ptr(ws), ws.numel(),
                                      _ptr(dev_status), _stream(stream)))
+    if expert_grads:
+        return (y, dlogits, dx, dw_r) + tuple(dws)
     return y, dlogits, dx, dw_r
 
 

@@ -188,3 +188,85 @@ def test_layer_backward_full_size_sampled_tokens(r3):
     # on samples, and against the oracle in full at the small sizes)
     ref_dw = f64(ds).T @ f64(case.x)
     assert rel_err(f64(dw_r), ref_dw) < 1e-5
+
+
+@pytest.mark.parametrize("T,d,E,K,F", [
+    (256, 256, 4, 2, 256),        # full tiles, every expert a multiple of 16 rows or not
+    (300, 2048, 16, 8, 768),      # the paper-like layer shape, ragged expert sizes
+    (77, 136, 6, 3, 72),          # ragged d, F; experts smaller than one 64-row block
+    (1500, 512, 3, 2, 264),       # experts spanning many 64-row blocks
+])
+def test_expert_weight_gradients(r3, T, d, E, K, F):
+    """r3_grouped_swiglu_bwd: dW_gate, dW_up, dW_down of every expert against the oracle, fed the
+    same stored bf16 pre-activations; an expert without rows gets zeros."""
+    rng = np.random.default_rng(T + d + 1)
+    pop = rng.random(E) ** 2 + 0.01
+    pop[E - 1] = 0.0                                  # the last expert is never picked
+    idx_np = np.argsort(-(rng.random((T, E)) * pop[None, :] + (pop[None, :] > 0)), axis=1)[:, :K]
+    assert not np.any(idx_np == E - 1)
+    _, offsets, ros, sor = O.permutation(idx_np, E)
+    bf = torch.bfloat16
+    g = torch.Generator().manual_seed(T)
+    x = torch.randn(T, d, generator=g).to(bf)
+    wg = (torch.randn(E, F, d, generator=g) * 0.05).to(bf)
+    wu = (torch.randn(E, F, d, generator=g) * 0.05).to(bf)
+    wd = (torch.randn(E, d, F, generator=g) * 0.05).to(bf)
+    xp = x[torch.from_numpy(sor.astype(np.int64)) // K].contiguous()
+    dout = torch.randn(T * K, d, generator=g).to(bf)
+    R = T * K
+    a = torch.empty(R, F, dtype=bf)
+    b = torch.empty(R, F, dtype=bf)
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        xe = f64(xp[lo:hi])
+        a[lo:hi] = torch.from_numpy(xe @ f64(wg[e]).T).to(bf)
+        b[lo:hi] = torch.from_numpy(xe @ f64(wu[e]).T).to(bf)
+    s = r3.make_shape(T, d, E, K, F)
+    st = r3.new_status("cuda")
+    args = (s, xp.cuda(), dout.cuda(), a.cuda(), b.cuda(), torch.from_numpy(offsets).cuda(),
+            wg.cuda(), wu.cuda(), wd.cuda())
+    dxp, dwg, dwu, dwd = r3.grouped_swiglu_bwd(*args, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    dxp_only = r3.grouped_swiglu_bwd_input(s, *args[2:])
+    assert torch.equal(dxp, dxp_only)
+    got = [f64(dwg), f64(dwu), f64(dwd)]
+    scale = [0.0, 0.0, 0.0]
+    refs = []
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        ref = O.swiglu_expert_bwd_weights(f64(xp[lo:hi]), f64(dout[lo:hi]), f32(wg[e]), f32(wu[e]),
+                                          f32(wd[e]))
+        refs.append(ref)
+        scale = [max(sc, float(np.abs(r).max())) for sc, r in zip(scale, ref)]
+    for e in range(E):
+        for k in range(3):
+            err = np.abs(got[k][e] - refs[e][k]).max() / scale[k]
+            assert err < TOL_BF16, (e, k, err)
+    assert float(dwg[E - 1].abs().max()) == 0.0 and float(dwd[E - 1].abs().max()) == 0.0
+    again = r3.grouped_swiglu_bwd(*args)
+    assert all(torch.equal(p, q) for p, q in zip((dxp, dwg, dwu, dwd), again))
+
+
+def test_layer_backward_with_expert_weight_gradients(r3):
+    from paper_2510_11370_b200 import synth
+    from tests.helpers import Case
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_w", T=700, d=256, E=16, K=4,
+                     F=136)
+    case = Case(w)
+    c = case.cuda()
+    s = r3.shape_of(w)
+    st = r3.new_status("cuda")
+    y, ds, dx, dw_r, dwg, dwu, dwd = r3.replay_layer_train(
+        s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"], c["w_down"], c["dy"],
+        dev_status=st, expert_grads=True)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    ref = O.layer_bwd_weights(f64(case.x), f64(case.w_r), case.idx_np(), f32(case.w_gate),
+                              f32(case.w_up), f32(case.w_down), f64(case.dy))
+    for k, got in enumerate((dwg, dwu, dwd)):
+        full = np.stack([ref[e][k] for e in range(w.E)])
+        assert rel_err(f64(got), full) < TOL_BF16
+    y0, ds0, dx0, dwr0 = r3.replay_layer_train(s, c["x"], c["w_r"], c["idx"], c["w_gate"],
+                                               c["w_up"], c["w_down"], c["dy"])
+    assert torch.equal(dx, dx0) and torch.equal(dw_r, dwr0) and torch.equal(y, y0)
