@@ -13,6 +13,7 @@ single bf16 layer (T=4096, d=2048, E=128, K=8, F=768).  One JSON line is printed
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
 import statistics
@@ -451,6 +452,98 @@ def run_stack(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_train(args, w):
+    """Forward plus the whole Update-stage backward of one replayed layer (r3_replay_layer_train
+    with expert-weight gradients), with the backward's pieces timed apart."""
+    import torch
+    from paper_2510_11370_b200 import build, synth
+    build.build()
+    from paper_2510_11370_b200 import r3
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    dev = torch.device("cuda", 0)
+    peaks = load_peaks()
+    s = r3.shape_of(w)
+    T, K, E, d, F = w.T, w.K, w.E, w.d, w.F
+    R = T * K
+    x = synth.activations(w, dev)
+    dy = synth.upstream_grad(w, dev)
+    w_r = synth.router_weight(w, dev)
+    wg, wu, wd = synth.expert_weights(w, dev)
+    _, lg = r3.capture_topk_ws(s, 1, x, w_r, want_idx=False, want_logits=True)
+    idx = synth.make_record(w, lg)
+    st = r3.new_status(dev)
+    ws = r3.workspace(r3.lib.r3_replay_layer_train_workspace_bytes(ctypes.byref(s)), dev)
+    dws = (torch.empty((E, F, d), dtype=torch.float32, device=dev),
+           torch.empty((E, F, d), dtype=torch.float32, device=dev),
+           torch.empty((E, d, F), dtype=torch.float32, device=dev))
+
+    def timed(fn, steps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    def step():
+        r3.replay_layer_train(s, x, w_r, idx, wg, wu, wd, dy, ws=ws, dev_status=st,
+                              expert_grads=True, dw_experts=dws)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.25)
+    t0 = time.time()
+    ms = timed(step, args.steps)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    assert st.item() == 0
+    # pieces
+    counts, offsets, ros, sor, xp = r3.permute(s, idx, x)
+    o, a, b = r3.grouped_swiglu_train(s, xp, offsets, wg, wu, wd)
+    gates = torch.rand((T, K), dtype=torch.float32, device=dev)
+    dout = torch.empty((R, d), dtype=w.act_dtype, device=dev)
+    bws = r3.workspace(r3.lib.r3_grouped_swiglu_bwd_workspace_bytes(ctypes.byref(s)), dev)
+    lws = r3.workspace(r3.replay_layer_workspace_bytes(s), dev)
+    dl = torch.randn((T, E), dtype=torch.float32, device=dev)
+    n = min(args.steps, 20)
+    seg = {
+        "forward": timed(lambda: r3.replay_layer(s, x, w_r, idx, wg, wu, wd, dy, ws=lws), n),
+        "scale_rows": timed(lambda: r3.scale_rows(s, dy, gates, ros, dout), n),
+        "dgrad": timed(lambda: r3.grouped_swiglu_bwd_input(s, dout, a, b, offsets, wg, wu, wd,
+                                                           ws=bws), n),
+        "dgrad_wgrad": timed(lambda: r3.grouped_swiglu_bwd(s, xp, dout, a, b, offsets, wg, wu, wd,
+                                                           ws=bws), n),
+        "input_grad_finish": timed(lambda: r3.input_grad_finish(s, dout, ros, sor, offsets, dl,
+                                                                idx, x, w_r), n),
+    }
+    seg["wgrad"] = seg["dgrad_wgrad"] - seg["dgrad"]
+    flop_fwd = 6.0 * R * d * F
+    wgrad_bytes = 3.0 * E * F * d * 4 + 2.0 * R * d * 2 + 3.0 * R * F * 2
+    line = {
+        "metric": METRIC, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "mode": "forward + backward (dx, dW_r, dW_experts)",
+                   "T": T, "d": d, "E": E, "K": K, "F": F,
+                   "l2": "weights (1.2 GB) and weight gradients (2.4 GB) exceed the 126 MB L2"},
+        "segments_ms": {k: round(v, 4) for k, v in seg.items()},
+        "tflops": {"step (18 R d F)": round(3 * flop_fwd / (ms * 1e-3) / 1e12, 1),
+                   "dgrad": round(flop_fwd / (seg["dgrad"] * 1e-3) / 1e12, 1),
+                   "wgrad": round(flop_fwd / (seg["wgrad"] * 1e-3) / 1e12, 1)},
+        "wgrad_gbs": round(wgrad_bytes / (seg["wgrad"] * 1e-3) / 1e9, 1),
+        "clocks": clocks, "peaks": peaks,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def run_capture(args, w):
     """Config 4, inference side: router logits + TopKMask of a decode batch for `w.layers` layers
     in one launch (r3_capture_topk_batched), records packed as uint8."""
@@ -598,6 +691,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stack", action="store_true",
                     help="with a multi-layer workload (c5_stack48): time all its blocks, weights resident")
+    ap.add_argument("--train", action="store_true",
+                    help="time forward + the whole backward of one layer (bf16 workloads)")
     args = ap.parse_args()
     from paper_2510_11370_b200 import synth
     if args.workload == "diag":
@@ -605,6 +700,8 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.impl != "reference" and args.workload == "c4_capture":
         return run_capture(args, w)
+    if args.impl != "reference" and args.train:
+        return run_train(args, w)
     if args.impl != "reference" and w.layers > 1 and args.stack:
         return run_stack(args, w)
     if args.impl == "reference":

@@ -335,7 +335,8 @@ r3_status r3_scale_rows(const r3_shape* shape, const void* dy, const float* gate
  * (dlogits is zero outside the record, so these are the full products dlogits W_r and
  * dlogits^T x.)  dxp [R,d], dlogits [T,E] float32, idx [T,K], x [T,d], w_router [E,d]
  * (router_w_dtype), dx [T,d], dw_router [E,d] float32; row_of_slot / slot_of_row / offsets from
- * r3_permute.  Sums run in float32 in slot order and in ascending token order: reproducible.  An
+ * r3_permute.  Sums run in float32 in a fixed order (dx: slot order; dw_router: eight interleaved
+ * partial sums over the expert's rows, added in order): reproducible.  An
  * expert that appears twice in a token's record contributes its term twice to dx, as the
  * gradient of the gate does.  No workspace. */
 r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp, const int32_t* row_of_slot,

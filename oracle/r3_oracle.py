@@ -381,3 +381,35 @@ def layer_bwd_weights(x, w_r, idx_infer, w_gate, w_up, w_down, dy, experts=None)
         do = g[tt, jj][:, None] * dy[tt]
         out[int(i)] = swiglu_expert_bwd_weights(x[tt], do, w_gate[i], w_up[i], w_down[i])
     return out
+
+
+# ----------------------------------------------------------------------------------------------
+# The exact backward chain of a stack of residual replayed blocks (benchmark configuration 5)
+# ----------------------------------------------------------------------------------------------
+def replay_stack_bwd_tokens(x_rows, layers, dy_rows, store=None):
+    """x_{l+1} = store(x_l + y_replay,l(x_l)) for L blocks, then the gradient of
+    <dy, x_L> back through every block with the recorded masks held constant:
+        g_L = dy,   g_l = store(g_{l+1} + dx_l(g_{l+1}))
+    where dx_l, ds_l, dW_r,l are layer_bwd_input of block l at its input x_l with upstream
+    gradient g_{l+1} (the residual path carries g_{l+1} unchanged).  Tokens are independent, so a
+    subset can be followed on its own; dW_r,l then holds the sum over these tokens only.
+    Returns dict(x_out, dx0, ds=[...], dw_r=[...]) with one entry per block."""
+    x = _f64(x_rows)
+    xs = []
+    for (w_r, idx_rows, w_gate, w_up, w_down) in layers:
+        xs.append(x)
+        s = router_logits(x, w_r)
+        y, _, _ = replay_output(x, s, np.asarray(idx_rows, dtype=np.int64), w_gate, w_up, w_down)
+        x = x + y
+        if store is not None:
+            x = _f64(store(x))
+    g = _f64(dy_rows)
+    dss, dwrs = [None] * len(layers), [None] * len(layers)
+    for l in range(len(layers) - 1, -1, -1):
+        w_r, idx_rows, w_gate, w_up, w_down = layers[l]
+        res = layer_bwd_input(xs[l], w_r, idx_rows, w_gate, w_up, w_down, g)
+        dss[l], dwrs[l] = res["ds"], res["dw_r"]
+        g = g + res["dx"]
+        if store is not None:
+            g = _f64(store(g))
+    return dict(x_out=x, dx0=g, ds=dss, dw_r=dwrs)

@@ -518,3 +518,72 @@ def test_expert_weight_gradients_autograd_second_opinion_and_special_cases():
     assert list(part) == [1] and all(np.array_equal(a, b) for a, b in zip(part[1], got[1]))
     z = O.layer_bwd_weights(x, w_r, idx, wg, wu, wd, np.zeros_like(dy))
     assert all(np.all(m == 0) for i in z for m in z[i])
+
+
+# ---------------------------------------------------------------------------------------------
+# exact backward chain of a residual stack
+# ---------------------------------------------------------------------------------------------
+def _tiny_stack(seed, L=3, T=4, d=5, E=4, K=2, F=3):
+    layers = []
+    for l in range(L):
+        x, w_r, idx, wg, wu, wd, dy = _tiny_layer(seed + l, T=T, d=d, E=E, K=K, F=F)
+        layers.append((w_r, idx, wg * 0.7, wu * 0.7, wd * 0.7))
+    x0, _, _, _, _, _, dy = _tiny_layer(seed + 100, T=T, d=d, E=E, K=K, F=F)
+    return x0, layers, dy
+
+
+def _stack_loss(x0, layers, dy):
+    x = x0
+    for (w_r, idx, wg, wu, wd) in layers:
+        y, _, _ = O.replay_output(x, O.router_logits(x, w_r), idx, wg, wu, wd)
+        x = x + y
+    return float(np.sum(dy * x))
+
+
+def test_stack_backward_chain_matches_central_differences():
+    x0, layers, dy = _tiny_stack(40)
+    got = O.replay_stack_bwd_tokens(x0, layers, dy)
+    h = 1e-6
+    num = np.zeros_like(x0)
+    for pos in np.ndindex(*x0.shape):
+        xp, xm = x0.copy(), x0.copy()
+        xp[pos] += h
+        xm[pos] -= h
+        num[pos] = (_stack_loss(xp, layers, dy) - _stack_loss(xm, layers, dy)) / (2 * h)
+    assert np.abs(got["dx0"] - num).max() / np.abs(num).max() < 1e-7
+    # router weight of the middle block
+    l = 1
+    w_r = layers[l][0]
+    numw = np.zeros_like(w_r)
+    for pos in np.ndindex(*w_r.shape):
+        keep = w_r[pos]
+        w_r[pos] = keep + h
+        up = _stack_loss(x0, layers, dy)
+        w_r[pos] = keep - h
+        dn = _stack_loss(x0, layers, dy)
+        w_r[pos] = keep
+        numw[pos] = (up - dn) / (2 * h)
+    assert np.abs(got["dw_r"][l] - numw).max() / np.abs(numw).max() < 1e-6
+
+
+def test_stack_backward_special_cases():
+    x0, layers, dy = _tiny_stack(50)
+    full = O.replay_stack_bwd_tokens(x0, layers, dy)
+    # tokens are independent: a subset gives the same rows
+    sel = np.array([0, 2])
+    sub = O.replay_stack_bwd_tokens(x0[sel], [(w, i[sel], a, b, c) for (w, i, a, b, c) in layers],
+                                    dy[sel])
+    assert np.allclose(sub["dx0"], full["dx0"][sel], atol=1e-13)
+    assert np.allclose(sub["ds"][0], full["ds"][0][sel], atol=1e-13)
+    # one block: the chain is the layer's gradient plus the identity path
+    one = O.replay_stack_bwd_tokens(x0, layers[:1], dy)
+    w_r, idx, wg, wu, wd = layers[0]
+    lay = O.layer_bwd_input(x0, w_r, idx, wg, wu, wd, dy)
+    assert np.allclose(one["dx0"], dy + lay["dx"], atol=1e-13)
+    # the last block's router gradient is that of the forward-only stack with the same dy
+    xL, dss = O.replay_stack_tokens(x0, layers, dy)
+    assert np.allclose(full["ds"][-1], dss[-1], atol=1e-13) and np.allclose(full["x_out"], xL)
+    # zero experts (W_down = 0): every block is the identity, so dx0 = dy and ds = 0
+    dead = [(w, i, a, b, np.zeros_like(c)) for (w, i, a, b, c) in layers]
+    z = O.replay_stack_bwd_tokens(x0, dead, dy)
+    assert np.array_equal(z["dx0"], dy) and all(np.all(s == 0) for s in z["ds"])
