@@ -330,11 +330,14 @@ r3_status r3_scale_rows(const r3_shape* shape, const void* dy, const float* gate
 /* Last step of the backward to the layer input.  The input x_t reaches the loss through its K
  * experts and through the training logits s = x W_r^T that feed the replay gate (the recorded
  * mask is a constant, Section 4.1):
- *   dx[t,:]        = sum_j dxp[row_of_slot[t,j], :] + sum_j dlogits[t, e_j] * W_r[e_j, :]
+ *   dx[t,:]        = dx_residual[t,:] + sum_j dxp[row_of_slot[t,j], :]
+ *                    + sum_j dlogits[t, e_j] * W_r[e_j, :]
  *   dw_router[e,:] = sum over tokens t whose record holds e of dlogits[t,e] * x[t,:]
  * (dlogits is zero outside the record, so these are the full products dlogits W_r and
  * dlogits^T x.)  dxp [R,d], dlogits [T,E] float32, idx [T,K], x [T,d], w_router [E,d]
- * (router_w_dtype), dx [T,d], dw_router [E,d] float32; row_of_slot / slot_of_row / offsets from
+ * (router_w_dtype), dx [T,d], dw_router [E,d] float32; dx_residual [T,d] (the gradient that
+ * reaches x around the layer, e.g. through a residual connection) or null for none, never the
+ * same buffer as dx; row_of_slot / slot_of_row / offsets from
  * r3_permute.  Sums run in float32 in a fixed order (dx: slot order; dw_router: eight interleaved
  * partial sums over the expert's rows, added in order): reproducible.  An
  * expert that appears twice in a token's record contributes its term twice to dx, as the
@@ -342,7 +345,8 @@ r3_status r3_scale_rows(const r3_shape* shape, const void* dy, const float* gate
 r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp, const int32_t* row_of_slot,
                                const int32_t* slot_of_row, const int32_t* offsets,
                                const float* dlogits, const void* idx, const void* x,
-                               const void* w_router, void* dx, float* dw_router, void* stream);
+                               const void* w_router, const void* dx_residual, void* dx,
+                               float* dw_router, void* stream);
 
 /* r3_replay_layer followed by its backward to the layer input and to the router weight, one
  * enqueue: y, dlogits as in r3_replay_layer, then dout = g dy, the expert input gradient
@@ -357,6 +361,25 @@ r3_status r3_replay_layer_train(const r3_shape* shape, const void* x, const void
                                 const void* w_down, const void* dy, void* y, float* dlogits,
                                 void* dx, float* dw_router, float* dw_gate, float* dw_up,
                                 float* dw_down, void* workspace, size_t ws_bytes,
+                                int32_t* dev_status, void* stream);
+
+/* L residual blocks x_{l+1} = x_l + y_replay,l(x_l) (as r3_replay_stack), then the exact backward
+ * chain of <dy, x_L>:  g_L = dy,  g_l = g_{l+1} + dx_l(g_{l+1}),  where block l's backward is
+ * r3_replay_layer_train's at its own input x_l with upstream gradient g_{l+1} and the residual
+ * path carries g_{l+1} through unchanged.  Block inputs are kept (L activations of [T,d]); each
+ * block's forward is run again in the backward pass instead of keeping its intermediates.
+ * Per-block tensors are stacked along a leading L: w_router [L,E,d], idx [L,T,K], w_gate / w_up
+ * [L,E,F,d], w_down [L,E,d,F]; dy [T,d] = dL/dx_L.  Outputs: x_out [T,d] = x_L, dlogits [L,T,E]
+ * (the exact router-logit gradients), dx0 [T,d] = dL/dx_0 (not the same buffer as dy),
+ * dw_router [L,E,d] float32, and dw_gate / dw_up [L,E,F,d], dw_down [L,E,d,F] float32 or all
+ * three null.  Activations and the gradients g_l are stored in bf16 between blocks.  bf16 only.
+ * workspace: r3_replay_stack_train_workspace_bytes(shape, L). */
+size_t r3_replay_stack_train_workspace_bytes(const r3_shape* shape, int32_t L);
+r3_status r3_replay_stack_train(const r3_shape* shape, int32_t L, const void* x0,
+                                const void* w_router, const void* idx, const void* w_gate,
+                                const void* w_up, const void* w_down, const void* dy, void* x_out,
+                                float* dlogits, void* dx0, float* dw_router, float* dw_gate,
+                                float* dw_up, float* dw_down, void* workspace, size_t ws_bytes,
                                 int32_t* dev_status, void* stream);
 
 /* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */

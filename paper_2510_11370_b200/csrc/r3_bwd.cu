@@ -44,13 +44,15 @@ scale_rows_kernel(const ActT* __restrict__ dy, const float* __restrict__ gates,
     }
 }
 
-// One CTA per token, a thread per 16-byte column piece: the K expert-path rows are summed in slot
-// order, then the K router-path rows ds_j W_r[e_j] are added in slot order.
+// One CTA per token, a thread per 16-byte column piece: starting from the residual-path gradient
+// (if any), the K expert-path rows are added in slot order, then the K router-path rows
+// ds_j W_r[e_j] in slot order.
 template <typename ActT, typename IdxT, typename WrT>
 __global__ void __launch_bounds__(256)
 dx_kernel(const ActT* __restrict__ dxp, const int32_t* __restrict__ row_of_slot,
           const float* __restrict__ dlogits, const IdxT* __restrict__ idx,
-          const WrT* __restrict__ w_r, ActT* __restrict__ dx, int T, int E, int K, int d) {
+          const WrT* __restrict__ w_r, const ActT* __restrict__ dres, ActT* __restrict__ dx, int T,
+          int E, int K, int d) {
     using V = Vec16<ActT>;
     constexpr int N = V::N;
     const int t = blockIdx.x;
@@ -60,6 +62,7 @@ dx_kernel(const ActT* __restrict__ dxp, const int32_t* __restrict__ row_of_slot,
         float acc[N];
 #pragma unroll
         for (int i = 0; i < N; ++i) acc[i] = 0.f;
+        if (dres) reinterpret_cast<const V*>(dres)[(size_t)t * row_vecs + c].unpack(acc);
         for (int j = 0; j < K; ++j) {
             const int32_t r = row_of_slot[(size_t)t * K + j];
             if (r < 0) continue;
@@ -155,14 +158,17 @@ extern "C" r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp
                                           const int32_t* row_of_slot, const int32_t* slot_of_row,
                                           const int32_t* offsets, const float* dlogits,
                                           const void* idx, const void* x, const void* w_router,
-                                          void* dx, float* dw_router, void* stream) {
+                                          const void* dx_residual, void* dx, float* dw_router,
+                                          void* stream) {
     r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
     if (shape->T == 0) return R3_OK;
     if (!dxp || !row_of_slot || !slot_of_row || !offsets || !dlogits || !idx || !x || !w_router ||
         !dx || !dw_router)
         return R3_ERR_INVALID_ARG;
-    if (!r3::aligned(dxp, 16) || !r3::aligned(dx, 16)) return R3_ERR_INVALID_ARG;
+    if (!r3::aligned(dxp, 16) || !r3::aligned(dx, 16) || !r3::aligned(dx_residual, 16) ||
+        dx_residual == dx)
+        return R3_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int T = shape->T, E = shape->E, K = shape->K, d = shape->d;
     const bool wr_bf16 = shape->router_w_dtype == R3_BF16;
@@ -170,11 +176,13 @@ extern "C" r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp
         if (wr_bf16)
             r3::dx_kernel<ActT, IdxT, __nv_bfloat16><<<T, 256, 0, cs>>>(
                 static_cast<const ActT*>(dxp), row_of_slot, dlogits, static_cast<const IdxT*>(idx),
-                static_cast<const __nv_bfloat16*>(w_router), static_cast<ActT*>(dx), T, E, K, d);
+                static_cast<const __nv_bfloat16*>(w_router),
+                static_cast<const ActT*>(dx_residual), static_cast<ActT*>(dx), T, E, K, d);
         else
             r3::dx_kernel<ActT, IdxT, float><<<T, 256, 0, cs>>>(
                 static_cast<const ActT*>(dxp), row_of_slot, dlogits, static_cast<const IdxT*>(idx),
-                static_cast<const float*>(w_router), static_cast<ActT*>(dx), T, E, K, d);
+                static_cast<const float*>(w_router), static_cast<const ActT*>(dx_residual),
+                static_cast<ActT*>(dx), T, E, K, d);
     }));
     R3_DISPATCH_ACT(shape, ActT,
         r3::dwr_kernel<ActT><<<dim3(E, (d + 63) / 64), 256, 0, cs>>>(

@@ -200,6 +200,35 @@ extern "C" size_t r3_replay_layer_train_workspace_bytes(const r3_shape* shape) {
     return r3::carve_train(shape, nullptr).total;
 }
 
+namespace r3 {
+// Forward of one layer (pre-activations kept), then its backward.  `dres` (may be null) is the
+// gradient that reaches x around the layer; the expert-weight outputs may all be null.
+static r3_status run_layer_train(const r3_shape* shape, const void* x, const void* w_router,
+                                 const void* idx, const void* w_gate, const void* w_up,
+                                 const void* w_down, const void* dy, const void* dres, void* y,
+                                 float* dlogits, void* dx, float* dw_router, float* dw_gate,
+                                 float* dw_up, float* dw_down, void* workspace,
+                                 int32_t* dev_status, void* stream) {
+    const TrainWs t = carve_train(shape, workspace);
+    const LayerWs w = carve(shape, t.inner);
+    r3_status st = run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y,
+                             dlogits, t.gates, t.inner, dev_status, stream, nullptr, t.pre_gate,
+                             t.pre_up);
+    if (st != R3_OK) return st;
+    // the expert outputs are no longer needed: their buffer takes dout = g dy
+    if ((st = r3_scale_rows(shape, dy, t.gates, w.row_of_slot, w.o, stream)) != R3_OK) return st;
+    st = dw_gate ? r3_grouped_swiglu_bwd(shape, w.xp, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
+                                         w_up, w_down, t.dxp, dw_gate, dw_up, dw_down, t.bwd_ws,
+                                         t.bwd_bytes, dev_status, stream)
+                 : r3_grouped_swiglu_bwd_input(shape, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
+                                               w_up, w_down, t.dxp, t.bwd_ws, t.bwd_bytes,
+                                               dev_status, stream);
+    if (st != R3_OK) return st;
+    return r3_input_grad_finish(shape, t.dxp, w.row_of_slot, w.slot_of_row, w.offsets, dlogits,
+                                idx, x, w_router, dres, dx, dw_router, stream);
+}
+}  // namespace r3
+
 extern "C" r3_status r3_replay_layer_train(const r3_shape* shape, const void* x,
                                            const void* w_router, const void* idx,
                                            const void* w_gate, const void* w_up,
@@ -220,22 +249,77 @@ extern "C" r3_status r3_replay_layer_train(const r3_shape* shape, const void* x,
     if (!workspace || !r3::aligned(workspace, 256) ||
         ws_bytes < r3_replay_layer_train_workspace_bytes(shape))
         return R3_ERR_WORKSPACE;
-    const r3::TrainWs t = r3::carve_train(shape, workspace);
-    const r3::LayerWs w = r3::carve(shape, t.inner);
-    st = r3::run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y, dlogits,
-                       t.gates, t.inner, dev_status, stream, nullptr, t.pre_gate, t.pre_up);
+    return r3::run_layer_train(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y,
+                               dlogits, dx, dw_router, dw_gate, dw_up, dw_down, workspace,
+                               dev_status, stream);
+}
+
+// ---- L residual blocks: forward, then the exact backward chain ---------------------------------
+extern "C" size_t r3_replay_stack_train_workspace_bytes(const r3_shape* shape, int32_t L) {
+    if (r3::check_shape(shape) != R3_OK || shape->act_dtype != R3_BF16 || L <= 0) return 0;
+    const size_t xb = r3::round_up((size_t)shape->T * shape->d * r3::act_bytes(shape), 256);
+    return ((size_t)L + 3) * xb + r3_replay_layer_train_workspace_bytes(shape);
+}
+
+extern "C" r3_status r3_replay_stack_train(const r3_shape* shape, int32_t L, const void* x0,
+                                           const void* w_router, const void* idx,
+                                           const void* w_gate, const void* w_up,
+                                           const void* w_down, const void* dy, void* x_out,
+                                           float* dlogits, void* dx0, float* dw_router,
+                                           float* dw_gate, float* dw_up, float* dw_down,
+                                           void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                           void* stream) {
+    r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
-    // the expert outputs are no longer needed: their buffer takes dout = g dy
-    if ((st = r3_scale_rows(shape, dy, t.gates, w.row_of_slot, w.o, stream)) != R3_OK) return st;
-    st = weights ? r3_grouped_swiglu_bwd(shape, w.xp, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
-                                         w_up, w_down, t.dxp, dw_gate, dw_up, dw_down, t.bwd_ws,
-                                         t.bwd_bytes, dev_status, stream)
-                 : r3_grouped_swiglu_bwd_input(shape, w.o, t.pre_gate, t.pre_up, w.offsets, w_gate,
-                                               w_up, w_down, t.dxp, t.bwd_ws, t.bwd_bytes,
-                                               dev_status, stream);
-    if (st != R3_OK) return st;
-    return r3_input_grad_finish(shape, t.dxp, w.row_of_slot, w.slot_of_row, w.offsets, dlogits,
-                                idx, x, w_router, dx, dw_router, stream);
+    if (shape->act_dtype != R3_BF16) return R3_ERR_UNSUPPORTED;
+    if (L <= 0) return R3_ERR_INVALID_ARG;
+    if (shape->T == 0) return R3_OK;
+    if (!x0 || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !x_out || !dlogits ||
+        !dx0 || !dw_router || dx0 == dy)
+        return R3_ERR_INVALID_ARG;
+    const bool weights = dw_gate || dw_up || dw_down;
+    if (weights && (!dw_gate || !dw_up || !dw_down)) return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_stack_train_workspace_bytes(shape, L))
+        return R3_ERR_WORKSPACE;
+    const size_t T = shape->T, d = shape->d, E = shape->E, F = shape->F, K = shape->K;
+    const size_t es = r3::act_bytes(shape);
+    const size_t xb = r3::round_up(T * d * es, 256);
+    char* ws = static_cast<char*>(workspace);
+    // x_1 .. x_{L-1} are kept for the backward pass (x_0 is the caller's, x_L goes to x_out)
+    auto kept = [&](int32_t l) { return static_cast<void*>(ws + (size_t)l * xb); };
+    void* grad[2] = {ws + (size_t)L * xb, ws + ((size_t)L + 1) * xb};
+    void* y_scratch = ws + ((size_t)L + 2) * xb;
+    void* inner = ws + ((size_t)L + 3) * xb;
+    const size_t rw = E * d * (shape->router_w_dtype == R3_BF16 ? 2 : 4);
+    const size_t ew = E * F * d * es, rec = T * K * r3::idx_bytes(shape);
+    auto at = [](const void* p, size_t off) { return static_cast<const char*>(p) + off; };
+    const void* cur = x0;
+    for (int32_t l = 0; l < L; ++l) {
+        void* nxt = (l == L - 1) ? x_out : kept(l + 1);
+        st = r3::run_layer(shape, cur, at(w_router, l * rw), at(idx, l * rec), at(w_gate, l * ew),
+                           at(w_up, l * ew), at(w_down, l * ew), dy, cur, nxt,
+                           dlogits + (size_t)l * T * E, nullptr, inner, dev_status, stream);
+        if (st != R3_OK) return st;
+        cur = nxt;
+    }
+    // g_L = dy;  g_l = g_{l+1} + (gradient through block l at x_l), block l's forward recomputed
+    const void* g = dy;
+    for (int32_t l = L - 1; l >= 0; --l) {
+        const void* xl = l == 0 ? x0 : kept(l);
+        void* g_out = l == 0 ? dx0 : grad[l & 1];
+        st = r3::run_layer_train(shape, xl, at(w_router, l * rw), at(idx, l * rec),
+                                 at(w_gate, l * ew), at(w_up, l * ew), at(w_down, l * ew), g, g,
+                                 y_scratch, dlogits + (size_t)l * T * E, g_out,
+                                 dw_router + (size_t)l * E * d,
+                                 weights ? dw_gate + (size_t)l * E * F * d : nullptr,
+                                 weights ? dw_up + (size_t)l * E * F * d : nullptr,
+                                 weights ? dw_down + (size_t)l * E * F * d : nullptr, inner,
+                                 dev_status, stream);
+        if (st != R3_OK) return st;
+        g = g_out;
+    }
+    return R3_OK;
 }
 
 // ---- a stack of L replayed MoE blocks with residual connections ------------------------------

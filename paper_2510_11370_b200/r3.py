@@ -39,6 +39,7 @@ EXPORTS = [
     "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
     "r3_grouped_swiglu_bwd", "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
     "r3_replay_layer_train_workspace_bytes", "r3_replay_layer_train",
+    "r3_replay_stack_train_workspace_bytes", "r3_replay_stack_train",
     "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
     "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
@@ -58,8 +59,11 @@ lib.r3_status_string.argtypes = [ctypes.c_int]
 lib.r3_grouped_swiglu_bwd_input.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, _P, _P]
 lib.r3_grouped_swiglu_train.argtypes = [_SP] + [_P] * 9 + [ctypes.c_size_t, _P, _P]
 lib.r3_scale_rows.argtypes = [_SP] + [_P] * 5
-lib.r3_input_grad_finish.argtypes = [_SP] + [_P] * 11
+lib.r3_input_grad_finish.argtypes = [_SP] + [_P] * 12
 lib.r3_replay_layer_train.argtypes = [_SP] + [_P] * 15 + [ctypes.c_size_t, _P, _P]
+lib.r3_replay_stack_train_workspace_bytes.restype = ctypes.c_size_t
+lib.r3_replay_stack_train_workspace_bytes.argtypes = [_SP, ctypes.c_int32]
+lib.r3_replay_stack_train.argtypes = [_SP, ctypes.c_int32] + [_P] * 15 + [ctypes.c_size_t, _P, _P]
 lib.r3_grouped_swiglu_bwd.argtypes = [_SP] + [_P] * 13 + [ctypes.c_size_t, _P, _P]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
            "r3_grouped_swiglu_bwd_workspace_bytes", "r3_replay_layer_train_workspace_bytes",
@@ -585,15 +589,15 @@ def scale_rows(s: Shape, dy, gates, row_of_slot, dout=None, *, stream=None):
 
 
 def input_grad_finish(s: Shape, dxp, row_of_slot, slot_of_row, offsets, dlogits, idx, x, w_router,
-                      *, stream=None):
+                      *, dx_residual=None, stream=None):
     """(dx [T,d], dw_router [E,d] float32) from the expert input gradient and dlogits."""
     dev = _dev(dxp)
     dx = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
     dw_r = torch.empty((s.E, s.d), dtype=torch.float32, device=dev)
     _check(lib.r3_input_grad_finish(ctypes.byref(s), _ptr(dxp), _ptr(row_of_slot),
                                     _ptr(slot_of_row), _ptr(offsets), _ptr(dlogits), _ptr(idx),
-                                    _ptr(x), _ptr(w_router), _ptr(dx), _ptr(dw_r),
-                                    _stream(stream)))
+                                    _ptr(x), _ptr(w_router), _ptr(dx_residual), _ptr(dx),
+                                    _ptr(dw_r), _stream(stream)))
     return dx, dw_r
 
 
@@ -641,6 +645,32 @@ def replay_layer_train(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, 
     if expert_grads:
         return (y, dlogits, dx, dw_r) + tuple(dws)
     return y, dlogits, dx, dw_r
+
+
+def replay_stack_train(s: Shape, L, x0, w_router, idx, w_gate, w_up, w_down, dy, *, ws=None,
+                       dev_status=None, stream=None, expert_grads=False):
+    """L residual blocks forward, then the exact backward chain:
+    (x_out, dlogits [L,T,E], dx0, dw_router [L,E,d]) (+ dw_gate, dw_up, dw_down)."""
+    dev = _dev(x0)
+    x_out = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    dx0 = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    dlogits = torch.empty((L, s.T, s.E), dtype=torch.float32, device=dev)
+    dw_r = torch.empty((L, s.E, s.d), dtype=torch.float32, device=dev)
+    dws = (None, None, None)
+    if expert_grads:
+        dws = (torch.empty((L, s.E, s.F, s.d), dtype=torch.float32, device=dev),
+               torch.empty((L, s.E, s.F, s.d), dtype=torch.float32, device=dev),
+               torch.empty((L, s.E, s.d, s.F), dtype=torch.float32, device=dev))
+    if ws is None:
+        ws = workspace(lib.r3_replay_stack_train_workspace_bytes(ctypes.byref(s), L), dev)
+    _check(lib.r3_replay_stack_train(ctypes.byref(s), L, _ptr(x0), _ptr(w_router), _ptr(idx),
+                                     _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(dy),
+                                     _ptr(x_out), _ptr(dlogits), _ptr(dx0), _ptr(dw_r),
+                                     _ptr(dws[0]), _ptr(dws[1]), _ptr(dws[2]), _ptr(ws),
+                                     ws.numel(), _ptr(dev_status), _stream(stream)))
+    if expert_grads:
+        return (x_out, dlogits, dx0, dw_r) + dws
+    return x_out, dlogits, dx0, dw_r
 
 
 def grouped_swiglu_bwd_input(s: Shape, dout, pre_gate, pre_up, offsets, w_gate, w_up, w_down,

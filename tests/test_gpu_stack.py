@@ -190,3 +190,67 @@ def test_residual_chain_of_48_blocks_full_size(r3):
         pytest.skip("needs about 75 GB of free device memory")
     sel = np.array([5, 4097, 9000, 16383])
     check_stack(r3, w, w.layers, sel, 2e-2, bf16_store, ds_layers=3)
+
+
+def check_stack_train(r3, w, L, sel, tol, expert_grads=False):
+    """r3_replay_stack_train against the oracle's exact chain on the tokens `sel` (all tokens when
+    sel covers them: then dW_r is compared too)."""
+    x0, dy, w_r, wg, wu, wd, idx = build_stack(w, L)
+    s = r3.shape_of(w)
+    st = r3.new_status("cuda")
+    out = r3.replay_stack_train(s, L, x0, w_r, idx, wg, wu, wd, dy, dev_status=st,
+                                expert_grads=expert_grads)
+    x_out, dlogits, dx0, dw_r = out[:4]
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    idx_np = idx.cpu().to(torch.int64).numpy()
+    layers = [(f64(w_r[l]), idx_np[l][sel], LayerExperts(wg, l), LayerExperts(wu, l),
+               LayerExperts(wd, l)) for l in range(L)]
+    ref = O.replay_stack_bwd_tokens(f64(x0)[sel], layers, f64(dy)[sel], store=bf16_store)
+    # stored activations and gradients pass through L bf16 roundings (see check_stack)
+    tol_chain = tol + np.sqrt(L) * 2.0 ** -8
+    err = lambda got, want: float(np.abs(got - want).max() / np.abs(want).max())
+    assert err(f64(x_out)[sel], ref["x_out"]) < tol_chain
+    assert err(f64(dx0)[sel], ref["dx0"]) < tol_chain
+    for l in range(L):
+        assert err(f64(dlogits[l])[sel], ref["ds"][l]) < tol_chain, l
+    if len(sel) == w.T:
+        for l in range(L):
+            assert err(f64(dw_r[l]), ref["dw_r"][l]) < tol_chain, l
+    # the forward half is r3_replay_stack's; a second run repeats the first bit for bit
+    x_fwd, _ = r3.replay_stack(s, L, x0, w_r, idx, wg, wu, wd, dy)
+    assert torch.equal(x_fwd, x_out)
+    again = r3.replay_stack_train(s, L, x0, w_r, idx, wg, wu, wd, dy, expert_grads=expert_grads)
+    assert all(torch.equal(a, b) for a, b in zip(out, again))
+    return out
+
+
+def test_small_stack_exact_backward_chain(r3):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="stack_bwd", T=300, d=256, E=16,
+                     K=4, F=128)
+    check_stack_train(r3, w, 3, np.arange(300), 2e-2)
+
+
+def test_one_block_stack_train_is_layer_train_plus_identity_path(r3):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="stack_bwd1", T=200, d=256, E=16,
+                     K=4, F=128)
+    x0, dy, w_r, wg, wu, wd, idx = build_stack(w, 1)
+    s = r3.shape_of(w)
+    x1, dl, dx0, dwr, dwg, dwu, dwd = r3.replay_stack_train(s, 1, x0, w_r, idx, wg, wu, wd, dy,
+                                                            expert_grads=True)
+    y, ds, dx, dwr1, g1, u1, d1 = r3.replay_layer_train(s, x0, w_r[0], idx[0], wg[0], wu[0],
+                                                        wd[0], dy, expert_grads=True)
+    assert torch.equal(dl[0], ds) and torch.equal(dwr[0], dwr1)
+    assert torch.equal(dwg[0], g1) and torch.equal(dwu[0], u1) and torch.equal(dwd[0], d1)
+    scale = float(dx0.float().abs().max())
+    assert (dx0.float() - (dy.float() + dx.float())).abs().max().item() <= scale * 2.0 ** -7
+
+
+def test_four_blocks_of_config5_shape_exact_backward_chain(r3):
+    """The configuration-5 block shape (T=16384, d=2048, E=128, K=8, F=768), four blocks chained,
+    sampled tokens followed by the oracle through the whole forward and backward chain."""
+    w = synth.WORKLOADS["c5_stack48"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 30e9:
+        pytest.skip("needs about 25 GB of free device memory")
+    check_stack_train(r3, w, 4, np.array([7, 4097, 9000, 16383]), 2e-2)
