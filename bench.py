@@ -384,7 +384,9 @@ def run_ours(args, w):
 
 def run_stack(args, w):
     """Config 5: `w.layers` MoE blocks back to back with all their weights resident
-    (r3_replay_blocks; every block has its own seeded input, record and weights)."""
+    (r3_replay_blocks; every block has its own seeded input, record and weights).  With --train:
+    the blocks chained through residual connections, forward and the exact backward chain
+    (r3_replay_stack_train, expert-weight gradients left out: 116 GB of float32 for 48 blocks)."""
     import torch
     from paper_2510_11370_b200 import build, synth
     build.build()
@@ -416,6 +418,13 @@ def run_stack(args, w):
     def step():
         r3.replay_blocks(s, L, x, w_r, idx, wg, wu, wd, dy, y=y, dlogits=dl, ws=ws, dev_status=st)
 
+    if args.train:
+        del y, ws
+        tws = r3.workspace(r3.lib.r3_replay_stack_train_workspace_bytes(ctypes.byref(s), L), dev)
+
+        def step():
+            r3.replay_stack_train(s, L, x[0], w_r, idx, wg, wu, wd, dy[0], ws=tws, dev_status=st)
+
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -433,12 +442,17 @@ def run_stack(args, w):
     ms = e0.elapsed_time(e1) / args.steps
     assert st.item() == 0
     clocks = sampler.stop(t0, t1)
-    flop = 6.0 * T * K * d * F * L
+    # forward 6 R d F per block; with --train: forward, forward again, and the 12 R d F of the
+    # two input-gradient products
+    flop = (24.0 if args.train else 6.0) * T * K * d * F * L
     line = {
         "metric": METRIC, "value": T / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "blocks": L, "T": T, "d": d, "E": E, "K": K, "F": F,
+                   "mode": ("residual chain, forward + exact backward (dx, dlogits, dW_r; block "
+                            "forward recomputed)" if args.train else "independent blocks, forward + "
+                            "router backward"),
                    "weights_gb": round(3 * L * E * F * d * 2 / 1e9, 1),
                    "l2": "58 GB of weights stream through the 126 MB L2 every step"},
         "layer_tokens_per_s": L * T / (ms * 1e-3),
@@ -447,7 +461,9 @@ def run_stack(args, w):
                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": round(flop / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
                      "peak_kind": f"bf16 matmul sustained, {peaks['source']}", "traffic": None},
-        "gpu_launches": LAUNCHES_PER_STEP * L * args.steps, "clocks": clocks, "peaks": peaks,
+        # --train: per block the forward, then the forward again plus 7 backward kernels
+        "gpu_launches": (2 * LAUNCHES_PER_STEP + 7 if args.train else LAUNCHES_PER_STEP) * L
+        * args.steps, "clocks": clocks, "peaks": peaks,
     }
     print(json.dumps(line), flush=True)
 
@@ -700,10 +716,10 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.impl != "reference" and args.workload == "c4_capture":
         return run_capture(args, w)
-    if args.impl != "reference" and args.train:
-        return run_train(args, w)
     if args.impl != "reference" and w.layers > 1 and args.stack:
         return run_stack(args, w)
+    if args.impl != "reference" and args.train:
+        return run_train(args, w)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -341,7 +341,7 @@ r3_status r3_scale_rows(const r3_shape* shape, const void* dy, const float* gate
  * r3_permute.  Sums run in float32 in a fixed order (dx: slot order; dw_router: eight interleaved
  * partial sums over the expert's rows, added in order): reproducible.  An
  * expert that appears twice in a token's record contributes its term twice to dx, as the
- * gradient of the gate does.  No workspace. */
+ * gradient of the gate does.  K <= 64 (R3_ERR_UNSUPPORTED beyond).  No workspace. */
 r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp, const int32_t* row_of_slot,
                                const int32_t* slot_of_row, const int32_t* offsets,
                                const float* dlogits, const void* idx, const void* x,

@@ -44,9 +44,37 @@ scale_rows_kernel(const ActT* __restrict__ dy, const float* __restrict__ gates,
     }
 }
 
+// N consecutive router-weight elements (N = 4 or 8, the address a multiple of 16 bytes) as floats.
+template <typename WrT, int N>
+__device__ __forceinline__ void load_row_piece(const WrT* p, float* out);
+template <> __device__ __forceinline__ void load_row_piece<float, 4>(const float* p, float* out) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <> __device__ __forceinline__ void load_row_piece<float, 8>(const float* p, float* out) {
+    load_row_piece<float, 4>(p, out);
+    load_row_piece<float, 4>(p + 4, out + 4);
+}
+template <>
+__device__ __forceinline__ void load_row_piece<__nv_bfloat16, 8>(const __nv_bfloat16* p,
+                                                                 float* out) {
+    Vec16<__nv_bfloat16> v = *reinterpret_cast<const Vec16<__nv_bfloat16>*>(p);
+    v.unpack(out);
+}
+template <>
+__device__ __forceinline__ void load_row_piece<__nv_bfloat16, 4>(const __nv_bfloat16* p,
+                                                                 float* out) {
+    const uint2 raw = *reinterpret_cast<const uint2*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+    out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+}
+
 // One CTA per token, a thread per 16-byte column piece: starting from the residual-path gradient
 // (if any), the K expert-path rows are added in slot order, then the K router-path rows
-// ds_j W_r[e_j] in slot order.
+// ds_j W_r[e_j] in slot order.  The token's K rows, experts and logit gradients are fetched once
+// into shared memory, so the row loads of the sums are independent of each other.
+constexpr int kDxMaxK = 64;
 template <typename ActT, typename IdxT, typename WrT>
 __global__ void __launch_bounds__(256)
 dx_kernel(const ActT* __restrict__ dxp, const int32_t* __restrict__ row_of_slot,
@@ -55,7 +83,19 @@ dx_kernel(const ActT* __restrict__ dxp, const int32_t* __restrict__ row_of_slot,
           int E, int K, int d) {
     using V = Vec16<ActT>;
     constexpr int N = V::N;
+    __shared__ int32_t s_row[kDxMaxK];
+    __shared__ int32_t s_e[kDxMaxK];
+    __shared__ float s_ds[kDxMaxK];
     const int t = blockIdx.x;
+    if (threadIdx.x < K) {
+        const int j = threadIdx.x;
+        s_row[j] = row_of_slot[(size_t)t * K + j];
+        const int e = idx_to_int(idx[(size_t)t * K + j]);
+        const bool ok = e >= 0 && e < E;
+        s_e[j] = ok ? e : -1;
+        s_ds[j] = ok ? dlogits[(size_t)t * E + e] : 0.f;
+    }
+    __syncthreads();
     const int row_vecs = d / N;
     const V* pv = reinterpret_cast<const V*>(dxp);
     for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
@@ -63,21 +103,24 @@ dx_kernel(const ActT* __restrict__ dxp, const int32_t* __restrict__ row_of_slot,
 #pragma unroll
         for (int i = 0; i < N; ++i) acc[i] = 0.f;
         if (dres) reinterpret_cast<const V*>(dres)[(size_t)t * row_vecs + c].unpack(acc);
+#pragma unroll 8
         for (int j = 0; j < K; ++j) {
-            const int32_t r = row_of_slot[(size_t)t * K + j];
+            const int32_t r = s_row[j];
             if (r < 0) continue;
             float f[N];
             pv[(size_t)r * row_vecs + c].unpack(f);
 #pragma unroll
             for (int i = 0; i < N; ++i) acc[i] += f[i];
         }
+#pragma unroll 4
         for (int j = 0; j < K; ++j) {
-            const int e = idx_to_int(idx[(size_t)t * K + j]);
-            if (e < 0 || e >= E) continue;
-            const float ds = dlogits[(size_t)t * E + e];
-            const WrT* wrow = w_r + (size_t)e * d + (size_t)c * N;
+            const int e = s_e[j];
+            if (e < 0) continue;
+            const float ds = s_ds[j];
+            float wv[N];
+            load_row_piece<WrT, N>(w_r + (size_t)e * d + (size_t)c * N, wv);
 #pragma unroll
-            for (int i = 0; i < N; ++i) acc[i] = fmaf(ds, to_f32<WrT>(wrow[i]), acc[i]);
+            for (int i = 0; i < N; ++i) acc[i] = fmaf(ds, wv[i], acc[i]);
         }
         V out;
         out.pack(acc);
@@ -166,7 +209,9 @@ extern "C" r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp
     if (!dxp || !row_of_slot || !slot_of_row || !offsets || !dlogits || !idx || !x || !w_router ||
         !dx || !dw_router)
         return R3_ERR_INVALID_ARG;
+    if (shape->K > r3::kDxMaxK) return R3_ERR_UNSUPPORTED;
     if (!r3::aligned(dxp, 16) || !r3::aligned(dx, 16) || !r3::aligned(dx_residual, 16) ||
+        !r3::aligned(w_router, 16) ||
         dx_residual == dx)
         return R3_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
