@@ -30,7 +30,7 @@ METRIC = "replayed-MoE-layer tokens/s (fwd+router bwd)"
 UNIT = "tokens/s"
 # kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, permute 4
 # (count, scan, rank), GEMM work lists 1, expert GEMMs 2, finish (gate + combine + dgates + dlogits) 1
-LAUNCHES_PER_STEP = 10
+LAUNCHES_PER_STEP = 8   # split_router_weight, router_tc, permute_maps_coop, permute_rows, build_work, two GEMMs, finish
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
 # from the ncu capture summarised in profiles/grouped_gemm_pair_c2_layer_bf16.md.
 GEMM_UP_DRAM_TRAFFIC_BYTES = 991.4e6   # 943.6 MB read + 47.8 MB written
@@ -462,6 +462,7 @@ def run_stack(args, w):
                      "frac": round(flop / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
                      "peak_kind": f"bf16 matmul sustained, {peaks['source']}", "traffic": None},
         # --train: per block the forward, then the forward again plus 7 backward kernels
+        # (scale_rows, build_work, two input-gradient GEMMs, swiglu_bwd, dx, dwr)
         "gpu_launches": (2 * LAUNCHES_PER_STEP + 7 if args.train else LAUNCHES_PER_STEP) * L
         * args.steps, "clocks": clocks, "peaks": peaks,
     }

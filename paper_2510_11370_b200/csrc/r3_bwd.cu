@@ -129,52 +129,58 @@ dx_kernel(const ActT* __restrict__ dxp, const int32_t* __restrict__ row_of_slot,
 }
 
 // dW_r[e, c] = sum over the rows r of expert e of ds[token(r), e] * x[token(r), c].  Grid
-// (E, blocks of 64 columns); each of the 8 warps takes the rows r = lo + warp, lo + warp + 8, ...
-// (four in flight at a time), a lane owns two columns; the 8 partial sums are added in warp order.
+// (E, blocks of 32 x N columns); each of the 8 warps takes the rows r = lo + warp, lo + warp + 8,
+// ... (four in flight at a time), a lane owns one 16-byte piece of the row; the 8 partial sums are
+// added in warp order.
 template <typename ActT>
 __global__ void __launch_bounds__(256)
 dwr_kernel(const ActT* __restrict__ x, const float* __restrict__ dlogits,
            const int32_t* __restrict__ offsets, const int32_t* __restrict__ slot_of_row,
            float* __restrict__ dw_r, int E, int K, int d) {
-    __shared__ float2 part[8][32];
+    using V = Vec16<ActT>;
+    constexpr int N = V::N;
+    __shared__ float part[8][32][N + 1];
     const int e = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int c = blockIdx.y * 64 + 2 * lane;
-    const bool in = c < d;                       // d is even
+    const int c = (blockIdx.y * 32 + lane) * N;
+    const bool in = c < d;                       // d is a multiple of 8
     const int lo = offsets[e], hi = offsets[e + 1];
-    float2 acc = make_float2(0.f, 0.f);
-    auto load = [&](int r, float& ds, float2& xv) {
-        ds = 0.f;
-        xv = make_float2(0.f, 0.f);
-        if (r < hi) {
-            const int t = slot_of_row[r] / K;
-            ds = dlogits[(size_t)t * E + e];
-            if (in) {
-                const ActT* px = x + (size_t)t * d + c;
-                xv = make_float2(to_f32<ActT>(px[0]), to_f32<ActT>(px[1]));
-            }
-        }
-    };
+    float acc[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) acc[i] = 0.f;
     for (int r = lo + warp; r < hi; r += 32) {
         float ds[4];
-        float2 xv[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) load(r + 8 * u, ds[u], xv[u]);
+        V xv[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            acc.x = fmaf(ds[u], xv[u].x, acc.x);
-            acc.y = fmaf(ds[u], xv[u].y, acc.y);
+            const int ru = r + 8 * u;
+            ds[u] = 0.f;
+            if (ru < hi) {
+                const int t = slot_of_row[ru] / K;
+                ds[u] = dlogits[(size_t)t * E + e];
+                if (in) xv[u] = *reinterpret_cast<const V*>(x + (size_t)t * d + c);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (r + 8 * u < hi && in) {
+                float f[N];
+                xv[u].unpack(f);
+#pragma unroll
+                for (int i = 0; i < N; ++i) acc[i] = fmaf(ds[u], f[i], acc[i]);
+            }
         }
     }
-    part[warp][lane] = acc;
-    __syncthreads();
-    if (warp == 0 && in) {
-        float2 sum = part[0][lane];
 #pragma unroll
-        for (int wv = 1; wv < 8; ++wv) {
-            sum.x += part[wv][lane].x;
-            sum.y += part[wv][lane].y;
+    for (int i = 0; i < N; ++i) part[warp][lane][i] = acc[i];
+    __syncthreads();
+    // thread (warp, lane) finishes column piece `lane`, elements warp, warp + 8, ... (< N)
+    if (in) {
+        for (int i = warp; i < N; i += 8) {
+            float sum = part[0][lane][i];
+#pragma unroll
+            for (int wv = 1; wv < 8; ++wv) sum += part[wv][lane][i];
+            dw_r[(size_t)e * d + c + i] = sum;
         }
-        *reinterpret_cast<float2*>(dw_r + (size_t)e * d + c) = sum;
     }
 }
 
@@ -230,7 +236,8 @@ extern "C" r3_status r3_input_grad_finish(const r3_shape* shape, const void* dxp
                 static_cast<ActT*>(dx), T, E, K, d);
     }));
     R3_DISPATCH_ACT(shape, ActT,
-        r3::dwr_kernel<ActT><<<dim3(E, (d + 63) / 64), 256, 0, cs>>>(
+        r3::dwr_kernel<ActT><<<dim3(E, (d + 32 * r3::Vec16<ActT>::N - 1) / (32 * r3::Vec16<ActT>::N)), 256, 0,
+                              cs>>>(
             static_cast<const ActT*>(x), dlogits, offsets, slot_of_row, dw_router, E, K, d));
     return r3::launch_status();
 }

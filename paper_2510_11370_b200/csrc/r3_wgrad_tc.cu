@@ -5,7 +5,7 @@
 // TMA box of 64 consecutive columns x 64 token rows lands as 64 swizzled 128-byte rows, and the
 // tcgen05 descriptors walk the rows as the k dimension.  One CTA per SM (cta_group::1), tiles of
 // 128 x 256 outputs, float32 accumulators in tensor memory (two stages, so a tile's epilogue runs
-// under the next tile's MMAs), items (problem, expert, n tile, m tile) dealt round-robin.
+// under the next tile's MMAs), items (expert, problem, n tile, m tile) dealt round-robin.
 //
 // The token count of an expert is ragged.  Rows of the last 64-row block that belong to the next
 // expert must not contribute: whole 16-row MMA steps beyond the expert's end are not issued, and
@@ -43,25 +43,27 @@ struct Problem {
     float* out;         // [E, M, N]
     int M, N;
     int mt, nt;         // tiles along M and N
-    int item0;          // first item of this problem
+    int tile0;          // first tile of this problem among an expert's tiles
 };
 struct Params {
     Problem p[MAX_PROBLEMS];
     int n_problems;
+    int tiles_per_expert;   // over all problems
     int total_items;
 };
 
 struct Item {
     int q, e, m0, n0;
 };
+// Items run expert by expert (all tiles of all problems of an expert are neighbours, so the CTAs
+// that run at the same time share that expert's operand rows in L2), then problem, n tile, m tile.
 __device__ __forceinline__ Item decode(const Params& P, int i) {
+    const int e = i / P.tiles_per_expert, t = i - e * P.tiles_per_expert;
     int q = 0;
 #pragma unroll
     for (int k = 1; k < MAX_PROBLEMS; ++k)
-        if (k < P.n_problems && i >= P.p[k].item0) q = k;
-    const int local = i - P.p[q].item0;
-    const int per_e = P.p[q].mt * P.p[q].nt;
-    const int e = local / per_e, rem = local - e * per_e;
+        if (k < P.n_problems && t >= P.p[k].tile0) q = k;
+    const int rem = t - P.p[q].tile0;
     const int n = rem / P.p[q].mt, m = rem - n * P.p[q].mt;
     return Item{q, e, m * WM, n * WN};
 }
@@ -284,7 +286,7 @@ r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, c
     const void* b_ptr[3] = {h, xp, xp};
     float* out[3] = {dw_down, dw_gate, dw_up};
     const int Ms[3] = {s->d, s->F, s->F}, Ns[3] = {s->F, s->d, s->d};
-    int items = 0;
+    int tiles = 0;
     for (int q = 0; q < 3; ++q) {
         Problem& p = P.p[q];
         if (!operand_map(&p.a, a_ptr[q], R, (uint64_t)Ms[q]) ||
@@ -295,10 +297,12 @@ r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, c
         p.N = Ns[q];
         p.mt = (Ms[q] + WM - 1) / WM;
         p.nt = (Ns[q] + WN - 1) / WN;
-        p.item0 = items;
-        items += s->E * p.mt * p.nt;
+        p.tile0 = tiles;
+        tiles += p.mt * p.nt;
     }
     P.n_problems = 3;
+    P.tiles_per_expert = tiles;
+    const int items = s->E * tiles;
     P.total_items = items;
     const int grid = items < sm_count() ? items : sm_count();
     wgrad_kernel<<<grid, THREADS, SMEM_BYTES, cs>>>(P, offsets, dev_status);
