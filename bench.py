@@ -293,7 +293,7 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     seg_ms = {n: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs)
               for i, n in enumerate(seg_names)}
-    algo_bytes = {                                  # algorithmic bytes per call (see DESIGN.md)
+    algo_bytes = {                                  # algorithmic bytes per call
         "logits": T * d * es + E * d * (2 if wk.router_w == "bf16" else 4) + T * E * 4,
         "gate_fwd": T * (E * 4 + K * 1 + K * 4),
         "permute": T * (K + d * es + K * 8 + K * d * es),

@@ -57,7 +57,7 @@ extern "C" {
 typedef enum {
     R3_OK = 0,
     R3_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, K > E, index type too narrow */
-    R3_ERR_UNSUPPORTED = 2,   /* a legal shape this build has no kernel for */
+    R3_ERR_UNSUPPORTED = 2,   /* a legal shape the library has no kernel for */
     R3_ERR_WORKSPACE = 3,     /* workspace missing, too small or misaligned */
     R3_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
     R3_ERR_SCRATCH_LIMIT = 5, /* the problem needs more than the library's fixed on-device scratch */

@@ -19,7 +19,9 @@ if not os.path.exists(_LIB_PATH):
 lib = ctypes.CDLL(_LIB_PATH)
 
 R3_OK = 0
+R3_ERR_INVALID_ARG, R3_ERR_UNSUPPORTED, R3_ERR_WORKSPACE, R3_ERR_CUDA = 1, 2, 3, 4
 R3_ERR_SCRATCH_LIMIT = 5
+R3_ERR_OUT_OF_PAGES = 6
 R3_F32, R3_BF16 = 0, 1
 R3_IDX_U8, R3_IDX_I16 = 1, 2
 DEV_OK, DEV_BAD_INDEX, DEV_DUP_INDEX, DEV_TIMEOUT = 0, 1, 2, 3

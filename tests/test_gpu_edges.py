@@ -132,3 +132,67 @@ def test_dispatch_of_more_chunks_than_fit_on_the_device_at_once(r3):
     assert np.all(np.diff(expert_of_row) >= 0)                          # grouped by expert
     same = np.diff(expert_of_row) == 0
     assert np.all(np.diff(sor // K)[same] > 0)                          # stable within an expert
+
+
+# ---- edge cases of the Update-stage backward entry points -------------------------------------
+def train_against_oracle(r3, case, tol=TOL_BF16):
+    w = case.w
+    s = r3.shape_of(w)
+    c = case.cuda()
+    st = r3.new_status("cuda")
+    y, ds, dx, dw_r, dwg, dwu, dwd = r3.replay_layer_train(
+        s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"], c["w_down"], c["dy"],
+        dev_status=st, expert_grads=True)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    args = (f64(case.x), f64(case.w_r), case.idx_np(), f32(case.w_gate), f32(case.w_up),
+            f32(case.w_down), f64(case.dy))
+    ref = O.layer_bwd_input(*args)
+    refw = O.layer_bwd_weights(*args)
+    assert rel_err(f64(y), ref["y"]) < tol and rel_err(f64(dx), ref["dx"]) < tol
+    if np.abs(ref["ds"]).max() > 0:
+        assert rel_err(f64(ds), ref["ds"]) < tol and rel_err(f64(dw_r), ref["dw_r"]) < tol
+    for k, got in enumerate((dwg, dwu, dwd)):
+        full = np.stack([refw[e][k] for e in range(w.E)])
+        assert rel_err(f64(got), full) < tol, k
+
+
+def test_backward_with_a_record_wider_than_the_fused_finish(r3):
+    """K = 12 > 8: the layer takes the four separate finishing kernels; the backward still gets
+    its gates."""
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_k12", T=150, d=128, E=16, K=12,
+                     F=64, sigma=0.3)
+    train_against_oracle(r3, Case(w))
+
+
+def test_backward_with_int16_record_and_many_experts(r3):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_wide", T=400, d=64, E=300, K=3,
+                     F=64, sigma=0.2)
+    assert w.idx_dtype == torch.int16
+    train_against_oracle(r3, Case(w))
+
+
+def test_backward_of_one_token_and_of_one_hot_expert(r3):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_one", T=1, d=128, E=16, K=4, F=64)
+    train_against_oracle(r3, Case(w))
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_hot", T=333, d=256, E=32, K=2,
+                     F=128)
+    case = Case(w)
+    case.idx = torch.tensor([[5, 17]], dtype=torch.uint8).repeat(w.T, 1)
+    train_against_oracle(r3, case)
+
+
+def test_backward_entry_points_reject_float32_and_accept_no_tokens(r3):
+    e = lambda *sh, dt=torch.bfloat16: torch.empty(sh, dtype=dt, device="cuda")
+    s0 = r3.make_shape(0, 64, 8, 2, 64)
+    ws = r3.workspace(4096, "cuda")
+    out = r3.replay_layer_train(s0, e(0, 64), e(8, 64, dt=torch.float32), e(0, 2, dt=torch.uint8),
+                                e(8, 64, 64), e(8, 64, 64), e(8, 64, 64), e(0, 64), ws=ws)
+    assert out[2].shape == (0, 64)
+    w = synth.scaled(synth.WORKLOADS["c1_tiny_fp32"], name="bwd_f32", T=16, d=64, E=8, K=2, F=64)
+    c = Case(w).cuda()
+    s = r3.shape_of(w)
+    with pytest.raises(r3.R3Error) as err:
+        r3.replay_layer_train(s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"], c["w_down"],
+                              c["dy"], ws=ws)
+    assert err.value.code == r3.R3_ERR_UNSUPPORTED
