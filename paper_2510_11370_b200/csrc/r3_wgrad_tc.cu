@@ -5,7 +5,7 @@
 // TMA box of 64 consecutive columns x 64 token rows lands as 64 swizzled 128-byte rows, and the
 // tcgen05 descriptors walk the rows as the k dimension.  One CTA per SM (cta_group::1), tiles of
 // 128 x 256 outputs, float32 accumulators in tensor memory (two stages, so a tile's epilogue runs
-// under the next tile's MMAs), items (expert, problem, n tile, m tile) dealt round-robin.
+// under the next tile's MMAs), items (expert, problem, m tile, n tile) dealt round-robin.
 //
 // The token count of an expert is ragged.  Rows of the last 64-row block that belong to the next
 // expert must not contribute: whole 16-row MMA steps beyond the expert's end are not issued, and
@@ -56,7 +56,8 @@ struct Item {
     int q, e, m0, n0;
 };
 // Items run expert by expert (all tiles of all problems of an expert are neighbours, so the CTAs
-// that run at the same time share that expert's operand rows in L2), then problem, n tile, m tile.
+// that run at the same time share that expert's operand rows in L2), then problem, m tile, n tile
+// (neighbouring CTAs write neighbouring 1 KB pieces of the same gradient rows).
 __device__ __forceinline__ Item decode(const Params& P, int i) {
     const int e = i / P.tiles_per_expert, t = i - e * P.tiles_per_expert;
     int q = 0;
@@ -64,7 +65,7 @@ __device__ __forceinline__ Item decode(const Params& P, int i) {
     for (int k = 1; k < MAX_PROBLEMS; ++k)
         if (k < P.n_problems && t >= P.p[k].tile0) q = k;
     const int rem = t - P.p[q].tile0;
-    const int n = rem / P.p[q].mt, m = rem - n * P.p[q].mt;
+    const int m = rem / P.p[q].nt, n = rem - m * P.p[q].nt;     // n fastest: neighbours fill a row
     return Item{q, e, m * WM, n * WN};
 }
 
