@@ -43,6 +43,9 @@
  *    trap, and skip the offending element.
  *  - T = 0 returns R3_OK without launching.  Experts with no rows are legal.
  *  - Results are bit-reproducible from run to run: no floating-point atomics are used anywhere.
+ *  - Host threads: the library keeps small host-side caches (encoded tensor maps, per-kernel
+ *    attributes, the helper stream).  Calls from several host threads must be serialised by the
+ *    caller; one process per GPU with one calling thread is the intended use.
  */
 #ifndef R3_H_
 #define R3_H_
