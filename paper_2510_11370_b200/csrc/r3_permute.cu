@@ -273,6 +273,142 @@ permute_maps_coop_kernel(const IdxT* __restrict__ idx, int32_t* chunk_counts, in
     }
 }
 
+// The same maps for at most kClusterMax chunks, all in ONE thread-block cluster: the per-chunk
+// counts stay in shared memory and are read across the cluster (distributed shared memory), and
+// the two grid-wide syncs become hardware cluster barriers.  CTA b owns tokens [256 b, 256 b + 256);
+// CTAs beyond the last chunk only take part in the barriers.
+constexpr int kClusterMax = 16;
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\t"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ int32_t ld_cluster_s32(const int32_t* own, uint32_t rank) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(own);
+    uint32_t ra;
+    int32_t v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+template <typename IdxT>
+__global__ void __launch_bounds__(kChunk)
+permute_maps_cluster_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ counts,
+                            int32_t* __restrict__ offsets, int32_t* __restrict__ row_of_slot,
+                            int32_t* __restrict__ slot_of_row, int T, int E, int K,
+                            int32_t* dev_status) {
+    extern __shared__ int32_t sm[];
+    int32_t* hist = sm;                                       // [E] this chunk's counts
+    int32_t* total = sm + E;                                  // [E] all chunks
+    int32_t* first = sm + 2 * E;                              // [E] first row of (expert, chunk)
+    uint32_t* bits = reinterpret_cast<uint32_t*>(sm + 3 * E); // [E][kWords]
+    __shared__ int32_t warp_sum[kChunk / 32];
+    const int lt = threadIdx.x, lane = lt & 31, warp = lt >> 5;
+    const int nb = gridDim.x, b = blockIdx.x;                 // one cluster: rank = blockIdx.x
+    const int t = b * kChunk + lt;
+    const IdxT* rec = idx + (size_t)(t < T ? t : 0) * K;
+
+    for (int e = lt; e < E; e += kChunk) hist[e] = 0;
+    for (int i = lt; i < E * kWords; i += kChunk) bits[i] = 0u;
+    __syncthreads();
+    int kept[8];                                   // slots 0..7: the expert, or -1 for a dropped pair
+#pragma unroll
+    for (int u = 0; u < 8; ++u) kept[u] = -1;
+    if (t < T) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            int e;
+            if (u < K && pair_ok(rec, u, E, e, dev_status)) {
+                kept[u] = e;
+                atomicAdd(&hist[e], 1);
+                atomicOr(&bits[e * kWords + (lt >> 5)], 1u << (lt & 31));
+            }
+        }
+        for (int j = 8; j < K; ++j) {
+            int e;
+            if (pair_ok(rec, j, E, e, dev_status)) {
+                atomicAdd(&hist[e], 1);
+                atomicOr(&bits[e * kWords + (lt >> 5)], 1u << (lt & 31));
+            }
+        }
+    }
+    cluster_barrier();                      // every chunk's counts are final and visible
+
+    for (int e = lt; e < E; e += kChunk) {
+        int32_t v[kClusterMax];
+#pragma unroll
+        for (int c = 0; c < kClusterMax; ++c)                 // all loads in flight together
+            v[c] = c < nb ? ld_cluster_s32(hist + e, (uint32_t)c) : 0;
+        int32_t before = 0, all = 0;
+#pragma unroll
+        for (int c = 0; c < kClusterMax; ++c) {
+            all += v[c];
+            if (c < b) before += v[c];
+        }
+        total[e] = all;
+        first[e] = before;
+    }
+    __syncthreads();
+    cluster_barrier();                      // nobody reads this CTA's counts after this point
+
+    // offsets: each thread owns a run of experts
+    const int per = (E + kChunk - 1) / kChunk;
+    int32_t mine = 0;
+    for (int i = 0; i < per; ++i) {
+        const int e = lt * per + i;
+        if (e < E) mine += total[e];
+    }
+    int32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_sum[warp] = inc;
+    __syncthreads();
+    int32_t run = inc - mine;
+    for (int w = 0; w < warp; ++w) run += warp_sum[w];
+    for (int i = 0; i < per; ++i) {
+        const int e = lt * per + i;
+        if (e < E) {
+            const int32_t cnt = total[e];
+            first[e] += run;                               // expert offset + rows of earlier chunks
+            if (b == 0) {
+                offsets[e] = run;
+                counts[e] = cnt;
+                if (e == E - 1) offsets[E] = run + cnt;
+            }
+            run += cnt;
+        }
+    }
+    __syncthreads();
+    if (t < T) {
+        for (int j0 = 0; j0 < K; j0 += 8) {
+            int32_t row[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                int e = kept[u];
+                row[u] = -1;
+                if (j < K && (j0 == 0 ? e >= 0 : pair_ok(rec, j, E, e, nullptr))) {
+                    const uint32_t* m = bits + e * kWords;
+                    int rank = __popc(m[lt >> 5] & ((1u << (lt & 31)) - 1u));
+                    for (int w = 0; w < (lt >> 5); ++w) rank += __popc(m[w]);
+                    row[u] = first[e] + rank;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u;
+                if (j < K) {
+                    if (row[u] >= 0) slot_of_row[row[u]] = t * K + j;
+                    row_of_slot[(size_t)t * K + j] = row[u];
+                }
+            }
+        }
+    }
+}
+
 // One warp per token: read x[t] once (16-byte pieces), write it to the token's K rows.
 template <int VEC_BYTES>
 __global__ void __launch_bounds__(256)
@@ -391,9 +527,55 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
     const int T = shape->T, E = shape->E, K = shape->K;
     const int NB = (T + r3::kChunk - 1) / r3::kChunk;
     int32_t* chunk_counts = static_cast<int32_t*>(workspace);
-    // one cooperative launch when all the chunk CTAs can be resident together
+    // up to 16 chunks: one thread-block cluster, counts exchanged through shared memory
     bool coop_done = false;
-    {
+    if (NB <= r3::kClusterMax) {
+        int cl = 1;
+        while (cl < NB) cl <<= 1;
+        const size_t smem = (size_t)E * (3 + r3::kWords) * sizeof(int32_t);
+        static int usable[2][r3::kClusterMax + 1] = {};        // per index type and cluster size
+        const int ti = shape->idx_type == R3_IDX_U8 ? 0 : 1;   // 0 = untested, 1 = ok, -1 = no
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cl;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3((unsigned)cl);
+        cfg.blockDim = dim3(r3::kChunk);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = cs;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (usable[ti][cl] == 0) {
+            usable[ti][cl] = -1;
+            if (smem <= 200 * 1024) {
+                cudaError_t a1 = cudaErrorUnknown, a2 = cudaErrorUnknown, q = cudaErrorUnknown;
+                int n = 0;
+                R3_DISPATCH_IDX(shape, IdxT, {
+                    auto kern = r3::permute_maps_cluster_kernel<IdxT>;
+                    a1 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              200 * 1024);
+                    a2 = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+                    q = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+                });
+                if (a1 == cudaSuccess && a2 == cudaSuccess && q == cudaSuccess && n >= 1)
+                    usable[ti][cl] = 1;
+                else
+                    cudaGetLastError();
+            }
+        }
+        if (usable[ti][cl] == 1) {
+            cudaError_t le = cudaErrorUnknown;
+            R3_DISPATCH_IDX(shape, IdxT, le = cudaLaunchKernelEx(
+                &cfg, r3::permute_maps_cluster_kernel<IdxT>, static_cast<const IdxT*>(idx), counts,
+                offsets, row_of_slot, slot_of_row, T, E, K, dev_status));
+            if (le != cudaSuccess) return R3_ERR_CUDA;
+            coop_done = true;
+        }
+    }
+    // one cooperative launch when all the chunk CTAs can be resident together
+    if (!coop_done) {
         const size_t smem = (size_t)E * (1 + r3::kWords) * sizeof(int32_t);
         int per_sm = 0;
         cudaError_t qe = cudaErrorUnknown;
