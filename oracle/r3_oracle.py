@@ -386,14 +386,15 @@ def layer_bwd_weights(x, w_r, idx_infer, w_gate, w_up, w_down, dy, experts=None)
 # ----------------------------------------------------------------------------------------------
 # The exact backward chain of a stack of residual replayed blocks (benchmark configuration 5)
 # ----------------------------------------------------------------------------------------------
-def replay_stack_bwd_tokens(x_rows, layers, dy_rows, store=None):
+def replay_stack_bwd_tokens(x_rows, layers, dy_rows, store=None, expert_grads=False):
     """x_{l+1} = store(x_l + y_replay,l(x_l)) for L blocks, then the gradient of
     <dy, x_L> back through every block with the recorded masks held constant:
         g_L = dy,   g_l = store(g_{l+1} + dx_l(g_{l+1}))
     where dx_l, ds_l, dW_r,l are layer_bwd_input of block l at its input x_l with upstream
     gradient g_{l+1} (the residual path carries g_{l+1} unchanged).  Tokens are independent, so a
     subset can be followed on its own; dW_r,l then holds the sum over these tokens only.
-    Returns dict(x_out, dx0, ds=[...], dw_r=[...]) with one entry per block."""
+    With expert_grads, dw_experts[l] = layer_bwd_weights of block l at (x_l, g_{l+1}).
+    Returns dict(x_out, dx0, ds=[...], dw_r=[...], dw_experts=[...]) with one entry per block."""
     x = _f64(x_rows)
     xs = []
     for (w_r, idx_rows, w_gate, w_up, w_down) in layers:
@@ -404,12 +405,14 @@ def replay_stack_bwd_tokens(x_rows, layers, dy_rows, store=None):
         if store is not None:
             x = _f64(store(x))
     g = _f64(dy_rows)
-    dss, dwrs = [None] * len(layers), [None] * len(layers)
+    dss, dwrs, dwes = [None] * len(layers), [None] * len(layers), [None] * len(layers)
     for l in range(len(layers) - 1, -1, -1):
         w_r, idx_rows, w_gate, w_up, w_down = layers[l]
         res = layer_bwd_input(xs[l], w_r, idx_rows, w_gate, w_up, w_down, g)
         dss[l], dwrs[l] = res["ds"], res["dw_r"]
+        if expert_grads:
+            dwes[l] = layer_bwd_weights(xs[l], w_r, idx_rows, w_gate, w_up, w_down, g)
         g = g + res["dx"]
         if store is not None:
             g = _f64(store(g))
-    return dict(x_out=x, dx0=g, ds=dss, dw_r=dwrs)
+    return dict(x_out=x, dx0=g, ds=dss, dw_r=dwrs, dw_experts=dwes)

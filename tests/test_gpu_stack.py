@@ -206,7 +206,8 @@ def check_stack_train(r3, w, L, sel, tol, expert_grads=False):
     idx_np = idx.cpu().to(torch.int64).numpy()
     layers = [(f64(w_r[l]), idx_np[l][sel], LayerExperts(wg, l), LayerExperts(wu, l),
                LayerExperts(wd, l)) for l in range(L)]
-    ref = O.replay_stack_bwd_tokens(f64(x0)[sel], layers, f64(dy)[sel], store=bf16_store)
+    ref = O.replay_stack_bwd_tokens(f64(x0)[sel], layers, f64(dy)[sel], store=bf16_store,
+                                    expert_grads=expert_grads and len(sel) == w.T)
     # stored activations and gradients pass through L bf16 roundings (see check_stack)
     tol_chain = tol + np.sqrt(L) * 2.0 ** -8
     err = lambda got, want: float(np.abs(got - want).max() / np.abs(want).max())
@@ -217,6 +218,11 @@ def check_stack_train(r3, w, L, sel, tol, expert_grads=False):
     if len(sel) == w.T:
         for l in range(L):
             assert err(f64(dw_r[l]), ref["dw_r"][l]) < tol_chain, l
+        if expert_grads:
+            for l in range(L):
+                for k in range(3):
+                    want = np.stack([ref["dw_experts"][l][e][k] for e in range(w.E)])
+                    assert err(f64(out[4 + k][l]), want) < tol_chain, (l, k)
     # the forward half is r3_replay_stack's; a second run repeats the first bit for bit
     x_fwd, _ = r3.replay_stack(s, L, x0, w_r, idx, wg, wu, wd, dy)
     assert torch.equal(x_fwd, x_out)
@@ -229,6 +235,12 @@ def test_small_stack_exact_backward_chain(r3):
     w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="stack_bwd", T=300, d=256, E=16,
                      K=4, F=128)
     check_stack_train(r3, w, 3, np.arange(300), 2e-2)
+
+
+def test_small_stack_exact_backward_chain_with_expert_weight_gradients(r3):
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="stack_bwd_w", T=260, d=128, E=8,
+                     K=2, F=136)
+    check_stack_train(r3, w, 3, np.arange(260), 2e-2, expert_grads=True)
 
 
 def test_one_block_stack_train_is_layer_train_plus_identity_path(r3):

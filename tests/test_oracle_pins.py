@@ -587,3 +587,23 @@ def test_stack_backward_special_cases():
     dead = [(w, i, a, b, np.zeros_like(c)) for (w, i, a, b, c) in layers]
     z = O.replay_stack_bwd_tokens(x0, dead, dy)
     assert np.array_equal(z["dx0"], dy) and all(np.all(s == 0) for s in z["ds"])
+
+
+def test_stack_expert_weight_gradients_match_central_differences():
+    """A weight of the FIRST block's experts reaches the loss through every later block."""
+    x0, layers, dy = _tiny_stack(60, L=2, T=4, d=4, E=3, K=2, F=3)
+    got = O.replay_stack_bwd_tokens(x0, layers, dy, expert_grads=True)
+    h = 1e-6
+    for which in range(3):
+        target = layers[0][2 + which]
+        num = np.zeros_like(target)
+        for pos in np.ndindex(*target.shape):
+            keep = target[pos]
+            target[pos] = keep + h
+            up = _stack_loss(x0, layers, dy)
+            target[pos] = keep - h
+            dn = _stack_loss(x0, layers, dy)
+            target[pos] = keep
+            num[pos] = (up - dn) / (2 * h)
+        mine = np.stack([got["dw_experts"][0][e][which] for e in range(target.shape[0])])
+        assert np.abs(mine - num).max() / np.abs(num).max() < 1e-6
