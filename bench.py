@@ -561,6 +561,78 @@ def run_train(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_ep(args, w):
+    """Expert-parallel replayed layer (tokens AND experts split over the ranks): every rank holds
+    E/N experts and routes w.T tokens of its own; two all-to-alls of rows per layer.  With one
+    rank the collectives are still made (NCCL, world size 1)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2510_11370_b200 import build, dist as r3dist, synth
+    build.build()
+    from paper_2510_11370_b200 import r3
+    from paper_2510_11370_b200.ep import EpRank, ep_replay_layer
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    rank, world = r3dist.env_rank_world()
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world)
+    peaks = load_peaks()
+    wk = synth.scaled(w, seed=w.seed + rank)
+    T, K, E, d, F = wk.T, wk.K, wk.E, wk.d, wk.F
+    el = E // world
+    x = synth.activations(wk, dev)
+    dy = synth.upstream_grad(wk, dev)
+    w_r = synth.router_weight(w, dev)                    # replicated: same seed on every rank
+    wg, wu, wd = (t[rank * el:(rank + 1) * el].contiguous() for t in synth.expert_weights(w, dev))
+    s = r3.shape_of(wk)
+    _, lg = r3.capture_topk_ws(s, 1, x, w_r, want_idx=False, want_logits=True)
+    idx = synth.make_record(wk, lg)
+    state = EpRank(rank, world, T, d, E, K, F)
+
+    def step():
+        return ep_replay_layer(state, x, w_r, idx, wg, wu, wd, dy)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    t1 = time.time()
+    ms_total = r3dist.max_over_ranks(e0.elapsed_time(e1), dev)
+    assert state.status.item() == 0
+    if rank == 0:
+        clocks = sampler.stop(t0, t1)
+        ms = ms_total / args.steps
+        line = {
+            "metric": METRIC, "value": world * T / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": wk.name, "mode": "expert parallel: E/N experts and T tokens per "
+                       "rank, NCCL all-to-all of rows (torch.distributed) there and back, one host "
+                       "synchronisation per layer for the split sizes", "T_per_gpu": T, "d": d,
+                       "E": E, "K": K, "F": F},
+            "clocks": clocks, "peaks": peaks,
+        }
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 def run_capture(args, w):
     """Config 4, inference side: router logits + TopKMask of a decode batch for `w.layers` layers
     in one launch (r3_capture_topk_batched), records packed as uint8."""
@@ -708,6 +780,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stack", action="store_true",
                     help="with a multi-layer workload (c5_stack48): time all its blocks, weights resident")
+    ap.add_argument("--ep", action="store_true",
+                    help="expert-parallel layer: experts split over the ranks, all-to-all of rows")
     ap.add_argument("--train", action="store_true",
                     help="time forward + the whole backward of one layer (bf16 workloads)")
     args = ap.parse_args()
@@ -717,6 +791,8 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.impl != "reference" and args.workload == "c4_capture":
         return run_capture(args, w)
+    if args.impl != "reference" and args.ep:
+        return run_ep(args, w)
     if args.impl != "reference" and w.layers > 1 and args.stack:
         return run_stack(args, w)
     if args.impl != "reference" and args.train:

@@ -385,6 +385,29 @@ r3_status r3_replay_stack_train(const r3_shape* shape, int32_t L, const void* x0
                                 float* dw_up, float* dw_down, void* workspace, size_t ws_bytes,
                                 int32_t* dev_status, void* stream);
 
+/* ---- expert parallelism: bookkeeping of the row exchange (an extension; the paper describes
+ * no parallelism) ------------------------------------------------------------------------------
+ *
+ * With the E experts split over N ranks (rank q owns the experts [q E/N, (q+1) E/N)) every rank
+ * runs r3_permute on its own tokens with GLOBAL expert numbers; the grouped rows bound for one rank
+ * are then a contiguous block, the blocks are exchanged with an all-to-all (the caller's:
+ * torch.distributed / NCCL), and the receiver holds [source rank][local expert][row].  The library
+ * supplies the reordering into the [local expert][source rank][row] order that r3_grouped_swiglu
+ * takes (with T = received rows, K = 1, E = E/N), and its inverse for the way back.
+ *
+ * r3_ep_regroup_map: recv_counts [n_src, e_local] int32 = rows received from each source for each
+ * local expert; rows = their sum (known to the host from the split sizes; a table that does not
+ * add up to it sets dev_status and writes nothing).  Writes perm [rows] (position in the new
+ * order -> arrival index) and offsets [e_local + 1] (first row of each local expert in the new
+ * order).  n_src * e_local <= 4096 (R3_ERR_UNSUPPORTED beyond).
+ * r3_ep_move_rows: inverse = 0: dst[j] = src[perm[j]];  inverse = 1: dst[perm[j]] = src[j], for
+ * rows of row_bytes bytes (a multiple of 16).  src and dst must not be the same buffer. */
+r3_status r3_ep_regroup_map(const int32_t* recv_counts, int32_t n_src, int32_t e_local,
+                            int32_t rows, int32_t* perm, int32_t* offsets, int32_t* dev_status,
+                            void* stream);
+r3_status r3_ep_move_rows(const void* src, void* dst, const int32_t* perm, int32_t rows,
+                          size_t row_bytes, int32_t inverse, void* stream);
+
 /* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */
 
 /* Eq. (kl), the k3 estimate of KL(pi_train || pi_infer), and Eq. (etdf), the Extreme Token

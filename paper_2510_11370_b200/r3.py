@@ -42,6 +42,7 @@ EXPORTS = [
     "r3_grouped_swiglu_bwd", "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
     "r3_replay_layer_train_workspace_bytes", "r3_replay_layer_train",
     "r3_replay_stack_train_workspace_bytes", "r3_replay_stack_train",
+    "r3_ep_regroup_map", "r3_ep_move_rows",
     "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
     "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
@@ -66,6 +67,8 @@ lib.r3_replay_layer_train.argtypes = [_SP] + [_P] * 15 + [ctypes.c_size_t, _P, _
 lib.r3_replay_stack_train_workspace_bytes.restype = ctypes.c_size_t
 lib.r3_replay_stack_train_workspace_bytes.argtypes = [_SP, ctypes.c_int32]
 lib.r3_replay_stack_train.argtypes = [_SP, ctypes.c_int32] + [_P] * 15 + [ctypes.c_size_t, _P, _P]
+lib.r3_ep_regroup_map.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _P, _P, _P, _P]
+lib.r3_ep_move_rows.argtypes = [_P, _P, _P, ctypes.c_int32, ctypes.c_size_t, ctypes.c_int32, _P]
 lib.r3_grouped_swiglu_bwd.argtypes = [_SP] + [_P] * 13 + [ctypes.c_size_t, _P, _P]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
            "r3_grouped_swiglu_bwd_workspace_bytes", "r3_replay_layer_train_workspace_bytes",
@@ -673,6 +676,29 @@ def replay_stack_train(s: Shape, L, x0, w_router, idx, w_gate, w_up, w_down, dy,
     if expert_grads:
         return (x_out, dlogits, dx0, dw_r) + dws
     return x_out, dlogits, dx0, dw_r
+
+
+def ep_regroup_map(recv_counts, rows: int, *, dev_status=None, stream=None):
+    """recv_counts [n_src, e_local] int32 (device) -> (perm [rows] int32, offsets [e_local+1])."""
+    n_src, e_local = recv_counts.shape
+    dev = _dev(recv_counts)
+    perm = torch.empty(max(rows, 1), dtype=torch.int32, device=dev)[:rows]
+    offsets = torch.empty(e_local + 1, dtype=torch.int32, device=dev)
+    _check(lib.r3_ep_regroup_map(_ptr(recv_counts), n_src, e_local, rows,
+                                 _ptr(perm) if rows else None, _ptr(offsets), _ptr(dev_status),
+                                 _stream(stream)))
+    return perm, offsets
+
+
+def ep_move_rows(src, perm, *, inverse=False, stream=None):
+    """Rows of `src` [rows, width] reordered by `perm` (see r3_ep_move_rows)."""
+    dst = torch.empty_like(src)
+    rows = src.shape[0]
+    if rows:
+        _check(lib.r3_ep_move_rows(_ptr(src), _ptr(dst), _ptr(perm), rows,
+                                   src.shape[1] * src.element_size(), 1 if inverse else 0,
+                                   _stream(stream)))
+    return dst
 
 
 def grouped_swiglu_bwd_input(s: Shape, dout, pre_gate, pre_up, offsets, w_gate, w_up, w_down,
