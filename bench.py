@@ -239,6 +239,19 @@ def run_ours(args, w):
     ms_per_step = ms_total / args.steps
     value = world * T * args.steps / (ms_total * 1e-3)
 
+    # ---- the same step timed one by one (outside the contract's K-step region): best and median -
+    n_single = min(max(args.steps, 20), 100)
+    single = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(n_single)]
+    for a, b in single:
+        a.record()
+        step()
+        b.record()
+    torch.cuda.synchronize()
+    single_ms = sorted(a.elapsed_time(b) for a, b in single)
+    per_step = {"best_ms": round(single_ms[0], 5), "median_ms": round(statistics.median(single_ms), 5),
+                "steps": n_single}
+
     # ---- per-kernel segments (same kernels through the per-step entry points, events between) --
     seg_names = ["logits", "gate_fwd", "permute", "expert_up_swiglu", "expert_down", "combine",
                  "dgates", "gate_bwd", "finish_fused", "permute_maps", "experts_gather"]
@@ -375,7 +388,7 @@ def run_ours(args, w):
                              "the 126 MB L2 every step" % (synth.layer_bytes(wk) / 1e9)},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
-            "kernels": kernels, "peaks": peaks,
+            "per_step": per_step, "kernels": kernels, "peaks": peaks,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
