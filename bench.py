@@ -239,6 +239,17 @@ def run_ours(args, w):
     ms_per_step = ms_total / args.steps
     value = world * T * args.steps / (ms_total * 1e-3)
 
+    def checksum(t):
+        """64-bit wrap-around sum of the tensor's raw 16/32/8-bit words."""
+        raw = t.contiguous().view(torch.int16 if t.element_size() == 2 else
+                                  torch.int32 if t.element_size() == 4 else torch.uint8)
+        return int(raw.to(torch.int64).sum().item())
+
+    inputs = {"torch": torch.__version__, "seed": wk.seed,
+              "checksums": {"x": checksum(x), "dy": checksum(dy), "w_router": checksum(w_r),
+                            "w_gate": checksum(wg), "w_up": checksum(wu), "w_down": checksum(wd),
+                            "record": checksum(idx)}}
+
     # ---- the same step timed one by one (outside the contract's K-step region): best and median -
     n_single = min(max(args.steps, 20), 100)
     single = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -388,7 +399,7 @@ def run_ours(args, w):
                              "the 126 MB L2 every step" % (synth.layer_bytes(wk) / 1e9)},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
-            "per_step": per_step, "kernels": kernels, "peaks": peaks,
+            "per_step": per_step, "inputs": inputs, "kernels": kernels, "peaks": peaks,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
