@@ -68,3 +68,22 @@ def ungroup_rows(rows, recv_counts):
     out = np.empty_like(np.asarray(rows))
     out[perm] = rows
     return out
+
+
+def dest_table(counts_all, me):
+    """counts_all [N][E].  For rank `me`: dst_base[e] = row, in the owner's
+    [local expert][source][row] buffer, of this rank's first row of expert e (rows of the owner's
+    earlier experts from every source, then the rows of expert e from the sources before `me`);
+    offsets_local [E/N + 1] = first row of each of `me`'s own experts in its buffer."""
+    counts = np.asarray(counts_all, dtype=np.int64)
+    n, e_total = counts.shape
+    el = e_total // n
+    dst_base = []
+    for e in range(e_total):
+        q, k = divmod(e, el)
+        before = sum(int(counts[s, q * el + k2]) for k2 in range(k) for s in range(n))
+        dst_base.append(before + sum(int(counts[s, e]) for s in range(me)))
+    offsets_local = [0]
+    for k in range(el):
+        offsets_local.append(offsets_local[-1] + sum(int(counts[s, me * el + k]) for s in range(n)))
+    return np.asarray(dst_base, dtype=np.int64), np.asarray(offsets_local, dtype=np.int64)

@@ -54,3 +54,24 @@ def test_regroup_special_cases():
     # no rows at all
     got, offsets = EP.regroup_rows(np.zeros((0, 2)), np.zeros((2, 3), dtype=int))
     assert got.shape == (0, 2) and list(offsets) == [0, 0, 0, 0]
+
+
+def test_dest_table_agrees_with_the_regrouped_order():
+    """Writing every source's block straight to dst_base must give the buffer that exchanging
+    and regrouping gives."""
+    n, e_total = 3, 6
+    counts = _counts(9, n, e_total)
+    el = e_total // n
+    for q in range(n):                                   # owner
+        rc = np.array([[counts[s, q * el + k] for k in range(el)] for s in range(n)])
+        # rows tagged (source, expert, i), in arrival order [source][expert][row]
+        tags = [(s, k, i) for s in range(n) for k in range(el) for i in range(rc[s, k])]
+        regrouped, offsets = EP.regroup_rows(np.array(tags).reshape(-1, 3), rc)
+        direct = np.full((len(tags), 3), -1)
+        for s in range(n):                               # every source writes its own rows
+            dst_base, _ = EP.dest_table(counts, s)
+            for k in range(el):
+                for i in range(rc[s, k]):
+                    direct[dst_base[q * el + k] + i] = (s, k, i)
+        assert np.array_equal(direct, regrouped)
+        assert np.array_equal(EP.dest_table(counts, q)[1], offsets)
