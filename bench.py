@@ -598,7 +598,8 @@ def run_ep(args, w):
     from paper_2510_11370_b200 import build, dist as r3dist, synth
     build.build()
     from paper_2510_11370_b200 import r3
-    from paper_2510_11370_b200.ep import EpRank, ep_replay_layer
+    from paper_2510_11370_b200.ep import (EpDirectRank, EpRank, PeerBuffers, ep_replay_layer,
+                                          ep_replay_layer_direct)
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
@@ -606,7 +607,7 @@ def run_ep(args, w):
     if not dist.is_initialized():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29533")
-        dist.init_process_group("nccl", rank=rank, world_size=world)
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
     peaks = load_peaks()
     wk = synth.scaled(w, seed=w.seed + rank)
     T, K, E, d, F = wk.T, wk.K, wk.E, wk.d, wk.F
@@ -618,10 +619,19 @@ def run_ep(args, w):
     s = r3.shape_of(wk)
     _, lg = r3.capture_topk_ws(s, 1, x, w_r, want_idx=False, want_logits=True)
     idx = synth.make_record(wk, lg)
-    state = EpRank(rank, world, T, d, E, K, F)
+    if args.ep_direct:
+        # rows written straight into the owners' buffers (symmetric memory), outputs pulled by
+        # address; capacity for the worst case (every row of every rank to one owner)
+        state = EpDirectRank(rank, world, T, d, E, K, F)
+        bufs = PeerBuffers.symmetric(world * T * K, d, wk.act_dtype, dev)
 
-    def step():
-        return ep_replay_layer(state, x, w_r, idx, wg, wu, wd, dy)
+        def step():
+            return ep_replay_layer_direct(state, bufs, x, w_r, idx, wg, wu, wd, dy)
+    else:
+        state = EpRank(rank, world, T, d, E, K, F)
+
+        def step():
+            return ep_replay_layer(state, x, w_r, idx, wg, wu, wd, dy)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -651,9 +661,14 @@ def run_ep(args, w):
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": wk.name, "mode": "expert parallel: E/N experts and T tokens per "
+            "config": {"workload": wk.name, "mode": (
+                       "expert parallel, direct form: E/N experts and T tokens per rank, rows "
+                       "written straight into the owners' symmetric-memory buffers, outputs pulled "
+                       "by address, all-gather of the counts and three barriers per layer"
+                       if args.ep_direct else
+                       "expert parallel: E/N experts and T tokens per "
                        "rank, NCCL all-to-all of rows (torch.distributed) there and back, one host "
-                       "synchronisation per layer for the split sizes", "T_per_gpu": T, "d": d,
+                       "synchronisation per layer for the split sizes"), "T_per_gpu": T, "d": d,
                        "E": E, "K": K, "F": F},
             "clocks": clocks, "peaks": peaks,
         }
@@ -810,6 +825,8 @@ def main():
                     help="with a multi-layer workload (c5_stack48): time all its blocks, weights resident")
     ap.add_argument("--ep", action="store_true",
                     help="expert-parallel layer: experts split over the ranks, all-to-all of rows")
+    ap.add_argument("--ep-direct", action="store_true",
+                    help="expert-parallel layer, rows written straight into the owners' buffers")
     ap.add_argument("--train", action="store_true",
                     help="time forward + the whole backward of one layer (bf16 workloads)")
     args = ap.parse_args()
@@ -819,7 +836,7 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.impl != "reference" and args.workload == "c4_capture":
         return run_capture(args, w)
-    if args.impl != "reference" and args.ep:
+    if args.impl != "reference" and (args.ep or args.ep_direct):
         return run_ep(args, w)
     if args.impl != "reference" and w.layers > 1 and args.stack:
         return run_stack(args, w)

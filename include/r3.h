@@ -408,6 +408,41 @@ r3_status r3_ep_regroup_map(const int32_t* recv_counts, int32_t n_src, int32_t e
 r3_status r3_ep_move_rows(const void* src, void* dst, const int32_t* perm, int32_t rows,
                           size_t row_bytes, int32_t inverse, void* stream);
 
+/* The same exchange without a collective for the rows: every rank writes its rows straight
+ * into the owners' buffers (plain stores to memory this GPU can address: its own, or a peer's
+ * mapped with peer access / symmetric memory, over NVLink), at the place they have in the owner's
+ * [local expert][source][row] order, and later fetches the expert outputs of its rows from the
+ * owners' output buffers by address.  No multicast load is involved anywhere.
+ *
+ * r3_ep_dest_table: counts_all [n_ranks, E] int32 (device; the ranks' `counts` of r3_permute after
+ * an all-gather).  Writes dst_base [E] (row, in the owner's buffer, of THIS rank's first row of
+ * every expert) and offsets_local [E / n_ranks + 1] (the offsets r3_grouped_swiglu takes for this
+ * rank's own experts).  n_ranks <= 64.
+ * r3_ep_dispatch_rows: copies x[t] to its K places; idx, row_of_slot and my_offsets (= offsets) are
+ * those of this rank's r3_permute (called without x); peer_buffers_host [n_ranks] is a HOST array
+ * of device addresses, entry q = base of rank q's receive buffer [rows_q, d].  The owners must
+ * not read the buffers before every rank's call has completed (a barrier of the job's own).
+ * r3_ep_slot_rows: row_ptr [T, K] (device, 64-bit addresses) = where the expert-output row of each
+ * (token, slot) pair will stand in the owners' OUTPUT buffers (peer_buffers_host: their bases);
+ * 0 for a pair that r3_permute dropped.
+ * r3_replay_finish_rows: r3_replay_finish with the rows given by address (row_ptr) instead of
+ * (o, row_of_slot).  K <= 8 and the rows of one token must fit in shared memory
+ * ((K + 2) d elements, else R3_ERR_UNSUPPORTED). */
+r3_status r3_ep_dest_table(const int32_t* counts_all, int32_t n_ranks, int32_t E, int32_t rank,
+                           int32_t* dst_base, int32_t* offsets_local, void* stream);
+r3_status r3_ep_dispatch_rows(const r3_shape* shape, int32_t n_ranks, const void* x,
+                              const void* idx, const int32_t* row_of_slot,
+                              const int32_t* my_offsets, const int32_t* dst_base,
+                              const unsigned long long* peer_buffers_host, void* stream);
+r3_status r3_ep_slot_rows(const r3_shape* shape, int32_t n_ranks, const void* idx,
+                          const int32_t* row_of_slot, const int32_t* my_offsets,
+                          const int32_t* dst_base, const unsigned long long* peer_buffers_host,
+                          unsigned long long* row_ptr, void* stream);
+r3_status r3_replay_finish_rows(const r3_shape* shape, const float* logits, const void* idx,
+                                const unsigned long long* row_ptr, const void* dy,
+                                const void* residual, void* y, float* gates_out, float* dlogits,
+                                int32_t* dev_status, void* stream);
+
 /* ---- training/inference discrepancy measures (Sections 3.1 and 3.2) -------------------------- */
 
 /* Eq. (kl), the k3 estimate of KL(pi_train || pi_infer), and Eq. (etdf), the Extreme Token

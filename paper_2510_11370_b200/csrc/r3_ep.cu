@@ -70,6 +70,145 @@ ep_move_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
 
 }  // namespace r3
 
+namespace r3 {
+
+constexpr int kEpMaxRanks = 64;
+struct EpPeers {
+    unsigned long long base[kEpMaxRanks];   // one buffer address per rank
+};
+
+// One CTA.  counts_all [n][E] = rows of every expert on every rank (after an all-gather).  For
+// rank `me`:  dst_base[e] = row, in the owner's [local expert][source][row] buffer, of this
+// rank's first row of expert e;  offsets_local [el + 1] = first row of each of this rank's own
+// experts in that buffer (what the grouped GEMM of this rank takes).
+__global__ void __launch_bounds__(1024)
+ep_dest_table_kernel(const int32_t* __restrict__ counts_all, int n, int E, int me,
+                     int32_t* __restrict__ dst_base, int32_t* __restrict__ offsets_local) {
+    const int el = E / n;
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+        const int q = e / el, k = e - q * el;
+        int32_t before = 0;                       // rows of the owner's earlier experts, all sources
+        for (int k2 = 0; k2 < k; ++k2)
+            for (int s = 0; s < n; ++s) before += counts_all[s * E + q * el + k2];
+        int32_t mine = before;
+        for (int s = 0; s < me; ++s) mine += counts_all[s * E + e];
+        dst_base[e] = mine;
+        if (q == me) {
+            offsets_local[k] = before;
+            if (k == el - 1) {
+                int32_t total = before;
+                for (int s = 0; s < n; ++s) total += counts_all[s * E + e];
+                offsets_local[el] = total;
+            }
+        }
+    }
+}
+
+// One warp per token: x[t] goes straight to its K places in the owners' expert-major buffers.
+template <typename IdxT>
+__global__ void __launch_bounds__(256)
+ep_dispatch_rows_kernel(const uint4* __restrict__ x, const IdxT* __restrict__ idx,
+                        const int32_t* __restrict__ row_of_slot,
+                        const int32_t* __restrict__ my_offsets,
+                        const int32_t* __restrict__ dst_base, const __grid_constant__ EpPeers peers,
+                        int T, int E, int K, int el, int row_vecs) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const uint4* src = x + (size_t)t * row_vecs;
+    for (int j = 0; j < K; ++j) {
+        const int32_t r = row_of_slot[(size_t)t * K + j];
+        if (r < 0) continue;
+        const int e = idx_to_int(idx[(size_t)t * K + j]);
+        const size_t row = (size_t)dst_base[e] + (size_t)(r - my_offsets[e]);
+        uint4* dst = reinterpret_cast<uint4*>(peers.base[e / el]) + row * row_vecs;
+        for (int c = lane; c < row_vecs; c += 32) dst[c] = src[c];
+    }
+}
+
+// Address of the expert-output row of every (token, slot) pair in the owners' output buffers.
+template <typename IdxT>
+__global__ void __launch_bounds__(256)
+ep_slot_rows_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ row_of_slot,
+                    const int32_t* __restrict__ my_offsets, const int32_t* __restrict__ dst_base,
+                    const __grid_constant__ EpPeers peers, unsigned long long* __restrict__ row_ptr,
+                    long long pairs, int el, unsigned long long row_bytes) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= pairs) return;
+    const int32_t r = row_of_slot[i];
+    unsigned long long p = 0;
+    if (r >= 0) {
+        const int e = idx_to_int(idx[i]);
+        p = peers.base[e / el] + ((unsigned long long)dst_base[e] + (r - my_offsets[e])) * row_bytes;
+    }
+    row_ptr[i] = p;
+}
+
+}  // namespace r3
+
+extern "C" r3_status r3_ep_dest_table(const int32_t* counts_all, int32_t n_ranks, int32_t E,
+                                      int32_t rank, int32_t* dst_base, int32_t* offsets_local,
+                                      void* stream) {
+    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || E <= 0 || E % n_ranks || rank < 0 ||
+        rank >= n_ranks || !counts_all || !dst_base || !offsets_local)
+        return R3_ERR_INVALID_ARG;
+    r3::ep_dest_table_kernel<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(
+        counts_all, n_ranks, E, rank, dst_base, offsets_local);
+    return r3::launch_status();
+}
+
+extern "C" r3_status r3_ep_dispatch_rows(const r3_shape* shape, int32_t n_ranks, const void* x,
+                                         const void* idx, const int32_t* row_of_slot,
+                                         const int32_t* my_offsets, const int32_t* dst_base,
+                                         const unsigned long long* peer_buffers_host,
+                                         void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || shape->E % n_ranks) return R3_ERR_INVALID_ARG;
+    if (shape->T == 0) return R3_OK;
+    if (!x || !idx || !row_of_slot || !my_offsets || !dst_base || !peer_buffers_host ||
+        !r3::aligned(x, 16))
+        return R3_ERR_INVALID_ARG;
+    r3::EpPeers peers = {};
+    for (int q = 0; q < n_ranks; ++q) {
+        if (!peer_buffers_host[q] || (peer_buffers_host[q] & 15)) return R3_ERR_INVALID_ARG;
+        peers.base[q] = peer_buffers_host[q];
+    }
+    const int row_vecs = (int)((size_t)shape->d * r3::act_bytes(shape) / 16);
+    const int wpb = 8;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    R3_DISPATCH_IDX(shape, IdxT,
+        r3::ep_dispatch_rows_kernel<IdxT><<<(shape->T + wpb - 1) / wpb, wpb * 32, 0, cs>>>(
+            static_cast<const uint4*>(x), static_cast<const IdxT*>(idx), row_of_slot, my_offsets,
+            dst_base, peers, shape->T, shape->E, shape->K, shape->E / n_ranks, row_vecs));
+    return r3::launch_status();
+}
+
+extern "C" r3_status r3_ep_slot_rows(const r3_shape* shape, int32_t n_ranks, const void* idx,
+                                     const int32_t* row_of_slot, const int32_t* my_offsets,
+                                     const int32_t* dst_base,
+                                     const unsigned long long* peer_buffers_host,
+                                     unsigned long long* row_ptr, void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || shape->E % n_ranks) return R3_ERR_INVALID_ARG;
+    if (shape->T == 0) return R3_OK;
+    if (!idx || !row_of_slot || !my_offsets || !dst_base || !peer_buffers_host || !row_ptr)
+        return R3_ERR_INVALID_ARG;
+    r3::EpPeers peers = {};
+    for (int q = 0; q < n_ranks; ++q) {
+        if (!peer_buffers_host[q] || (peer_buffers_host[q] & 15)) return R3_ERR_INVALID_ARG;
+        peers.base[q] = peer_buffers_host[q];
+    }
+    const long long pairs = (long long)shape->T * shape->K;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    R3_DISPATCH_IDX(shape, IdxT,
+        r3::ep_slot_rows_kernel<IdxT><<<(unsigned)((pairs + 255) / 256), 256, 0, cs>>>(
+            static_cast<const IdxT*>(idx), row_of_slot, my_offsets, dst_base, peers, row_ptr, pairs,
+            shape->E / n_ranks, (unsigned long long)shape->d * r3::act_bytes(shape)));
+    return r3::launch_status();
+}
+
 extern "C" r3_status r3_ep_regroup_map(const int32_t* recv_counts, int32_t n_src, int32_t e_local,
                                        int32_t rows, int32_t* perm, int32_t* offsets,
                                        int32_t* dev_status, void* stream) {

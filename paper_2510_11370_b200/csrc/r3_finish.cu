@@ -207,10 +207,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-template <typename ActT, typename IdxT>
+// PTR: the expert-output row of slot (t, j) is given by its address row_ptr[t, j] (0 = no row)
+// instead of by a row number into `o` - the rows may then live in several buffers, also in another
+// GPU's memory that this GPU can address (plain bulk copies, no multicast).
+template <typename ActT, typename IdxT, bool PTR>
 __global__ void __launch_bounds__(kTokThreads)
 replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __restrict__ idx,
                             const ActT* __restrict__ o, const int32_t* __restrict__ row_of_slot,
+                            const unsigned long long* __restrict__ row_ptr,
                             const ActT* __restrict__ dy, const ActT* __restrict__ residual,
                             ActT* __restrict__ y, float* __restrict__ gates_out,
                             float* __restrict__ dlogits, int E, int K, int d, int W,
@@ -235,7 +239,16 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
     if (warp == 0) {
         // ---- ask for the rows ---------------------------------------------------------------------
         int32_t r = -1;
-        if (lane < K) r = row_of_slot[(size_t)t * K + lane];
+        const ActT* src_row = nullptr;
+        if (lane < K) {
+            if (PTR) {
+                src_row = reinterpret_cast<const ActT*>(row_ptr[(size_t)t * K + lane]);
+                r = src_row ? 0 : -1;
+            } else {
+                r = row_of_slot[(size_t)t * K + lane];
+                if (r >= 0) src_row = o + (size_t)r * d;
+            }
+        }
         if (lane == 0) {
             tc::mbar_init(bar, 1);
             flags[0] = 0;
@@ -250,8 +263,7 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
         }
         __syncwarp();
         if (lane < K) {
-            if (r >= 0)
-                bulk_load(s_rows + (uint32_t)lane * row_bytes, o + (size_t)r * d, row_bytes, bar);
+            if (r >= 0) bulk_load(s_rows + (uint32_t)lane * row_bytes, src_row, row_bytes, bar);
         } else if (lane == K) {
             bulk_load(s_rows + (uint32_t)K * row_bytes, dy + (size_t)t * d, row_bytes, bar);
         } else if (lane == K + 1) {
@@ -382,27 +394,42 @@ static int pick_team_fused(int row_vecs) {
 }
 
 template <typename ActT, typename IdxT>
-static void launch_finish(const r3_shape* s, const float* logits, const void* idx, const void* o,
-                          const int32_t* row_of_slot, const void* dy, const void* residual,
-                          void* y, float* gates_out, float* dlogits, int32_t* dev_status,
-                          cudaStream_t cs) {
+static r3_status launch_finish(const r3_shape* s, const float* logits, const void* idx,
+                               const void* o, const int32_t* row_of_slot,
+                               const unsigned long long* row_ptr, const void* dy,
+                               const void* residual, void* y, float* gates_out, float* dlogits,
+                               int32_t* dev_status, cudaStream_t cs) {
     const int T = s->T, K = s->K, d = s->d, E = s->E;
     int W = 1;
     while (W < K && W < 32) W <<= 1;
     // staged kernel: one CTA per token, its K + 2 rows in shared memory (when they fit)
     const size_t smem = kTokHeader + 128 + (size_t)(K + 1 + (residual ? 1 : 0)) * d * sizeof(ActT);
-    if (smem <= (size_t)kTokSmemLimit / 2) {
-        auto kern = replay_finish_staged_kernel<ActT, IdxT>;
+    if (smem <= (size_t)kTokSmemLimit / 2 && row_ptr) {
+        auto kern = replay_finish_staged_kernel<ActT, IdxT, true>;
         static bool attr_set = false;          // one flag per instantiation
         if (!attr_set) {
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
             attr_set = true;
         }
         kern<<<T, kTokThreads, smem, cs>>>(
-            logits, static_cast<const IdxT*>(idx), static_cast<const ActT*>(o), row_of_slot,
+            logits, static_cast<const IdxT*>(idx), nullptr, nullptr, row_ptr,
             static_cast<const ActT*>(dy), static_cast<const ActT*>(residual), static_cast<ActT*>(y),
             gates_out, dlogits, E, K, d, W, dev_status);
-        return;
+        return R3_OK;
+    }
+    if (row_ptr) return R3_ERR_UNSUPPORTED;    // rows by address need the staged kernel
+    if (smem <= (size_t)kTokSmemLimit / 2) {
+        auto kern = replay_finish_staged_kernel<ActT, IdxT, false>;
+        static bool attr_set = false;          // one flag per instantiation
+        if (!attr_set) {
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
+            attr_set = true;
+        }
+        kern<<<T, kTokThreads, smem, cs>>>(
+            logits, static_cast<const IdxT*>(idx), static_cast<const ActT*>(o), row_of_slot, nullptr,
+            static_cast<const ActT*>(dy), static_cast<const ActT*>(residual), static_cast<ActT*>(y),
+            gates_out, dlogits, E, K, d, W, dev_status);
+        return R3_OK;
     }
     const int tpt = pick_team_fused(d / Vec16<ActT>::N);
     const unsigned grid = (unsigned)((T + 256 / tpt - 1) / (256 / tpt));
@@ -418,6 +445,7 @@ static void launch_finish(const r3_shape* s, const float* logits, const void* id
         default: R3_FIN(256); break;
     }
 #undef R3_FIN
+    return R3_OK;
 }
 
 }  // namespace r3
@@ -436,7 +464,26 @@ extern "C" r3_status r3_replay_finish(const r3_shape* shape, const float* logits
         return R3_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     R3_DISPATCH_ACT(shape, ActT, R3_DISPATCH_IDX(shape, IdxT,
-        (r3::launch_finish<ActT, IdxT>(shape, logits, idx, o, row_of_slot, dy, residual, y,
-                                       gates_out, dlogits, dev_status, cs))));
-    return r3::launch_status();
+        (st = r3::launch_finish<ActT, IdxT>(shape, logits, idx, o, row_of_slot, nullptr, dy,
+                                            residual, y, gates_out, dlogits, dev_status, cs))));
+    return st != R3_OK ? st : r3::launch_status();
+}
+
+extern "C" r3_status r3_replay_finish_rows(const r3_shape* shape, const float* logits,
+                                           const void* idx, const unsigned long long* row_ptr,
+                                           const void* dy, const void* residual, void* y,
+                                           float* gates_out, float* dlogits, int32_t* dev_status,
+                                           void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->K > r3::kFusedMaxK) return R3_ERR_UNSUPPORTED;
+    if (shape->T == 0) return R3_OK;
+    if (!logits || !idx || !row_ptr || !dy || !y || !dlogits) return R3_ERR_INVALID_ARG;
+    if (!r3::aligned(dy, 16) || !r3::aligned(y, 16) || !r3::aligned(residual, 16))
+        return R3_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    R3_DISPATCH_ACT(shape, ActT, R3_DISPATCH_IDX(shape, IdxT,
+        (st = r3::launch_finish<ActT, IdxT>(shape, logits, idx, nullptr, nullptr, row_ptr, dy,
+                                            residual, y, gates_out, dlogits, dev_status, cs))));
+    return st != R3_OK ? st : r3::launch_status();
 }

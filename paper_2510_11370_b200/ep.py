@@ -100,6 +100,121 @@ class EpRank:
         return y, dlogits, gates
 
 
+class EpDirectRank:
+    """One rank of the direct-write form: no collective carries rows.  After an all-gather of the
+    per-expert counts every rank knows where each of its rows stands in its owner's
+    [local expert][source][row] buffer, writes it there itself (r3_ep_dispatch_rows: plain stores
+    into buffers this GPU can address - peers' memory over NVLink) and, once the owners have run
+    their experts, pulls the outputs of its rows by address (r3_replay_finish_rows).  Two
+    barriers of the job separate the phases; the receive and output buffers of all ranks must
+    be addressable from every rank (peer access or symmetric memory)."""
+
+    def __init__(self, rank: int, world: int, T: int, d: int, E: int, K: int, F: int,
+                 act=torch.bfloat16, router_w=torch.float32, idx_dtype=torch.uint8):
+        if E % world:
+            raise ValueError("the number of experts must be a multiple of the number of ranks")
+        self.rank, self.world, self.e_local = rank, world, E // world
+        self.shape = r3.make_shape(T, d, E, K, F, act=act, router=router_w, idx=idx_dtype)
+        self.d, self.F, self.E, self.act = d, F, E, act
+        self.status = None
+
+    def route(self, x, w_router, idx):
+        """Logits and dispatch maps of this rank's tokens.  Returns counts [E] int32 (device)."""
+        s = self.shape
+        self.status = r3.new_status(x.device)
+        self.x, self.idx = x, idx
+        _, self.logits = r3.capture_topk_ws(s, 1, x, w_router, want_idx=False, want_logits=True)
+        self.counts, self.offsets, self.row_of_slot, _, _ = r3.permute(s, idx,
+                                                                       dev_status=self.status)
+        return self.counts
+
+    def plan(self, counts_all):
+        """counts_all [N, E] (all-gathered).  Returns the rows this rank will receive."""
+        self.dst_base, self.offsets_local = r3.ep_dest_table(counts_all.contiguous(), self.rank)
+        el = self.e_local
+        mine = counts_all[:, self.rank * el:(self.rank + 1) * el]
+        self.recv_rows = int(mine.sum().item())
+        return self.recv_rows
+
+    def send(self, receive_buffers):
+        """receive_buffers: base addresses of every rank's [rows, d] receive buffer."""
+        r3.ep_dispatch_rows(self.shape, self.world, self.x, self.idx, self.row_of_slot,
+                            self.offsets, self.dst_base, receive_buffers)
+
+    def experts(self, received, w_gate, w_up, w_down, out):
+        """This rank's experts on its receive buffer (already in expert-major order)."""
+        if self.recv_rows:
+            s_local = r3.make_shape(self.recv_rows, self.d, self.e_local, 1, self.F, act=self.act)
+            r3.grouped_swiglu(s_local, received, self.offsets_local, w_gate, w_up, w_down, out,
+                              dev_status=self.status)
+        return out
+
+    def finish(self, output_buffers, dy):
+        """output_buffers: base addresses of every rank's expert-output buffer."""
+        row_ptr = r3.ep_slot_rows(self.shape, self.world, self.idx, self.row_of_slot, self.offsets,
+                                  self.dst_base, output_buffers)
+        y, gates, dlogits = r3.replay_finish_rows(self.shape, self.logits, self.idx, row_ptr, dy,
+                                                  dev_status=self.status)
+        return y, dlogits, gates
+
+
+class PeerBuffers:
+    """The receive and output buffers of all ranks as seen from this rank: the rank's own two
+    tensors, the base addresses of everybody's, and the job's barrier."""
+
+    def __init__(self, received, outputs, receive_addresses, output_addresses, barrier):
+        self.received, self.outputs = received, outputs
+        self.receive_addresses, self.output_addresses = receive_addresses, output_addresses
+        self.barrier = barrier
+
+    @classmethod
+    def single(cls, capacity_rows: int, d: int, dtype, device):
+        """A job of one rank: the rank's own memory, no barrier needed beyond stream order."""
+        rec = torch.empty((max(capacity_rows, 1), d), dtype=dtype, device=device)
+        out = torch.empty_like(rec)
+        return cls(rec, out, [rec.data_ptr()], [out.data_ptr()], lambda: None)
+
+    @classmethod
+    def symmetric(cls, capacity_rows: int, d: int, dtype, device, group=None):
+        """Buffers of the same size on every rank, mapped into every rank's address space
+        (torch symmetric memory: NVLink peer mappings).  capacity_rows must cover the worst case
+        this job can route to one rank (at most world x T x K)."""
+        import torch.distributed._symmetric_memory as symm
+        group = group if group is not None else dist.group.WORLD
+        rec = symm.empty((max(capacity_rows, 1), d), dtype=dtype, device=device)
+        out = symm.empty((max(capacity_rows, 1), d), dtype=dtype, device=device)
+        h_rec = symm.rendezvous(rec, group=group)
+        h_out = symm.rendezvous(out, group=group)
+
+        def barrier():
+            torch.cuda.current_stream().synchronize()
+            dist.barrier(group=group)
+
+        return cls(rec, out, list(h_rec.buffer_ptrs), list(h_out.buffer_ptrs), barrier)
+
+
+def ep_replay_layer_direct(state: "EpDirectRank", buffers: PeerBuffers, x, w_router, idx, w_gate,
+                           w_up, w_down, dy, group=None):
+    """One expert-parallel replayed layer in the direct-write form: (y, dlogits, gates).  The only
+    collective is the all-gather of the [E] row counts."""
+    counts = state.route(x, w_router, idx)
+    if state.world > 1:
+        counts_all = torch.empty((state.world, state.E), dtype=counts.dtype, device=counts.device)
+        dist.all_gather_into_tensor(counts_all, counts, group=group)
+    else:
+        counts_all = counts.view(1, -1)
+    rows = state.plan(counts_all)
+    if rows > buffers.received.shape[0]:
+        raise ValueError("receive buffer too small for the rows routed to this rank")
+    state.send(buffers.receive_addresses)
+    buffers.barrier()                       # every rank's rows have landed everywhere
+    state.experts(buffers.received, w_gate, w_up, w_down, buffers.outputs)
+    buffers.barrier()                       # every owner's outputs are complete
+    result = state.finish(buffers.output_addresses, dy)
+    buffers.barrier()                       # nobody overwrites a buffer that is still being read
+    return result
+
+
 def ep_replay_layer(state: EpRank, x, w_router, idx, w_gate, w_up, w_down, dy, group=None):
     """One expert-parallel replayed layer on this rank with torch.distributed collectives:
     (y [T,d], dlogits [T,E], gates [T,K]).  w_gate / w_up / w_down hold this rank's experts."""

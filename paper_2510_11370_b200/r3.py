@@ -42,7 +42,8 @@ EXPORTS = [
     "r3_grouped_swiglu_bwd", "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
     "r3_replay_layer_train_workspace_bytes", "r3_replay_layer_train",
     "r3_replay_stack_train_workspace_bytes", "r3_replay_stack_train",
-    "r3_ep_regroup_map", "r3_ep_move_rows",
+    "r3_ep_regroup_map", "r3_ep_move_rows", "r3_ep_dest_table", "r3_ep_dispatch_rows",
+    "r3_ep_slot_rows", "r3_replay_finish_rows",
     "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
     "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
@@ -68,6 +69,10 @@ lib.r3_replay_stack_train_workspace_bytes.restype = ctypes.c_size_t
 lib.r3_replay_stack_train_workspace_bytes.argtypes = [_SP, ctypes.c_int32]
 lib.r3_replay_stack_train.argtypes = [_SP, ctypes.c_int32] + [_P] * 15 + [ctypes.c_size_t, _P, _P]
 lib.r3_ep_regroup_map.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _P, _P, _P, _P]
+lib.r3_ep_dest_table.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _P, _P, _P]
+lib.r3_ep_dispatch_rows.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, _P]
+lib.r3_ep_slot_rows.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, _P]
+lib.r3_replay_finish_rows.argtypes = [_SP] + [_P] * 10
 lib.r3_ep_move_rows.argtypes = [_P, _P, _P, ctypes.c_int32, ctypes.c_size_t, ctypes.c_int32, _P]
 lib.r3_grouped_swiglu_bwd.argtypes = [_SP] + [_P] * 13 + [ctypes.c_size_t, _P, _P]
 for _n in ("r3_permute_workspace_bytes", "r3_grouped_swiglu_workspace_bytes",
@@ -688,6 +693,53 @@ def ep_regroup_map(recv_counts, rows: int, *, dev_status=None, stream=None):
                                  _ptr(perm) if rows else None, _ptr(offsets), _ptr(dev_status),
                                  _stream(stream)))
     return perm, offsets
+
+
+def _peer_array(addresses):
+    return (ctypes.c_uint64 * len(addresses))(*[int(a) for a in addresses])
+
+
+def ep_dest_table(counts_all, rank: int, *, stream=None):
+    """counts_all [n_ranks, E] int32 (device) -> (dst_base [E], offsets_local [E/n_ranks + 1])."""
+    n, E = counts_all.shape
+    dev = _dev(counts_all)
+    dst_base = torch.empty(E, dtype=torch.int32, device=dev)
+    offsets_local = torch.empty(E // n + 1, dtype=torch.int32, device=dev)
+    _check(lib.r3_ep_dest_table(_ptr(counts_all), n, E, rank, _ptr(dst_base), _ptr(offsets_local),
+                                _stream(stream)))
+    return dst_base, offsets_local
+
+
+def ep_dispatch_rows(s: Shape, n_ranks: int, x, idx, row_of_slot, my_offsets, dst_base,
+                     peer_addresses, *, stream=None):
+    """x[t] straight into the owners' receive buffers (peer_addresses: their base addresses)."""
+    arr = _peer_array(peer_addresses)
+    _check(lib.r3_ep_dispatch_rows(ctypes.byref(s), n_ranks, _ptr(x), _ptr(idx), _ptr(row_of_slot),
+                                   _ptr(my_offsets), _ptr(dst_base), arr, _stream(stream)))
+
+
+def ep_slot_rows(s: Shape, n_ranks: int, idx, row_of_slot, my_offsets, dst_base, peer_addresses,
+                 *, stream=None):
+    """[T, K] addresses of the pairs' expert-output rows in the owners' output buffers."""
+    row_ptr = torch.empty((s.T, s.K), dtype=torch.int64, device=_dev(idx))
+    arr = _peer_array(peer_addresses)
+    _check(lib.r3_ep_slot_rows(ctypes.byref(s), n_ranks, _ptr(idx), _ptr(row_of_slot),
+                               _ptr(my_offsets), _ptr(dst_base), arr, _ptr(row_ptr),
+                               _stream(stream)))
+    return row_ptr
+
+
+def replay_finish_rows(s: Shape, logits, idx, row_ptr, dy, *, residual=None, dev_status=None,
+                       stream=None):
+    """r3_replay_finish with the expert-output rows given by address.  (y, gates, dlogits)."""
+    dev = _dev(idx)
+    y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    gates = torch.empty((s.T, s.K), dtype=torch.float32, device=dev)
+    dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
+    _check(lib.r3_replay_finish_rows(ctypes.byref(s), _ptr(logits), _ptr(idx), _ptr(row_ptr),
+                                     _ptr(dy), _ptr(residual), _ptr(y), _ptr(gates), _ptr(dlogits),
+                                     _ptr(dev_status), _stream(stream)))
+    return y, gates, dlogits
 
 
 def ep_move_rows(src, perm, *, inverse=False, stream=None):

@@ -129,3 +129,87 @@ def test_process_group_of_one_runs_the_real_collectives(r3):
     finally:
         if created:
             dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("n,E", [(1, 8), (2, 8), (4, 16), (8, 16)])
+def test_destination_table_against_the_oracle(r3, n, E):
+    rng = np.random.default_rng(n + E)
+    counts = rng.integers(0, 50, size=(n, E))
+    counts[rng.random(counts.shape) < 0.2] = 0
+    dev_counts = torch.from_numpy(counts.astype(np.int32)).cuda()
+    for me in range(n):
+        dst_base, offsets_local = r3.ep_dest_table(dev_counts, me)
+        ref_base, ref_off = EP.dest_table(counts, me)
+        assert np.array_equal(dst_base.cpu().numpy(), ref_base)
+        assert np.array_equal(offsets_local.cpu().numpy(), ref_off)
+
+
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_direct_write_ranks_equal_the_single_gpu_layer(r3, world):
+    """The direct-write form with `world` ranks on one GPU: every rank's buffers live on this GPU,
+    so "a peer's memory" is simply another tensor; the phases run rank after rank with the
+    barriers of a real job replaced by program order.  Bit-identical to the plain layer."""
+    from paper_2510_11370_b200.ep import EpDirectRank
+    T, d, E, K, F = 640, 256, 16, 4, 128
+    w, x, dy, w_r, wg, wu, wd, idx = _case(T, d, E, K, F)
+    dev = "cuda"
+    xs, dys, idxs = x.to(dev), dy.to(dev), idx.to(dev)
+    w_r_d, wg_d, wu_d, wd_d = w_r.to(dev), wg.to(dev), wu.to(dev), wd.to(dev)
+    y_ref, ds_ref, g_ref = r3.replay_layer(r3.shape_of(w), xs, w_r_d, idxs, wg_d, wu_d, wd_d, dys)
+    Tl, el = T // world, E // world
+    tok = lambda q: slice(q * Tl, (q + 1) * Tl)
+    ranks = [EpDirectRank(q, world, Tl, d, E, K, F) for q in range(world)]
+    counts_all = torch.stack([rk.route(xs[tok(q)], w_r_d, idxs[tok(q)])
+                              for q, rk in enumerate(ranks)])           # the all-gather
+    recv = [torch.full((max(rk.plan(counts_all), 1), d), float("nan"), dtype=torch.bfloat16,
+                       device=dev) for rk in ranks]
+    outs = [torch.empty_like(b) for b in recv]
+    for rk in ranks:
+        rk.send([b.data_ptr() for b in recv])
+    torch.cuda.synchronize()                                             # barrier 1
+    assert sum(rk.recv_rows for rk in ranks) == T * K
+    for q, rk in enumerate(ranks):
+        assert not torch.isnan(recv[q][:rk.recv_rows].float()).any()     # every row was written
+        ex = slice(q * el, (q + 1) * el)
+        rk.experts(recv[q], wg_d[ex].contiguous(), wu_d[ex].contiguous(), wd_d[ex].contiguous(),
+                   outs[q])
+    torch.cuda.synchronize()                                             # barrier 2
+    for q, rk in enumerate(ranks):
+        y, dlogits, gates = rk.finish([b.data_ptr() for b in outs], dys[tok(q)])
+        torch.cuda.synchronize()
+        assert rk.status.item() == 0
+        assert torch.equal(y, y_ref[tok(q)]) and torch.equal(dlogits, ds_ref[tok(q)])
+        assert torch.equal(gates, g_ref[tok(q)])
+
+
+def test_direct_form_driver_with_one_rank(r3):
+    """ep_replay_layer_direct as a job of one rank (its own buffers), and, where this torch build
+    can set it up for a group of one, with symmetric-memory buffers."""
+    import torch.distributed as dist
+    from paper_2510_11370_b200.ep import EpDirectRank, PeerBuffers, ep_replay_layer_direct
+    T, d, E, K, F = 300, 256, 16, 4, 128
+    w, x, dy, w_r, wg, wu, wd, idx = _case(T, d, E, K, F)
+    c = [t.cuda() for t in (x, w_r, idx, wg, wu, wd, dy)]
+    y0, ds0, g0 = r3.replay_layer(r3.shape_of(w), *c)
+    bufs = PeerBuffers.single(T * K, d, torch.bfloat16, "cuda")
+    y, dlogits, gates = ep_replay_layer_direct(EpDirectRank(0, 1, T, d, E, K, F), bufs, *c)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y0) and torch.equal(dlogits, ds0) and torch.equal(gates, g0)
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    created = not dist.is_initialized()
+    if created:
+        os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        try:
+            sym = PeerBuffers.symmetric(T * K, d, torch.bfloat16, torch.device("cuda", 0))
+        except Exception as exc:                     # set-up of symmetric memory, not the library
+            pytest.skip(f"symmetric memory unavailable for a group of one here: {exc!r}"[:200])
+        y, dlogits, gates = ep_replay_layer_direct(EpDirectRank(0, 1, T, d, E, K, F), sym, *c)
+        torch.cuda.synchronize()
+        assert torch.equal(y, y0) and torch.equal(dlogits, ds0) and torch.equal(gates, g0)
+    finally:
+        if created:
+            dist.destroy_process_group()
