@@ -30,7 +30,7 @@
 // item boundary, because the peer CTA learns its next item late; it was slower.)
 //
 // Roles (192 threads per CTA): warp 0 lane 0 = TMA producer (both CTAs, into a 6-stage ring of
-// 128B-swizzled tiles), warp 1 lane 0 of the leader CTA = MMA issuer (two accumulator stages of
+// 128B-swizzled tiles), warp 1 of the leader CTA = MMA issuer (one elected lane) (two accumulator stages of
 // 256 columns, so the epilogue of an item overlaps the main loop of the next), warps 2..5 =
 // epilogue (tcgen05.ld -> transpose through shared memory -> 16-byte global stores).
 //
@@ -292,39 +292,50 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer (leader CTA only) ---------------------------
-        if (lane == 0 && rank == 0) {
+        // The whole warp of the leader CTA walks the barriers; one elected lane issues the MMAs
+        // and commits (the compiler then sees a warp-uniform loop around a single-thread region).
+        if (rank == 0) {
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
+            int n_next = w_begin < w_end ? items[w_begin].z : 0;
             for (int w = w_begin; ok && w < w_end; w += w_step) {
-                const int n = items[w].z;
+                const int n = n_next;
+                if (w + w_step < w_end) n_next = items[w + w_step].z;   // lands during this item
                 const uint32_t idesc = instr_desc_bf16(2 * BMF, n) | (MODE >= 2 ? kInstrDescAMajorMN : 0u);
-                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status)) break;
+                if (!__all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag,
+                                                       dev_status)))
+                    break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNT);
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag, dev_status)) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, abort_flag,
+                                                           dev_status))) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    const uint64_t da = MODE >= 2 ? smem_desc_mn_sw128(sa, A_BYTES / 2)
-                                                  : smem_desc_sw128(sa);
-                    const uint64_t db = smem_desc_sw128(sb);
-                    // per MMA (16 along k): K-major tiles move 32 bytes inside the swizzled row,
-                    // the MN-major tile moves two groups of 8 k rows = 2048 bytes
-                    constexpr uint64_t a_step = MODE >= 2 ? (2048 >> 4) : 2;
+                    if (elect_one()) {
+                        const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                        const uint64_t da = MODE >= 2 ? smem_desc_mn_sw128(sa, A_BYTES / 2)
+                                                      : smem_desc_sw128(sa);
+                        const uint64_t db = smem_desc_sw128(sb);
+                        // per MMA (16 along k): K-major tiles move 32 bytes inside the swizzled
+                        // row, the MN-major tile moves two groups of 8 k rows = 2048 bytes
+                        constexpr uint64_t a_step = MODE >= 2 ? (2048 >> 4) : 2;
 #pragma unroll
-                    for (int kk = 0; kk < BK / UK; ++kk) {
-                        tc_mma_bf16_pair(d_tmem, da + a_step * kk, db + (uint64_t)(kk * 2), idesc,
-                                         (kb | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < BK / UK; ++kk) {
+                            tc_mma_bf16_pair(d_tmem, da + a_step * kk, db + (uint64_t)(kk * 2), idesc,
+                                             (kb | kk) != 0 ? 1u : 0u);
+                        }
+                        tc_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
                     }
-                    tc_commit_pair(empty_bar(stage), 3);   // frees the stage in both CTAs
+                    __syncwarp();
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit_pair(tfull_bar(acc), 3);         // accumulator complete, both CTAs
+                if (elect_one()) tc_commit_pair(tfull_bar(acc), 3);   // accumulator complete, both CTAs
+                __syncwarp();
                 if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
             }
         }

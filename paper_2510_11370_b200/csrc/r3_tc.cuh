@@ -177,6 +177,13 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t tmem_base, uint32_t c
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
                  ::"r"(tmem_base), "r"(cols) : "memory");
 }
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t p;
+    asm volatile("{\n\t.reg .pred P;\n\t.reg .b32 r;\n\telect.sync r|P, 0xffffffff;\n\t"
+                 "selp.u32 %0, 1, 0, P;\n\t}" : "=r"(p));
+    return p != 0;
+}
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
