@@ -23,11 +23,15 @@
 // features, so lanes 0-63 hold the gate pre-activations and lanes 64-127 the up projections; the
 // epilogue exchanges them through shared memory to form the SwiGLU product.
 //
-// Items are ordered (expert, feature tile, token tile) and dealt to the clusters round-robin, so
-// the clusters running at any moment work on neighbouring items: their copies of a shared weight
-// tile or token tile meet in L2, and the weights stream from HBM once.  (Handing the items out
-// from a device counter instead balanced the clusters better but drained the copy ring at every
-// item boundary, because the peer CTA learns its next item late; it was slower.)
+// Items are ordered (expert, feature tile, token tile).  Every cluster takes three items by
+// position (cluster c: c, c + C, c + 2C for C clusters) and claims the rest in list order from a
+// device counter, so the clusters running at any moment work on neighbouring items (their copies
+// of a shared weight or token tile meet in L2 and the weights stream from HBM once) and no
+// cluster idles while another still holds a queue.  Claims run three items ahead of the copies:
+// the leader CTA's producer thread issues the atomic for item s + 4 when it starts item s, hands
+// item s + 3 to the peer CTA's producer through distributed shared memory, and both producers
+// publish each item's descriptor to the other warps of their CTA through a tagged ring in shared
+// memory, so nobody waits on a claim.  The last cluster to finish re-arms the counter.
 //
 // Roles (192 threads per CTA): warp 0 lane 0 = TMA producer (both CTAs, into a 6-stage ring of
 // 128B-swizzled tiles), warp 1 of the leader CTA = MMA issuer (one elected lane) (two accumulator stages of
@@ -58,7 +62,10 @@ constexpr int EPI_WARPS = 4;
 constexpr int THREADS = (2 + EPI_WARPS) * 32;
 constexpr int EPI_BYTES = 28 * 1024;             // transpose / exchange buffers of the epilogue
 constexpr int BAR_BYTES = 256;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + 1024;  // + alignment
+constexpr int RING = 16;                         // item descriptors / claims in flight per CTA
+constexpr int SCHED_BYTES = RING * 32 + RING * 8;
+constexpr int STATIC_ITEMS = 3;                  // items per cluster taken by position
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + SCHED_BYTES + 1024;
 constexpr int FEAT0 = BMF;         // h features per item in MODE 0 (64 per CTA, gate + up rows)
 constexpr int FEAT1 = 2 * BMF;     // o features per item in MODE 1
 
@@ -70,7 +77,8 @@ struct alignas(64) PairMaps {
 };
 
 // ---- work list -------------------------------------------------------------------------------
-// Per list: int32 header[kHeaderInts] = {number of items, ...}, then one int4 per item =
+// Per list: int32 header[kHeaderInts] = {number of items, claim counter, clusters finished, 0},
+// then one int4 per item =
 // {expert | feature tile << 16, first row, N (multiple of 16), valid rows}, ordered
 // (expert, feature tile, token tile).  An expert with cnt rows is cut into nt = ceil(cnt / 256)
 // token tiles of equal size q (rounded up to 16; the last one holds what is left).
@@ -84,7 +92,7 @@ __host__ __device__ inline int split_rows(int cnt, int nt) {      // rows per ti
 // One CTA per list (blockIdx.x = 0: up projection with nf0 feature tiles, 1: down with nf1).
 __global__ void __launch_bounds__(1024)
 build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
-                  int32_t* __restrict__ list0, int32_t* __restrict__ list1) {
+                  int32_t* __restrict__ list0, int32_t* __restrict__ list1, int pairs) {
     __shared__ int32_t s_items[1025];
     __shared__ int32_t w_items[32];
     const int nf = blockIdx.x == 0 ? nf0 : nf1;
@@ -116,7 +124,11 @@ build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
     if (tid == 1023) s_items[1024] = w_items[warp] + ii;
     __syncthreads();
     const int32_t I = s_items[1024];
-    if (tid == 0) list[0] = I;
+    if (tid == 0) {
+        list[0] = I;
+        list[1] = STATIC_ITEMS * pairs;          // first item handed out by the counter
+        list[2] = 0;
+    }
     for (int32_t i = tid; i < I; i += 1024) {
         int lo = 0, hi = E;                      // last e with s_items[e] <= i
         while (hi - lo > 1) {
@@ -133,6 +145,66 @@ build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
     }
 }
 
+// ---- item hand-over inside a CTA pair ---------------------------------------------------------
+// Descriptor ring (shared memory of one CTA): slot = sequence number % RING, 32 bytes = the item
+// (n = 0: no more items) and a tag = sequence number + 1 written last.  Written by the CTA's
+// producer thread when it starts the item, read by the MMA and epilogue warps.
+__device__ __forceinline__ void desc_put(uint8_t* ring, int seq, const int4& d) {
+    volatile int32_t* slot = reinterpret_cast<volatile int32_t*>(ring + (seq % RING) * 32);
+    slot[0] = d.x;
+    slot[1] = d.y;
+    slot[2] = d.z;
+    slot[3] = d.w;
+    __threadfence_block();
+    slot[4] = seq + 1;
+}
+__device__ __forceinline__ bool desc_get(uint8_t* ring, int seq, int4* d, volatile int* abort_flag,
+                                         int32_t* dev_status) {
+    volatile int32_t* slot = reinterpret_cast<volatile int32_t*>(ring + (seq % RING) * 32);
+    if (slot[4] != seq + 1) {
+        const long long t0 = clock64();
+        while (slot[4] != seq + 1) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_CLOCKS) {
+                *abort_flag = 1;
+                report(dev_status, R3_DEV_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    __threadfence_block();
+    *d = make_int4(slot[0], slot[1], slot[2], slot[3]);
+    return true;
+}
+// Claim ring (shared memory of the peer CTA, written by the leader's producer through the
+// cluster's distributed shared memory): one 64-bit word per slot = tag (sequence + 1) << 32 | item.
+__device__ __forceinline__ void claim_post(uint32_t peer_ring, int seq, int item) {
+    const unsigned long long v = ((unsigned long long)(uint32_t)(seq + 1) << 32) | (uint32_t)item;
+    asm volatile("st.volatile.shared::cluster.u64 [%0], %1;"
+                 ::"r"(peer_ring + (uint32_t)(seq % RING) * 8u), "l"(v) : "memory");
+}
+__device__ __forceinline__ bool claim_get(uint8_t* ring, int seq, int* item, volatile int* abort_flag,
+                                          int32_t* dev_status) {
+    volatile unsigned long long* slot =
+        reinterpret_cast<volatile unsigned long long*>(ring) + (seq % RING);
+    unsigned long long v = *slot;
+    if ((uint32_t)(v >> 32) != (uint32_t)(seq + 1)) {
+        const long long t0 = clock64();
+        for (;;) {
+            v = *slot;
+            if ((uint32_t)(v >> 32) == (uint32_t)(seq + 1)) break;
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_CLOCKS) {
+                *abort_flag = 1;
+                report(dev_status, R3_DEV_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    *item = (int)(uint32_t)v;
+    return true;
+}
+
 // ---- the GEMM kernel --------------------------------------------------------------------------
 // GATHER (up projection only): the token operand is read from the un-permuted activations
 // x [T, d], row slot_of_row[r] / K for grouped row r, with TMA gather4 copies (each lane of the
@@ -140,7 +212,7 @@ build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
 // block), so the permuted copy of x never has to exist.
 template <int MODE, bool GATHER>
 __global__ void __launch_bounds__(THREADS, 1)
-grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* __restrict__ list,
+grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
                          const int32_t* __restrict__ slot_of_row, int K,
                          __nv_bfloat16* __restrict__ out, __nv_bfloat16* __restrict__ pre_gate,
                          __nv_bfloat16* __restrict__ pre_up, int Kdim, int Nout,
@@ -157,13 +229,16 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
     uint8_t* misc = epi_ptr + EPI_BYTES + 128;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+    uint8_t* desc_ring = epi_ptr + EPI_BYTES + BAR_BYTES;
+    uint8_t* claim_ring = desc_ring + RING * 32;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
     const int pair = blockIdx.x >> 1;
     const int w_step = gridDim.x >> 1;
     const int w_begin = pair, w_end = list[0];
-    const int4* items = reinterpret_cast<const int4*>(list + kHeaderInts);
+    const int4* __restrict__ items = reinterpret_cast<const int4*>(list + kHeaderInts);
+    const int4 kNone = make_int4(0, 0, 0, 0);          // n = 0 ends the item stream
     // MODE 3 walks the k blocks of both weight matrices alternately
     const int kblocks = (MODE == 3 ? 2 : 1) * ((Kdim + BK - 1) / BK);
 
@@ -174,6 +249,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
             mbar_init(tempty_bar(a), 2 * EPI_WARPS);       // epilogue warps of both CTAs
         }
         *abort_flag = 0;
+        for (int i = 0; i < SCHED_BYTES / 4; ++i) reinterpret_cast<volatile int32_t*>(desc_ring)[i] = 0;
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
@@ -188,7 +264,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        const int4 kNone = make_int4(0, 0, 0, 0);
+        int seq = 0;
         // token (row of x) of rows 4*lane .. 4*lane+3 of this CTA's half of item `it`
         auto load_tokens = [&](const int4& it, int* tok) {
             const int half = it.z >> 1;
@@ -210,6 +286,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
             it_cur = it_nxt;
             it_nxt = w + 2 * w_step < w_end ? items[w + 2 * w_step] : kNone;
             load_tokens(it_cur, nxt);             // lands while this item's copies are issued
+            if (lane == 0) desc_put(desc_ring, seq, it);
+            ++seq;
             const int e = it.x & 0xffff, f = it.x >> 16, n = it.z, half = n >> 1;
             for (int kb = 0; kb < kblocks; ++kb) {
                 int free_ok = 1;
@@ -235,6 +313,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
             }
         }
         if (lane == 0) {
+            desc_put(desc_ring, seq, kNone);
             for (int s = 0; ok && s < STAGES; ++s) {
                 ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -246,8 +325,45 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int w = w_begin; ok && w < w_end; w += w_step) {
-                const int4 it = items[w];
+            const int I = w_end, P = w_step;
+            int32_t* counter = list + 1;
+            const uint32_t peer_claims = mapa_shared(smem_u32(claim_ring), 1);
+            int seq = 0;
+            int idx_cur = pair;
+            int4 it_cur = idx_cur < I ? items[idx_cur] : kNone;
+            // leader only: items seq + 1 and seq + 2, the descriptor of seq + 1, and the claim in
+            // flight (it becomes item seq + 3 when the next item starts)
+            int idx_n1 = pair + P, idx_n2 = pair + 2 * P;
+            int4 it_n1 = kNone;
+            int pending = I;
+            if (rank == 0) {
+                if (idx_n1 < I) it_n1 = items[idx_n1];
+                if (idx_n2 < I) pending = atomicAdd(counter, 1);
+            }
+            while (ok && idx_cur < I) {
+                const int4 it = it_cur;
+                desc_put(desc_ring, seq, it);
+                int idx_next;
+                if (rank == 0) {
+                    const int claimed = pending;                     // item seq + 3
+                    claim_post(peer_claims, seq + 3, claimed);
+                    pending = claimed < I ? atomicAdd(counter, 1) : I;
+                    idx_next = idx_n1;
+                    it_cur = it_n1;
+                    it_n1 = idx_n2 < I ? items[idx_n2] : kNone;      // lands during this item
+                    idx_n1 = idx_n2;
+                    idx_n2 = claimed;
+                } else {
+                    if (seq + 1 < STATIC_ITEMS) {
+                        idx_next = pair + (seq + 1) * P;
+                    } else if (!claim_get(claim_ring, seq + 1, &idx_next, abort_flag, dev_status)) {
+                        ok = false;
+                        break;
+                    }
+                    it_cur = idx_next < I ? items[idx_next] : kNone; // lands during this item
+                }
+                idx_cur = idx_next;
+                ++seq;
                 const int e = it.x & 0xffff, f = it.x >> 16, n = it.z, half = n >> 1;
                 const CUtensorMap* bmap = &maps.b[(half >> 3) - 1];
                 for (int kb = 0; kb < kblocks; ++kb) {
@@ -283,6 +399,15 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            desc_put(desc_ring, seq, kNone);
+            if (rank == 0) {
+                // all of this cluster's claims have returned; the last cluster re-arms the counter
+                __threadfence();
+                if (atomicAdd(list + 2, 1) == P - 1) {
+                    atomicExch(counter, STATIC_ITEMS * P);
+                    atomicExch(list + 2, 0);
+                }
+            }
             // Tail: every stage's release (signalled from the leader's tensor core, also into the
             // peer CTA) must have landed before this CTA may leave.
             for (int s = 0; ok && s < STAGES; ++s) {
@@ -298,10 +423,11 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            int n_next = w_begin < w_end ? items[w_begin].z : 0;
-            for (int w = w_begin; ok && w < w_end; w += w_step) {
-                const int n = n_next;
-                if (w + w_step < w_end) n_next = items[w + w_step].z;   // lands during this item
+            for (int seq = 0; ok; ++seq) {
+                int4 it;
+                if (!desc_get(desc_ring, seq, &it, abort_flag, dev_status)) break;
+                const int n = it.z;
+                if (n == 0) break;
                 const uint32_t idesc = instr_desc_bf16(2 * BMF, n) | (MODE >= 2 ? kInstrDescAMajorMN : 0u);
                 if (!__all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag,
                                                        dev_status)))
@@ -347,8 +473,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, const int32_t* _
         int chunk_no = 0;
         bool alive = true;                            // false after a wait ran out: the barrier
                                                       // protocol goes on, the work is skipped
-        for (int w = w_begin; w < w_end; w += w_step) {
-            const int4 it = items[w];
+        for (int seq = 0;; ++seq) {
+            int4 it;
+            if (!desc_get(desc_ring, seq, &it, abort_flag, dev_status)) break;
+            if (it.z == 0) break;
             const int f = it.x >> 16, row0 = it.y, n = it.z, valid = it.w;
             if (alive) {
                 const bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, dev_status);
@@ -515,7 +643,7 @@ static int resident_pairs(Kern kern) {
 }
 
 template <int MODE, bool GATHER>
-static r3_status launch_pair(const PairMaps& maps, int pairs, const int32_t* list,
+static r3_status launch_pair(const PairMaps& maps, int pairs, int32_t* list,
                              const int32_t* slot_of_row, int K, void* out, int Kdim, int Nout,
                              int32_t* dev_status, cudaStream_t cs, void* pre_gate = nullptr,
                              void* pre_up = nullptr) {
@@ -612,7 +740,7 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
                                                 list_bytes(R, s->E, nf0));
     static TokenMapCache cache_xp, cache_h;
     if (phases & kPhaseUp) {
-        build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1);
+        build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1, pairs);
         PairMaps m;
         if (!make_map_3d(&m.a0, w_gate, s->E, s->F, s->d, BMF / 2) ||
             !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2))
@@ -684,7 +812,7 @@ r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, cons
     const bool weights = dw_gate != nullptr;
     int32_t* list_h = reinterpret_cast<int32_t*>(w);
     int32_t* list_x = reinterpret_cast<int32_t*>(w + list_bytes(R, s->E, nf_h));
-    build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf_h, nf_x, list_h, list_x);
+    build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf_h, nf_x, list_h, list_x, pairs);
 
     // dh = dout W_down   (weights transposed: contraction over d)
     static TokenMapCache cache_do;
