@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 LAUNCHES_PER_STEP = 8   # split_router_weight, router_tc, permute_maps_coop, permute_rows, build_work, two GEMMs, finish
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
 # from the ncu capture summarised in profiles/grouped_gemm_pair_c2_layer_bf16.md.
-GEMM_UP_DRAM_TRAFFIC_BYTES = 990.6e6   # 943.6 MB read + 47.0 MB written
+GEMM_UP_DRAM_TRAFFIC_BYTES = 990.4e6   # 942.9 MB read + 47.5 MB written
 
 
 def load_peaks():
