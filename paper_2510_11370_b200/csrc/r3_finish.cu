@@ -237,10 +237,14 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
     int my_e = -1;
     float g = 0.f;
     if (warp == 0) {
-        // ---- ask for the rows ---------------------------------------------------------------------
+        // ---- the token's record and row numbers first (independent loads), then the logit of
+        // each recorded expert, so that only two memory latencies precede the copies ------------
+        const IdxT* rec = idx + (size_t)t * K;
+        const float* lrow = logits + (size_t)t * E;
         int32_t r = -1;
         const ActT* src_row = nullptr;
         if (lane < K) {
+            my_e = idx_to_int(rec[lane]);
             if (PTR) {
                 src_row = reinterpret_cast<const ActT*>(row_ptr[(size_t)t * K + lane]);
                 r = src_row ? 0 : -1;
@@ -249,6 +253,9 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
                 if (r >= 0) src_row = o + (size_t)r * d;
             }
         }
+        float s = -INFINITY;
+        if (lane < K) s = lrow[min(max(my_e, 0), E - 1)];      // in flight while the rows are asked for
+        // ---- ask for the rows ---------------------------------------------------------------------
         if (lane == 0) {
             tc::mbar_init(bar, 1);
             flags[0] = 0;
@@ -272,16 +279,11 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
                           row_bytes, bar);
         }
         // ---- replay gate while the copies fly: the first W lanes, one slot each -----------------
-        const IdxT* rec = idx + (size_t)t * K;
-        const float* lrow = logits + (size_t)t * E;
         int bad = 0;
-        float s = -INFINITY;
-        if (lane < K) {
-            my_e = idx_to_int(rec[lane]);
-            if (my_e < 0 || my_e >= E) bad |= 1;
-            for (int j2 = 0; j2 < lane; ++j2)
-                if (idx_to_int(rec[j2]) == my_e) bad |= 2;
-            s = lrow[min(max(my_e, 0), E - 1)];
+        if (lane < K && (my_e < 0 || my_e >= E)) bad |= 1;
+        for (int j2 = 0; j2 < K; ++j2) {
+            const int e2 = __shfl_sync(0xffffffffu, my_e, j2);
+            if (j2 < lane && lane < K && e2 == my_e) bad |= 2;
         }
         for (int ofs = W / 2; ofs > 0; ofs >>= 1) bad |= __shfl_xor_sync(0xffffffffu, bad, ofs, W);
         if (bad && lane == 0)
