@@ -49,56 +49,127 @@ replay_gate_fwd_kernel(const float* __restrict__ logits, const IdxT* __restrict_
                 expf(row[min(max(idx_to_int(rec[j]), 0), E - 1)] - m) * inv;
 }
 
-// One warp per token.  Lanes hold up to 32 slots at a time (e_j, v_j = g_j (dg_j - c)); every lane
-// then assembles its 4-float pieces of the dense row from those slots and writes them, zeros
-// included, so the row is written exactly once.
+// K <= 8: one lane per token.  The lane reads its record, fetches the K recorded logits (K
+// independent loads in flight per lane) and forms the softmax in registers.  The sums are taken in
+// the order of the W-lane butterfly above (W = K rounded up to a power of two, missing slots add
+// 0), so both kernels give the same bits.
+template <typename IdxT>
+__global__ void __launch_bounds__(128)
+replay_gate_fwd_lane_kernel(const float* __restrict__ logits, const IdxT* __restrict__ idx,
+                            float* __restrict__ gates, int T, int E, int K, int W,
+                            int32_t* dev_status) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const IdxT* rec = idx + (size_t)t * K;
+    const float* row = logits + (size_t)t * E;
+    int e[8];
+    int bad = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) e[j] = j < K ? idx_to_int(rec[j]) : -1 - j;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        if (j < K) {
+            if (e[j] < 0 || e[j] >= E) bad |= 1;
+#pragma unroll
+            for (int j2 = 0; j2 < j; ++j2)
+                if (e[j2] == e[j]) bad |= 2;
+        }
+    }
+    if (bad) report(dev_status, (bad & 1) ? R3_DEV_BAD_INDEX : R3_DEV_DUP_INDEX);
+    float sv[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sv[j] = j < K ? row[min(max(e[j], 0), E - 1)] : -INFINITY;
+    float m = sv[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) m = fmaxf(m, sv[j]);
+    float ex[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) ex[j] = j < K ? expf(sv[j] - m) : 0.f;
+    float sum;
+    if (W == 8) sum = ((ex[0] + ex[4]) + (ex[2] + ex[6])) + ((ex[1] + ex[5]) + (ex[3] + ex[7]));
+    else if (W == 4) sum = (ex[0] + ex[2]) + (ex[1] + ex[3]);
+    else if (W == 2) sum = ex[0] + ex[1];
+    else sum = ex[0];
+    const float inv = bad ? 0.f : 1.f / sum;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (j < K) gates[(size_t)t * K + j] = ex[j] * inv;
+}
+
+// One warp per NT tokens, taken together so that their loads are in flight at once.  Per token
+// the lanes hold up to 32 slots (e_j, v_j = g_j (dg_j - c)); every lane then assembles its 4-float
+// pieces of the dense row from those slots and writes them, zeros included, so the row is written
+// exactly once.
+constexpr int kGateBwdTokens = 4;
 template <typename IdxT>
 __global__ void __launch_bounds__(256)
 replay_gate_bwd_kernel(const float* __restrict__ gates, const float* __restrict__ dgates,
                        const IdxT* __restrict__ idx, float* __restrict__ dlogits,
                        int T, int E, int K) {
+    constexpr int NT = kGateBwdTokens;
     const int lane = threadIdx.x & 31;
-    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (t >= T) return;
-    const size_t base = (size_t)t * K;
-
-    float c = 0.f;
-    for (int j = lane; j < K; j += 32) c += gates[base + j] * dgates[base + j];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-
-    float* out = dlogits + (size_t)t * E;
+    const long long t0 = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * NT;
+    if (t0 >= T) return;
     const int nchunk = (E + 3) >> 2;
     if (K <= 32) {
-        int e = -1;
-        float v = 0.f;
-        if (lane < K) {
-            e = idx_to_int(idx[base + lane]);
-            v = gates[base + lane] * (dgates[base + lane] - c);
-        }
-        for (int ch = lane; ch < ((nchunk + 31) & ~31); ch += 32) {
-            float r[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int j = 0; j < K; ++j) {
-                const int ej = __shfl_sync(0xffffffffu, e, j);
-                const float vj = __shfl_sync(0xffffffffu, v, j);
-                if ((ej >> 2) == ch) r[ej & 3] = vj;
+        float gl[NT], dl[NT];
+        int e[NT];
+#pragma unroll
+        for (int a = 0; a < NT; ++a) {
+            gl[a] = 0.f;
+            dl[a] = 0.f;
+            e[a] = -1;
+            if (t0 + a < T && lane < K) {
+                const size_t at = (size_t)(t0 + a) * K + lane;
+                gl[a] = gates[at];
+                dl[a] = dgates[at];
+                e[a] = idx_to_int(idx[at]);
             }
-            if (ch < nchunk) {
-                const int e0 = ch << 2;
-                if (e0 + 3 < E && (E & 3) == 0) {
-                    *reinterpret_cast<float4*>(out + e0) = make_float4(r[0], r[1], r[2], r[3]);
-                } else {
-                    for (int q = 0; q < 4 && e0 + q < E; ++q) out[e0 + q] = r[q];
+        }
+        float v[NT];
+#pragma unroll
+        for (int a = 0; a < NT; ++a) {
+            float c = gl[a] * dl[a];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+            v[a] = gl[a] * (dl[a] - c);
+        }
+#pragma unroll
+        for (int a = 0; a < NT; ++a) {
+            if (t0 + a >= T) break;                       // uniform across the warp
+            float* out = dlogits + (size_t)(t0 + a) * E;
+            for (int ch = lane; ch < ((nchunk + 31) & ~31); ch += 32) {
+                float r[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int j = 0; j < K; ++j) {
+                    const int ej = __shfl_sync(0xffffffffu, e[a], j);
+                    const float vj = __shfl_sync(0xffffffffu, v[a], j);
+                    if ((ej >> 2) == ch) r[ej & 3] = vj;
+                }
+                if (ch < nchunk) {
+                    const int e0 = ch << 2;
+                    if (e0 + 3 < E && (E & 3) == 0) {
+                        *reinterpret_cast<float4*>(out + e0) = make_float4(r[0], r[1], r[2], r[3]);
+                    } else {
+                        for (int q = 0; q < 4 && e0 + q < E; ++q) out[e0 + q] = r[q];
+                    }
                 }
             }
         }
     } else {
         // rare wide-K case: zero the row, then scatter (same warp, ordered by __syncwarp)
-        for (int i = lane; i < E; i += 32) out[i] = 0.f;
-        __syncwarp();
-        for (int j = lane; j < K; j += 32) {
-            const int e = idx_to_int(idx[base + j]);
-            if (e >= 0 && e < E) out[e] = gates[base + j] * (dgates[base + j] - c);
+        for (int a = 0; a < NT && t0 + a < T; ++a) {
+            const size_t base = (size_t)(t0 + a) * K;
+            float* out = dlogits + (size_t)(t0 + a) * E;
+            float c = 0.f;
+            for (int j = lane; j < K; j += 32) c += gates[base + j] * dgates[base + j];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+            for (int i = lane; i < E; i += 32) out[i] = 0.f;
+            __syncwarp();
+            for (int j = lane; j < K; j += 32) {
+                const int e = idx_to_int(idx[base + j]);
+                if (e >= 0 && e < E) out[e] = gates[base + j] * (dgates[base + j] - c);
+            }
         }
     }
 }
@@ -112,6 +183,11 @@ static void launch_gate_fwd(const r3_shape* s, const float* logits, const void* 
     const int block = 256;
     const unsigned grid = (unsigned)((threads + block - 1) / block);
     const IdxT* ip = static_cast<const IdxT*>(idx);
+    if (s->K <= 8) {
+        replay_gate_fwd_lane_kernel<IdxT><<<(unsigned)((s->T + 127) / 128), 128, 0, st>>>(
+            logits, ip, gates, s->T, s->E, s->K, W, dev_status);
+        return;
+    }
 #define R3_GF(WW) replay_gate_fwd_kernel<IdxT, WW><<<grid, block, 0, st>>>( \
         logits, ip, gates, s->T, s->E, s->K, dev_status)
     switch (W) {
@@ -148,7 +224,8 @@ extern "C" r3_status r3_replay_gate_bwd(const r3_shape* shape, const float* gate
     if (!gates || !dgates || !idx || !dlogits) return R3_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int wpb = 8;
-    const unsigned grid = (unsigned)((shape->T + wpb - 1) / wpb);
+    const int tpb = wpb * r3::kGateBwdTokens;               // tokens per block
+    const unsigned grid = (unsigned)((shape->T + tpb - 1) / tpb);
     R3_DISPATCH_IDX(shape, IdxT,
         r3::replay_gate_bwd_kernel<IdxT><<<grid, wpb * 32, 0, cs>>>(
             gates, dgates, static_cast<const IdxT*>(idx), dlogits, shape->T, shape->E, shape->K));

@@ -9,6 +9,12 @@
 // the same fp32 TMEM accumulator: x is exact in bf16, so the logits keep float32-level accuracy
 // while the contraction runs on the tensor pipe.
 //
+// When the tiles are few (a single layer's decode batch, or the training logits of a few thousand
+// tokens: at most half as many tiles as SMs), two CTAs of a cluster share a tile: each contracts
+// half of the k blocks into its own accumulator and finishes half of the tile's tokens, reading
+// the other CTA's partial logits through distributed shared memory (the sum of the two partials is
+// the same number in both CTAs).
+//
 // One CTA of 12 warps per 128-token tile: warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA
 // issuer, warps 2-5 read the finished accumulator out of TMEM into a [128][E + 1] float tile in
 // shared memory (the copy ring is free by then).  All 12 warps then finish tokens out of that
@@ -59,7 +65,8 @@ split_router_weight_kernel(const float* __restrict__ w, __nv_bfloat16* __restric
 template <typename IdxT, int SLOTS, int NT>
 __device__ __forceinline__ void finish_tokens(const float* tile, int LD, const int* rows, int n_rows,
                                               int lane, int E, int K, size_t out_row0,
-                                              IdxT* idx_out, float* logits_out) {
+                                              IdxT* idx_out, float* logits_out,
+                                              uint32_t peer_tile) {
     uint32_t key[NT][SLOTS];
 #pragma unroll
     for (int a = 0; a < NT; ++a) {
@@ -68,7 +75,13 @@ __device__ __forceinline__ void finish_tokens(const float* tile, int LD, const i
             const int e = lane + 32 * sl;
             key[a][sl] = 0u;                             // 0 = no candidate (below every real key)
             if (a < n_rows && e < E) {
-                const float v = tile[(size_t)rows[a] * LD + e];
+                float v = tile[(size_t)rows[a] * LD + e];
+                if (peer_tile) {                         // the other half of the contraction
+                    float w;
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];"
+                                 : "=f"(w) : "r"(peer_tile + 4u * (uint32_t)(rows[a] * LD + e)));
+                    v += w;
+                }
                 if (logits_out) logits_out[(out_row0 + rows[a]) * E + e] = v;
                 const uint32_t u = __float_as_uint(v);
                 const uint32_t k2 = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
@@ -107,7 +120,7 @@ template <typename IdxT, int KM>
 __global__ void __launch_bounds__(THREADS, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                  IdxT* __restrict__ idx_out, float* __restrict__ logits_out, int T, int d, int E,
-                 int K, int planes, int stages, uint32_t tmem_cols) {
+                 int K, int planes, int stages, uint32_t tmem_cols, int ksplit) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -124,8 +137,12 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int layer = blockIdx.y;
-    const int t0 = blockIdx.x * BM;
+    // ksplit = 2: the two CTAs of a cluster (consecutive blockIdx.x) share a tile
+    const int rank = ksplit == 2 ? (int)cluster_ctarank() : 0;
+    const int t0 = (ksplit == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x) * BM;
     const int kblocks = (d + BK - 1) / BK;
+    const int kb_per = (kblocks + ksplit - 1) / ksplit;
+    const int kb0 = rank * kb_per, kb1 = min(kblocks, kb0 + kb_per);    // this CTA's k blocks
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -143,7 +160,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int kb = 0; kb < kblocks; ++kb) {
+            for (int kb = kb0; kb < kb1; ++kb) {
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, nullptr)) break;
                 const uint32_t sa = base + stage * stage_bytes, sb = sa + A_BYTES;
                 mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
@@ -161,7 +178,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int kb = 0; kb < kblocks && ok; ++kb) {
+            for (int kb = kb0; kb < kb1 && ok; ++kb) {
                 if (!mbar_wait(full_bar(stage), phase, abort_flag, nullptr)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t sa = base + stage * stage_bytes, sb = sa + A_BYTES;
@@ -171,12 +188,12 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 #pragma unroll
                     for (int kk = 0; kk < BK / UK; ++kk)
                         tc_mma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
-                                    idesc, (kb | p | kk) != 0 ? 1u : 0u);
+                                    idesc, ((kb - kb0) | p | kk) != 0 ? 1u : 0u);
                 }
                 tc_commit(empty_bar(stage));
                 if (++stage == stages) { stage = 0; phase ^= 1u; }
             }
-            if (ok) tc_commit(acc_bar);
+            if (ok && kb1 > kb0) tc_commit(acc_bar);
         }
         __syncwarp();
     } else if (warp < 6) {
@@ -185,10 +202,12 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         // float tile in shared memory (the copy ring is free once the accumulator is complete)
         const int q = warp & 3;
         float* tile = reinterpret_cast<float*>(base_ptr);
-        if (__all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, nullptr))) {
+        float* trow = tile + (size_t)(q * 32 + lane) * (E + 1);
+        if (kb1 <= kb0) {
+            for (int c = 0; c < E; ++c) trow[c] = 0.f;      // no k block fell to this CTA
+        } else if (__all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, nullptr))) {
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            float* trow = tile + (size_t)(q * 32 + lane) * (E + 1);
             for (int c = 0; c < E; c += 32) {
                 float v[32];
                 tc_ld32(taddr + c, v);
@@ -199,14 +218,19 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             }
         }
     }
-    // ------------------------------ epilogue, part 2: all six warps, a few tokens each ---------
+    // ------------------------------ epilogue, part 2: all twelve warps, a few tokens each -------
     tc_fence_before();
     __syncthreads();
+    if (ksplit == 2) cluster_sync_all();       // the other CTA's partial logits are in its tile
     if (!*abort_flag) {
         const float* tile = reinterpret_cast<const float*>(base_ptr);
-        const int n_tok = min(BM, T - t0);
+        const uint32_t peer_tile = ksplit == 2 ? mapa_shared(smem_u32(tile), (uint32_t)(rank ^ 1)) : 0u;
+        // with a shared tile each CTA finishes half of its tokens
+        const int n_all = min(BM, T - t0);
+        const int tok_lo = ksplit == 2 ? rank * (BM / 2) : 0;
+        const int n_tok = ksplit == 2 ? min(n_all, tok_lo + BM / 2) : n_all;
         constexpr int NT = 4, NW = THREADS / 32;
-        for (int r0 = warp * NT; r0 < n_tok; r0 += NW * NT) {
+        for (int r0 = tok_lo + warp * NT; r0 < n_tok; r0 += NW * NT) {
             int rows[NT];
 #pragma unroll
             for (int a = 0; a < NT; ++a) rows[a] = min(r0 + a, n_tok - 1);
@@ -214,10 +238,10 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             const size_t out_row0 = (size_t)layer * T + t0;
             if (E <= 128)
                 finish_tokens<IdxT, 4, NT>(tile, E + 1, rows, n_rows, lane, E, K, out_row0, idx_out,
-                                           logits_out);
+                                           logits_out, peer_tile);
             else
                 finish_tokens<IdxT, 8, NT>(tile, E + 1, rows, n_rows, lane, E, K, out_row0, idx_out,
-                                           logits_out);
+                                           logits_out, peer_tile);
         }
     }
 
@@ -227,6 +251,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         __syncthreads();
     }
+    if (ksplit == 2) cluster_sync_all();       // the other CTA may still be reading this tile
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
@@ -258,10 +283,21 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
         wplanes = workspace;
     }
     const int stage_bytes = A_BYTES + planes * s->E * BK * 2;
+    const int tiles = (s->T + BM - 1) / BM;
+    const int kblocks = (s->d + BK - 1) / BK;
+    // Few enough tiles that twice as many CTAs still get an SM each: two CTAs of a cluster share
+    // a tile (half of the k blocks and half of the tokens each).  With more tiles than that the
+    // shared form needs two CTAs per SM with half the ring each, which measured slower on the
+    // 48-layer decode batch (29.4 us against 24.7 us).
+    const int ksplit = ((long long)2 * tiles * L <= sm_count() && kblocks >= 2) ? 2 : 1;
     int stages = (SMEM_LIMIT - BAR_BYTES - 1024) / stage_bytes;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
     if (stages < 2) return R3_ERR_UNSUPPORTED;
-    const int smem = stages * stage_bytes + BAR_BYTES + 1024;
+    const int tile_bytes = BM * (s->E + 1) * 4;        // the logits tile re-uses the ring
+    int ring = stages * stage_bytes;
+    if (ring < tile_bytes) ring = (tile_bytes + 1023) & ~1023;
+    if (ring + BAR_BYTES + 1024 > SMEM_LIMIT) return R3_ERR_UNSUPPORTED;
+    const int smem = ring + BAR_BYTES + 1024;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < s->E) tmem_cols <<= 1;
 
@@ -269,7 +305,18 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
     if (!make_map_2d(&mx, x, (uint64_t)L * s->T, (uint64_t)s->d, BM) ||
         !make_map_2d(&mw, wplanes, (uint64_t)L * planes * s->E, (uint64_t)s->d, (uint32_t)s->E))
         return R3_ERR_CUDA;
-    dim3 grid((s->T + BM - 1) / BM, L);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)ksplit;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3((unsigned)(tiles * ksplit), (unsigned)L);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = cs;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
 #define R3_RT(IDX, KM)                                                                          \
     do {                                                                                        \
         auto kern = router_tc_kernel<IDX, KM>;                                                  \
@@ -280,8 +327,10 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
                 return R3_ERR_CUDA;                                                             \
             attr_smem = SMEM_LIMIT;                                                             \
         }                                                                                       \
-        kern<<<grid, THREADS, smem, cs>>>(mx, mw, static_cast<IDX*>(idx_out), logits_out, s->T, \
-                                          s->d, s->E, s->K, planes, stages, tmem_cols);         \
+        if (cudaLaunchKernelEx(&cfg, kern, mx, mw, static_cast<IDX*>(idx_out), logits_out,      \
+                               (int)s->T, (int)s->d, (int)s->E, (int)s->K, planes, stages,      \
+                               tmem_cols, ksplit) != cudaSuccess)                               \
+            return R3_ERR_CUDA;                                                                 \
     } while (0)
     const bool u8 = s->idx_type == R3_IDX_U8;
     if (s->K <= 8) { if (u8) R3_RT(uint8_t, 8); else R3_RT(int16_t, 8); }
