@@ -366,18 +366,39 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
         const float val = g * (dg - cs);
         float* out = dlogits + (size_t)t * E;
         const int nchunk = (E + 3) >> 2;
+        if ((E & 3) == 0 && (size_t)E * sizeof(float) <= (size_t)(K + 1) * row_bytes) {
+            // the row buffers are free now: build the dense row there (zeros, then the K values)
+            // and write it out in 16-byte pieces - a dozen instructions per lane instead of a scan
+            // of the K slots by every lane
+            float* stage = reinterpret_cast<float*>(smem_tok + kTokHeader + 128);
+            for (int ch = lane; ch < nchunk; ch += 32)
+                reinterpret_cast<float4*>(stage)[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
+            __syncwarp();
+            if (lane < K && my_e >= 0 && my_e < E) stage[my_e] = val;
+            __syncwarp();
+            for (int ch = lane; ch < nchunk; ch += 32)
+                reinterpret_cast<float4*>(out)[ch] = reinterpret_cast<const float4*>(stage)[ch];
+        } else
         for (int ch = lane; ch < ((nchunk + 31) & ~31); ch += 32) {
-            float q[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int j = 0; j < K; ++j) {
-                const int ej = __shfl_sync(0xffffffffu, my_e, j);
-                const float vj = __shfl_sync(0xffffffffu, val, j);
-                if ((ej >> 2) == ch) q[ej & 3] = vj;
+            float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;          // selects, no branches
+#pragma unroll
+            for (int j = 0; j < kFusedMaxK; ++j) {
+                if (j < K) {
+                    const int ej = __shfl_sync(0xffffffffu, my_e, j);
+                    const float vj = __shfl_sync(0xffffffffu, val, j);
+                    const int w = (ej >> 2) == ch ? (ej & 3) : -1;
+                    q0 = w == 0 ? vj : q0;
+                    q1 = w == 1 ? vj : q1;
+                    q2 = w == 2 ? vj : q2;
+                    q3 = w == 3 ? vj : q3;
+                }
             }
             if (ch < nchunk) {
                 const int e0 = ch << 2;
                 if ((E & 3) == 0) {
-                    *reinterpret_cast<float4*>(out + e0) = make_float4(q[0], q[1], q[2], q[3]);
+                    *reinterpret_cast<float4*>(out + e0) = make_float4(q0, q1, q2, q3);
                 } else {
+                    const float q[4] = {q0, q1, q2, q3};
                     for (int k2 = 0; k2 < 4 && e0 + k2 < E; ++k2) out[e0 + k2] = q[k2];
                 }
             }

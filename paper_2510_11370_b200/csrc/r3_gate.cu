@@ -105,7 +105,7 @@ template <typename IdxT>
 __global__ void __launch_bounds__(256)
 replay_gate_bwd_kernel(const float* __restrict__ gates, const float* __restrict__ dgates,
                        const IdxT* __restrict__ idx, float* __restrict__ dlogits,
-                       int T, int E, int K) {
+                       int T, int E, int K, bool staged) {
     constexpr int NT = kGateBwdTokens;
     const int lane = threadIdx.x & 31;
     const long long t0 = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * NT;
@@ -134,22 +134,59 @@ replay_gate_bwd_kernel(const float* __restrict__ gates, const float* __restrict_
             for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
             v[a] = gl[a] * (dl[a] - c);
         }
+        if (staged) {
+            // dense rows built in shared memory (zeros, then the K values) and written out in
+            // 16-byte pieces: a dozen instructions per lane and token, where the scan below of
+            // the K slots by every lane made the kernel issue-bound
+            extern __shared__ __align__(16) float stage_all[];
+            float* stage = stage_all + (size_t)(threadIdx.x >> 5) * NT * E;
+#pragma unroll
+            for (int a = 0; a < NT; ++a)
+                for (int ch = lane; ch < nchunk; ch += 32)
+                    reinterpret_cast<float4*>(stage + a * E)[ch] = make_float4(0.f, 0.f, 0.f, 0.f);
+            __syncwarp();
+#pragma unroll
+            for (int a = 0; a < NT; ++a)
+                if (e[a] >= 0 && e[a] < E) stage[a * E + e[a]] = v[a];
+            __syncwarp();
+#pragma unroll
+            for (int a = 0; a < NT; ++a) {
+                if (t0 + a >= T) break;                   // uniform across the warp
+                float4* out = reinterpret_cast<float4*>(dlogits + (size_t)(t0 + a) * E);
+                for (int ch = lane; ch < nchunk; ch += 32)
+                    out[ch] = reinterpret_cast<const float4*>(stage + a * E)[ch];
+            }
+            return;
+        }
 #pragma unroll
         for (int a = 0; a < NT; ++a) {
             if (t0 + a >= T) break;                       // uniform across the warp
             float* out = dlogits + (size_t)(t0 + a) * E;
             for (int ch = lane; ch < ((nchunk + 31) & ~31); ch += 32) {
-                float r[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int j = 0; j < K; ++j) {
+                // selects, no branches: the kernel is bound by instruction issue otherwise
+                float r0 = 0.f, r1 = 0.f, r2 = 0.f, r3 = 0.f;
+                auto place = [&](int j) {
                     const int ej = __shfl_sync(0xffffffffu, e[a], j);
                     const float vj = __shfl_sync(0xffffffffu, v[a], j);
-                    if ((ej >> 2) == ch) r[ej & 3] = vj;
+                    const int q = (ej >> 2) == ch ? (ej & 3) : -1;
+                    r0 = q == 0 ? vj : r0;
+                    r1 = q == 1 ? vj : r1;
+                    r2 = q == 2 ? vj : r2;
+                    r3 = q == 3 ? vj : r3;
+                };
+                if (K <= 8) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < K) place(j);
+                } else {
+                    for (int j = 0; j < K; ++j) place(j);
                 }
                 if (ch < nchunk) {
                     const int e0 = ch << 2;
                     if (e0 + 3 < E && (E & 3) == 0) {
-                        *reinterpret_cast<float4*>(out + e0) = make_float4(r[0], r[1], r[2], r[3]);
+                        *reinterpret_cast<float4*>(out + e0) = make_float4(r0, r1, r2, r3);
                     } else {
+                        const float r[4] = {r0, r1, r2, r3};
                         for (int q = 0; q < 4 && e0 + q < E; ++q) out[e0 + q] = r[q];
                     }
                 }
@@ -226,8 +263,13 @@ extern "C" r3_status r3_replay_gate_bwd(const r3_shape* shape, const float* gate
     const int wpb = 8;
     const int tpb = wpb * r3::kGateBwdTokens;               // tokens per block
     const unsigned grid = (unsigned)((shape->T + tpb - 1) / tpb);
+    // rows staged in shared memory when they are 16-byte pieces and a block's rows fit 32 KB
+    const size_t stage_bytes = (size_t)tpb * shape->E * sizeof(float);
+    const bool staged = shape->K <= 32 && (shape->E & 3) == 0 && stage_bytes <= 32 * 1024 &&
+                        (reinterpret_cast<uintptr_t>(dlogits) & 15) == 0;
     R3_DISPATCH_IDX(shape, IdxT,
-        r3::replay_gate_bwd_kernel<IdxT><<<grid, wpb * 32, 0, cs>>>(
-            gates, dgates, static_cast<const IdxT*>(idx), dlogits, shape->T, shape->E, shape->K));
+        r3::replay_gate_bwd_kernel<IdxT><<<grid, wpb * 32, staged ? stage_bytes : 0, cs>>>(
+            gates, dgates, static_cast<const IdxT*>(idx), dlogits, shape->T, shape->E, shape->K,
+            staged));
     return r3::launch_status();
 }
