@@ -364,3 +364,35 @@ def test_grouped_swiglu_f32(r3, T, d, E, K, F):
 ])
 def test_grouped_swiglu_bf16_tensor_cores(r3, T, d, E, K, F):
     run_swiglu_case(r3, T, d, E, K, F, torch.bfloat16, TOL_BF16)
+
+
+def test_expert_down_twice_from_one_work_list(r3):
+    """The down projection reads the work list the up projection left in the workspace.  Its
+    clusters claim items from a counter in that list; the launch re-arms the counter when it
+    ends, so a second launch from the same list computes every item again.  T and E are chosen
+    so that the list holds several times as many items as there are clusters (most of them are
+    claimed from the counter, not taken by position)."""
+    T, d, E, K, F = 6000, 1024, 24, 4, 264
+    act = torch.bfloat16
+    rng = np.random.default_rng(5)
+    idx_np = np.argsort(-rng.random((T, E)), axis=1)[:, :K]
+    _, offsets, ros, sor = O.permutation(idx_np, E)
+    x = torch.randn(T, d).to(act)
+    wg = (torch.randn(E, F, d) * 0.05).to(act).cuda()
+    wu = (torch.randn(E, F, d) * 0.05).to(act).cuda()
+    wd = (torch.randn(E, d, F) * 0.05).to(act).cuda()
+    xp = x[torch.from_numpy(sor.astype(np.int64)) // K].contiguous().cuda()
+    off = torch.from_numpy(offsets).cuda()
+    s = r3.make_shape(T, d, E, K, F, act=act)
+    st = r3.new_status("cuda")
+    whole = r3.grouped_swiglu(s, xp, off, wg, wu, wd, dev_status=st)
+    ws = r3.workspace(r3.grouped_swiglu_workspace_bytes(s), "cuda")
+    r3.expert_up_swiglu(s, xp, off, wg, wu, ws, dev_status=st)
+    o1 = torch.full((T * K, d), float("nan"), dtype=act, device="cuda")
+    o2 = torch.full((T * K, d), float("nan"), dtype=act, device="cuda")
+    r3.expert_down(s, wd, o1, ws, dev_status=st)
+    r3.expert_down(s, wd, o2, ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert torch.equal(o1, whole)
+    assert torch.equal(o2, whole)
