@@ -400,6 +400,41 @@ def run_ours(args, w):
            "d2h_bytes_per_step": int(yh.numel() * es + dlh.numel() * 4),
            "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps}
 
+    # the same with several batches in flight (r3_replay_layer_host_enqueue): every step still copies
+    # its inputs in and its results out; the copies of one step run beside the kernels of another
+    lanes = []
+    depth = int(os.environ.get("R3_BENCH_E2E_DEPTH", "2"))
+    for _ in range(depth):
+        lanes.append(dict(x=xh.clone().pin_memory(), dy=dyh.clone().pin_memory(),
+                          idx=idxh.clone().pin_memory(),
+                          y=torch.empty_like(yh).pin_memory(), dl=torch.empty_like(dlh).pin_memory(),
+                          ws=r3.workspace(r3.replay_layer_host_workspace_bytes(s), dev),
+                          stream=torch.cuda.Stream(device=dev)))
+    torch.cuda.synchronize()
+
+    def pipelined(n):
+        for i in range(n):
+            ln = lanes[i % depth]
+            r3.replay_layer_host_enqueue(s, ln["x"], w_r, ln["idx"], wg, wu, wd, ln["dy"], ln["y"],
+                                         ln["dl"], ws=ln["ws"], dev_status=st, stream=ln["stream"])
+        for ln in lanes:
+            ln["stream"].synchronize()
+
+    pipelined(2 * depth)
+    r3dist.barrier()
+    torch.cuda.synchronize()
+    tp0 = time.perf_counter()
+    pipelined(e2e_steps)
+    torch.cuda.synchronize()
+    tp1 = time.perf_counter()
+    r3dist.barrier()
+    pipe_ms = r3dist.max_over_ranks((tp1 - tp0) * 1e3, dev)
+    assert st.item() == 0
+    assert all(torch.equal(ln["y"].to(dev), y) for ln in lanes)
+    e2e["batches_in_flight"] = {"depth": depth, "value": world * T * e2e_steps / (pipe_ms * 1e-3), "unit": UNIT,
+                            "ms_per_step": pipe_ms / e2e_steps, "steps": e2e_steps,
+                            "timing": "host clock around the enqueues and the synchronisation of every stream"}
+
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
     # ---- the oracle on this machine's host cores (rank 0, single-GPU runs only) ---------------------

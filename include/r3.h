@@ -281,6 +281,19 @@ r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host, const 
                                const void* w_down, const void* dy_host, void* y_host,
                                float* dlogits_host, void* workspace, size_t ws_bytes,
                                int32_t* dev_status, void* stream);
+/* The same without the final synchronisation: copies in, layer and copies out are enqueued on
+ * `stream` and the call returns.  y_host and dlogits_host hold the result once the caller has
+ * synchronised the stream; the host buffers and the workspace must stay untouched until then
+ * (pageable host memory makes the copies synchronous: use pinned memory).  A caller that feeds a
+ * sequence of batches keeps two or more of them in flight, each with its own stream, workspace and
+ * host buffers: the copies of one batch then run beside the kernels of another.  Errors as
+ * r3_replay_layer_host. */
+r3_status r3_replay_layer_host_enqueue(const r3_shape* shape, const void* x_host,
+                                       const void* w_router, const void* idx_host,
+                                       const void* w_gate, const void* w_up, const void* w_down,
+                                       const void* dy_host, void* y_host, float* dlogits_host,
+                                       void* workspace, size_t ws_bytes, int32_t* dev_status,
+                                       void* stream);
 
 /* ---- Update-stage backward to the layer input (Section 4.1, purpose (b)) ------------------------ */
 

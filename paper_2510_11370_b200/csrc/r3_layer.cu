@@ -435,12 +435,13 @@ extern "C" size_t r3_replay_layer_host_workspace_bytes(const r3_shape* shape) {
     return r3::carve_host(shape, nullptr).total;
 }
 
-extern "C" r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host,
-                                          const void* w_router, const void* idx_host,
-                                          const void* w_gate, const void* w_up,
-                                          const void* w_down, const void* dy_host, void* y_host,
-                                          float* dlogits_host, void* workspace, size_t ws_bytes,
-                                          int32_t* dev_status, void* stream) {
+extern "C" r3_status r3_replay_layer_host_enqueue(const r3_shape* shape, const void* x_host,
+                                                  const void* w_router, const void* idx_host,
+                                                  const void* w_gate, const void* w_up,
+                                                  const void* w_down, const void* dy_host,
+                                                  void* y_host, float* dlogits_host,
+                                                  void* workspace, size_t ws_bytes,
+                                                  int32_t* dev_status, void* stream) {
     r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
     if (shape->T == 0) return R3_OK;
@@ -478,7 +479,21 @@ extern "C" r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_h
         cudaMemcpyAsync(dlogits_host, h.dlogits, T * shape->E * 4, cudaMemcpyDeviceToHost, cs) !=
             cudaSuccess)
         return R3_ERR_CUDA;
-    return cudaStreamSynchronize(cs) == cudaSuccess ? R3_OK : R3_ERR_CUDA;
+    return R3_OK;
+}
+
+extern "C" r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host,
+                                          const void* w_router, const void* idx_host,
+                                          const void* w_gate, const void* w_up,
+                                          const void* w_down, const void* dy_host, void* y_host,
+                                          float* dlogits_host, void* workspace, size_t ws_bytes,
+                                          int32_t* dev_status, void* stream) {
+    const r3_status st = r3_replay_layer_host_enqueue(shape, x_host, w_router, idx_host, w_gate,
+                                                      w_up, w_down, dy_host, y_host, dlogits_host,
+                                                      workspace, ws_bytes, dev_status, stream);
+    if (st != R3_OK || shape->T == 0) return st;
+    return cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) == cudaSuccess ? R3_OK
+                                                                                   : R3_ERR_CUDA;
 }
 
 extern "C" const char* r3_status_string(r3_status s) {

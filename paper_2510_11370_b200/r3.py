@@ -36,7 +36,7 @@ EXPORTS = [
     "r3_combine_residual", "r3_combine_bwd_gates", "r3_replay_finish",
     "r3_replay_layer_workspace_bytes",
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
-    "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host",
+    "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host", "r3_replay_layer_host_enqueue",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
     "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
     "r3_grouped_swiglu_bwd", "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
@@ -102,6 +102,7 @@ lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_finish.argtypes = [_SP] + [_P] * 11
 lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_layer_host.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
+lib.r3_replay_layer_host_enqueue.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 lib.r3_prob_discrepancy_workspace_bytes.restype = ctypes.c_size_t
 lib.r3_prob_discrepancy_workspace_bytes.argtypes = [ctypes.c_int64]
 lib.r3_prob_discrepancy.argtypes = [_P, _P, ctypes.c_int64, _P, ctypes.c_int32, _P, _P, _P,
@@ -457,6 +458,18 @@ def replay_layer_host(s: Shape, x_host, w_router, idx_host, w_gate, w_up, w_down
                                     _ptr(dy_host, True), _ptr(y_host, True),
                                     _ptr(dlogits_host, True), _ptr(ws), ws.numel(),
                                     _ptr(dev_status), _stream(stream)))
+    return y_host, dlogits_host
+
+
+def replay_layer_host_enqueue(s: Shape, x_host, w_router, idx_host, w_gate, w_up, w_down, dy_host,
+                              y_host, dlogits_host, *, ws, dev_status=None, stream=None):
+    """As replay_layer_host without the final synchronisation: the result is in y_host and
+    dlogits_host once `stream` has been synchronised."""
+    _check(lib.r3_replay_layer_host_enqueue(ctypes.byref(s), _ptr(x_host, True), _ptr(w_router),
+                                            _ptr(idx_host, True), _ptr(w_gate), _ptr(w_up),
+                                            _ptr(w_down), _ptr(dy_host, True), _ptr(y_host, True),
+                                            _ptr(dlogits_host, True), _ptr(ws), ws.numel(),
+                                            _ptr(dev_status), _stream(stream)))
     return y_host, dlogits_host
 
 

@@ -2,6 +2,8 @@
 on the benchmark configurations.  Small configurations are compared element by element; the
 large ones compare all integer work and the gates exactly/fully, and the expert-dependent
 outputs on sampled tokens that the oracle evaluates one by one."""
+import copy
+
 import numpy as np
 import pytest
 import torch
@@ -221,3 +223,46 @@ def test_config4_capture_then_replay_round_trip(r3):
                                    case.w_gate, case.w_up, case.w_down, f64(case.dy[sel]))
     assert np.abs(f64(y)[sel] - y_ref).max() / np.abs(y_ref).max() < TOL_BF16
     assert np.abs(f64(ds)[sel] - ds_ref).max() / np.abs(ds_ref).max() < TOL_BF16
+
+
+def test_host_buffer_layer_and_two_batches_in_flight(r3):
+    """r3_replay_layer_host gives the device path's bits, and r3_replay_layer_host_enqueue with two
+    batches in flight (own stream, workspace and pinned buffers each) gives, for each batch, the
+    bits of running it alone."""
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], T=1000)
+    cases = [Case(w, device="cuda")]
+    cases.append(copy.copy(cases[0]))
+    cases[1].x = cases[1].x.flip(0).contiguous()          # a second batch with other rows
+    cases[1].dy = cases[1].dy.flip(0).contiguous()
+    cases[1].idx = cases[1].idx.flip(0).contiguous()
+    s = r3.shape_of(w)
+    st = r3.new_status("cuda")
+    dev = {k: getattr(cases[0], k).cuda() for k in ("w_r", "w_gate", "w_up", "w_down")}
+    alone, bufs = [], []
+    for c in cases:
+        y, ds, _ = r3.replay_layer(s, c.x.cuda(), dev["w_r"], c.idx.cuda(), dev["w_gate"],
+                                   dev["w_up"], dev["w_down"], c.dy.cuda(), dev_status=st)
+        torch.cuda.synchronize()
+        alone.append((y.cpu(), ds.cpu()))
+        bufs.append(dict(x=c.x.pin_memory(), dy=c.dy.pin_memory(), idx=c.idx.pin_memory(),
+                         y=torch.empty((w.T, w.d), dtype=c.x.dtype).pin_memory(),
+                         ds=torch.empty((w.T, w.E), dtype=torch.float32).pin_memory(),
+                         ws=r3.workspace(r3.replay_layer_host_workspace_bytes(s), "cuda"),
+                         stream=torch.cuda.Stream()))
+    b = bufs[0]
+    r3.replay_layer_host(s, b["x"], dev["w_r"], b["idx"], dev["w_gate"], dev["w_up"], dev["w_down"],
+                         b["dy"], b["y"], b["ds"], ws=b["ws"], dev_status=st)
+    assert torch.equal(b["y"], alone[0][0]) and torch.equal(b["ds"], alone[0][1])
+    for rounds in range(3):
+        for b in bufs:
+            b["y"].zero_()
+            b["ds"].zero_()
+        for b in bufs:
+            r3.replay_layer_host_enqueue(s, b["x"], dev["w_r"], b["idx"], dev["w_gate"],
+                                         dev["w_up"], dev["w_down"], b["dy"], b["y"], b["ds"],
+                                         ws=b["ws"], dev_status=st, stream=b["stream"])
+        for b in bufs:
+            b["stream"].synchronize()
+        for b, (y, ds) in zip(bufs, alone):
+            assert torch.equal(b["y"], y) and torch.equal(b["ds"], ds)
+    assert st.item() == 0
