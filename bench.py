@@ -360,10 +360,15 @@ def run_ours(args, w):
     # dominant kernel: the up-projection grouped GEMM (4 R d F of the 6 R d F expert FLOPs).
     # Its events bracket the call, which also holds the one-CTA tile-list kernel (a few us).
     achieved = flops["expert_up_swiglu"] / (seg_ms["expert_up_swiglu"] * 1e-3) / 1e12
+    # a timed region of a quarter second or more runs under the power cap like the sustained
+    # matmul loop of the peak measurement; a shorter one is a burst
+    long_run = ms_total >= 250.0
+    peak = peaks["bf16_tflops_sustained"] if long_run else peaks["bf16_tflops"]
     roofline = {"bound": "tensor", "kernel": "grouped_gemm_pair_kernel<0> (gate/up + SwiGLU)",
-                "achieved": round(achieved, 2), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": round(achieved / peaks["bf16_tflops"], 4),
-                "peak_kind": f"bf16 matmul burst, {peaks['source']}",
+                "achieved": round(achieved, 2), "peak": peak, "unit": "TFLOP/s",
+                "frac": round(achieved / peak, 4),
+                "peak_kind": f"bf16 matmul {'sustained' if long_run else 'burst'}, {peaks['source']}",
+                "frac_of_burst": round(achieved / peaks["bf16_tflops"], 4),
                 "frac_of_sustained": round(achieved / peaks["bf16_tflops_sustained"], 4),
                 "frac_of_nominal_2250": round(achieved / 2250.0, 4),
                 "traffic": GEMM_UP_DRAM_TRAFFIC_BYTES if wk.name == "c2_layer_bf16" else None}
@@ -870,8 +875,10 @@ def run_diag(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default: 1000 for the one-layer step, so that the clock "
+                         "sampler sees the timed region; 50 for the other modes)")
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_layer_bf16")
     ap.add_argument("--ref-tokens", type=int, default=4096,
@@ -887,6 +894,10 @@ def main():
                     help="time forward + the whole backward of one layer (bf16 workloads)")
     args = ap.parse_args()
     from paper_2510_11370_b200 import synth
+    if args.steps is None:
+        plain = (args.impl == "ours" and args.workload == "c2_layer_bf16" and not
+                 (args.ep or args.ep_direct or args.stack or args.train))
+        args.steps = 1000 if plain else 50
     if args.workload == "diag":
         return run_diag(args)
     w = synth.WORKLOADS[args.workload]
