@@ -357,6 +357,15 @@ def run_ours(args, w):
             ent["tflops"] = round(flops[n] / (seg_ms[n] * 1e-3) / 1e12, 1)
         kernels[n] = ent
 
+    # the row copy alone: the dispatch with rows minus the maps-only dispatch (the maps are a
+    # latency-bound 16-CTA launch; the copy moves all of the dispatch's bytes but 72 per token)
+    rows_ms = seg_ms["permute"] - seg_ms["permute_maps"]
+    if rows_ms > 0:
+        rows_gbs = T * (d * es + K * 4 + K * d * es) / (rows_ms * 1e-3) / 1e9
+        kernels["permute_rows"] = {"ms": round(rows_ms, 5), "hbm_gbs": round(rows_gbs, 1),
+                                   "frac_of_measured_hbm": round(rows_gbs / peaks["hbm_gbs"], 3),
+                                   "derived": "permute - permute_maps"}
+
     # dominant kernel: the up-projection grouped GEMM (4 R d F of the 6 R d F expert FLOPs).
     # Its events bracket the call, which also holds the one-CTA tile-list kernel (a few us).
     achieved = flops["expert_up_swiglu"] / (seg_ms["expert_up_swiglu"] * 1e-3) / 1e12
