@@ -253,31 +253,34 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
                 if (r >= 0) src_row = o + (size_t)r * d;
             }
         }
-        float s = -INFINITY;
-        if (lane < K) s = lrow[min(max(my_e, 0), E - 1)];      // in flight while the rows are asked for
         // ---- ask for the rows ---------------------------------------------------------------------
+        // dy and the residual row do not wait for the row numbers: their copies start at once
+        // (bytes may land before the barrier is told how many to expect; its one pending
+        // arrival, the expect_tx below, keeps the phase open until then)
         if (lane == 0) {
             tc::mbar_init(bar, 1);
             flags[0] = 0;
             tc::fence_barrier_init();
         }
-        const unsigned have = __ballot_sync(0xffffffffu, r >= 0);
         __syncwarp();
         const uint32_t s_rows = tc::smem_u32(orow);
-        if (lane == 0) {
-            *have_s = have;
-            tc::mbar_expect_tx(bar, row_bytes * (uint32_t)(__popc(have) + 1 + (residual ? 1 : 0)));
-        }
-        __syncwarp();
-        if (lane < K) {
-            if (r >= 0) bulk_load(s_rows + (uint32_t)lane * row_bytes, src_row, row_bytes, bar);
-        } else if (lane == K) {
+        if (lane == K) {
             bulk_load(s_rows + (uint32_t)K * row_bytes, dy + (size_t)t * d, row_bytes, bar);
         } else if (lane == K + 1) {
             if (residual)
                 bulk_load(s_rows + (uint32_t)(K + 1) * row_bytes, residual + (size_t)t * d,
                           row_bytes, bar);
         }
+        float s = -INFINITY;
+        if (lane < K) s = lrow[min(max(my_e, 0), E - 1)];      // in flight while the rows are asked for
+        const unsigned have = __ballot_sync(0xffffffffu, r >= 0);
+        if (lane == 0) {
+            *have_s = have;
+            tc::mbar_expect_tx(bar, row_bytes * (uint32_t)(__popc(have) + 1 + (residual ? 1 : 0)));
+        }
+        __syncwarp();
+        if (lane < K && r >= 0)
+            bulk_load(s_rows + (uint32_t)lane * row_bytes, src_row, row_bytes, bar);
         // ---- replay gate while the copies fly: the first W lanes, one slot each -----------------
         int bad = 0;
         if (lane < K && (my_e < 0 || my_e >= E)) bad |= 1;
