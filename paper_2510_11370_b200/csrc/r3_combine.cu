@@ -169,6 +169,11 @@ gather_staged_kernel(const ActT* __restrict__ o, const int32_t* __restrict__ row
     const bool has_res = DO_Y && residual != nullptr;
     const int extra_dy = K, extra_res = K + (DO_DG ? 1 : 0);     // row slots after the K rows
 
+    // the token's gates are read while the copies fly, not after them
+    float gj[kStageMaxK];
+#pragma unroll
+    for (int u = 0; u < kStageMaxK; ++u) gj[u] = (DO_Y && u < K) ? gates[(size_t)t * K + u] : 0.f;
+
     if (warp == 0) {
         int32_t r = -1;
         if (lane < K) r = row_of_slot[(size_t)t * K + lane];
@@ -177,25 +182,26 @@ gather_staged_kernel(const ActT* __restrict__ o, const int32_t* __restrict__ row
             flags[0] = 0;
             tc::fence_barrier_init();
         }
-        const unsigned have = __ballot_sync(0xffffffffu, r >= 0);
         __syncwarp();
         const uint32_t s_rows = tc::smem_u32(orow);
-        if (lane == 0) {
-            *have_s = have;
-            tc::mbar_expect_tx(bar, row_bytes * (uint32_t)(__popc(have) + (DO_DG ? 1 : 0) +
-                                                           (has_res ? 1 : 0)));
-        }
-        __syncwarp();
-        if (lane < K) {
-            if (r >= 0)
-                bulk_row_load(s_rows + (uint32_t)lane * row_bytes, o + (size_t)r * d, row_bytes, bar);
-        } else if (DO_DG && lane == K) {
+        // dy and the residual row do not wait for the row numbers (bytes may land before the
+        // barrier is told how many to expect: its one pending arrival keeps the phase open)
+        if (DO_DG && lane == K) {
             bulk_row_load(s_rows + (uint32_t)extra_dy * row_bytes, dy + (size_t)t * d, row_bytes, bar);
         } else if (lane == K + 1) {
             if (has_res)
                 bulk_row_load(s_rows + (uint32_t)extra_res * row_bytes, residual + (size_t)t * d,
                               row_bytes, bar);
         }
+        const unsigned have = __ballot_sync(0xffffffffu, r >= 0);
+        if (lane == 0) {
+            *have_s = have;
+            tc::mbar_expect_tx(bar, row_bytes * (uint32_t)(__popc(have) + (DO_DG ? 1 : 0) +
+                                                           (has_res ? 1 : 0)));
+        }
+        __syncwarp();
+        if (lane < K && r >= 0)
+            bulk_row_load(s_rows + (uint32_t)lane * row_bytes, o + (size_t)r * d, row_bytes, bar);
         // one thread waits for the copies; the others sleep at the barrier below
         if (lane == 0) flags[1] = tc::mbar_wait(bar, 0u, flags, nullptr) ? 1 : 0;
     }
@@ -207,9 +213,6 @@ gather_staged_kernel(const ActT* __restrict__ o, const int32_t* __restrict__ row
     for (int u = 0; u < kStageMaxK; ++u) dacc[u] = 0.f;
     if (ready) {
         const unsigned have = *have_s;
-        float gj[kStageMaxK];
-#pragma unroll
-        for (int u = 0; u < kStageMaxK; ++u) gj[u] = (DO_Y && u < K) ? gates[(size_t)t * K + u] : 0.f;
         for (int c = tid; c < row_vecs; c += kStageThreads) {
             float gr[N], acc[N];
             if (DO_DG) orow[(size_t)extra_dy * row_vecs + c].unpack(gr);

@@ -470,13 +470,17 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
             ::"r"(rows0 + (uint32_t)lane * row_bytes), "l"(x + (size_t)(t0 + lane) * row_bytes),
               "r"(row_bytes), "r"(bar) : "memory");
     int32_t r[8];
-    // destination rows of this lane's token (fetched while the copy flies); K > 8 goes in rounds
+    // destination rows of this lane's token, fetched while the copy flies; K > 8 goes in rounds
+    const int32_t* rows = row_of_slot + (size_t)(t0 + (lane < nt ? lane : 0)) * K;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) r[u] = (lane < nt && u < K) ? rows[u] : -1;
     const bool ok = __all_sync(0xffffffffu, tc::mbar_wait(bar, 0u, flags, nullptr));
     if (ok && lane < nt) {
-        const int32_t* rows = row_of_slot + (size_t)(t0 + lane) * K;
         for (int j0 = 0; j0 < K; j0 += 8) {
+            if (j0 > 0) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) r[u] = j0 + u < K ? rows[j0 + u] : -1;
+                for (int u = 0; u < 8; ++u) r[u] = j0 + u < K ? rows[j0 + u] : -1;
+            }
 #pragma unroll
             for (int u = 0; u < 8; ++u)
                 if (r[u] >= 0)
