@@ -246,6 +246,21 @@ r3_status r3_replay_layer(const r3_shape* shape, const void* x, const void* w_ro
                           const void* w_down, const void* dy, void* y, float* dlogits,
                           float* gates_out, void* workspace, size_t ws_bytes,
                           int32_t* dev_status, void* stream);
+/* The same layer for another pass over the SAME record: the rollout's record is replayed in the
+ * Recompute stage and again in the Update stage (Section 5.1, settings of the method; Section 6.3),
+ * so the dispatch (counts, offsets, both maps) and the expert
+ * work lists that the preceding r3_replay_layer call left in `workspace` still hold; this call
+ * copies the rows of the new x with those maps and skips the dispatch.  `workspace` must be the
+ * one that call used, untouched since, with the same shape and the same idx (idx is still read:
+ * the gate needs it); x, the weights and dy may differ.  Results are bit-identical to
+ * r3_replay_layer on the same arguments.  Passing a workspace that holds no such dispatch gives
+ * undefined results (rows are copied to whatever row numbers it holds: call r3_replay_layer
+ * first). */
+r3_status r3_replay_layer_same_record(const r3_shape* shape, const void* x, const void* w_router,
+                          const void* idx, const void* w_gate, const void* w_up,
+                          const void* w_down, const void* dy, void* y, float* dlogits,
+                          float* gates_out, void* workspace, size_t ws_bytes,
+                          int32_t* dev_status, void* stream);
 
 /* L independent replayed MoE blocks enqueued back to back: block l is r3_replay_layer on its own
  * input x[l], record idx[l], weights and upstream gradient dy[l] (a model's MoE blocks with the

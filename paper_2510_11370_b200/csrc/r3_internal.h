@@ -30,8 +30,10 @@ r3_status launch_build_tiles(const int32_t* offsets, int E, int BM, int32_t* til
 // tc_work_bytes() of scratch for the two device-built work lists (the up phase builds both from
 // `offsets`; the down phase reads the list the up phase left there).
 size_t tc_work_bytes(const r3_shape* shape);
-// phases: bit 0 = gate/up projections + SwiGLU (xp -> h), bit 1 = down projection (h -> o).
-enum { kPhaseUp = 1, kPhaseDown = 2 };
+// phases: bit 0 = gate/up projections + SwiGLU (xp -> h), bit 1 = down projection (h -> o),
+// bit 2 = the work lists in `work` were built by an earlier call from the same offsets: the up
+// phase does not build them again.
+enum { kPhaseUp = 1, kPhaseDown = 2, kPhaseKeepLists = 4 };
 // pre_gate / pre_up (optional, [R,F] bf16): the up phase also stores xp W_gate^T and xp W_up^T.
 // Token operand of the up projection: either the permuted rows `xp` [R, d], or (xp == nullptr) the
 // un-permuted activations `x` [T, d] gathered in place through `slot_of_row` [R].
@@ -66,6 +68,17 @@ bool router_tc_supported(const r3_shape* shape);
 size_t router_tc_workspace_bytes(const r3_shape* shape, int L);
 r3_status launch_router_tc(const r3_shape* shape, int L, const void* x, const void* w_router,
                            void* idx_out, float* logits_out, void* workspace, cudaStream_t stream);
+
+// r3_grouped_swiglu (with pre_gate / pre_up: r3_grouped_swiglu_train) on a workspace whose work
+// lists an earlier call built from the same offsets.
+r3_status grouped_swiglu_keep_lists(const r3_shape* shape, const void* xp, const int32_t* offsets,
+                                    const void* w_gate, const void* w_up, const void* w_down,
+                                    void* o, void* pre_gate, void* pre_up, void* workspace,
+                                    size_t ws_bytes, int32_t* dev_status, void* stream);
+
+// The row copy of the dispatch alone: xp[row_of_slot[t, j]] = x[t] (maps from an earlier r3_permute).
+r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_t* row_of_slot,
+                              void* xp, cudaStream_t stream);
 
 // Number of SMs of the current device (cached).
 int sm_count();

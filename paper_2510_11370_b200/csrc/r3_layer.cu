@@ -4,6 +4,7 @@
 #include <mutex>
 
 #include "r3_common.cuh"
+#include "r3_internal.h"
 
 namespace r3 {
 
@@ -102,7 +103,8 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
                            const void* w_down, const void* dy, const void* residual, void* y,
                            float* dlogits, float* gates_out, void* workspace,
                            int32_t* dev_status, void* stream, cudaEvent_t dy_ready = nullptr,
-                           void* pre_gate = nullptr, void* pre_up = nullptr) {
+                           void* pre_gate = nullptr, void* pre_up = nullptr,
+                           bool same_record = false) {
     const LayerWs w = carve(shape, workspace);
     float* gates = gates_out ? gates_out : w.gates;
     r3_status st;
@@ -125,14 +127,22 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
         if ((st = r3_replay_gate_fwd(shape, w.logits, idx, gates, dev_status, stream)) != R3_OK)
             return st;
     }
-    if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row, w.xp,
-                         w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
-        return st;
-    st = pre_gate ? r3_grouped_swiglu_train(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
-                                            pre_gate, pre_up, w.swiglu_ws, w.swiglu_bytes,
-                                            dev_status, stream)
-                  : r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
-                                      w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
+    if (same_record) {
+        // the maps and the GEMM work lists of the previous call on this workspace still hold:
+        // only the rows are copied again
+        if ((st = launch_permute_rows(shape, x, w.row_of_slot, w.xp, cs)) != R3_OK) return st;
+        st = grouped_swiglu_keep_lists(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, pre_gate,
+                                       pre_up, w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
+    } else {
+        if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row,
+                             w.xp, w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
+            return st;
+        st = pre_gate ? r3_grouped_swiglu_train(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
+                                                pre_gate, pre_up, w.swiglu_ws, w.swiglu_bytes,
+                                                dev_status, stream)
+                      : r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
+                                          w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
+    }
     if (st != R3_OK) return st;
     if (fused && side && cudaStreamWaitEvent(cs, side->join, 0) != cudaSuccess) return R3_ERR_CUDA;
     // dy is first needed here (host-buffer entry point: it may still be on its way)
@@ -163,6 +173,25 @@ extern "C" r3_status r3_replay_layer(const r3_shape* shape, const void* x, const
         return R3_ERR_WORKSPACE;
     return r3::run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y, dlogits,
                          gates_out, workspace, dev_status, stream);
+}
+
+extern "C" r3_status r3_replay_layer_same_record(const r3_shape* shape, const void* x,
+                                                 const void* w_router, const void* idx,
+                                                 const void* w_gate, const void* w_up,
+                                                 const void* w_down, const void* dy, void* y,
+                                                 float* dlogits, float* gates_out, void* workspace,
+                                                 size_t ws_bytes, int32_t* dev_status,
+                                                 void* stream) {
+    r3_status st = r3::check_shape(shape);
+    if (st != R3_OK) return st;
+    if (shape->T == 0) return R3_OK;
+    if (!x || !w_router || !idx || !w_gate || !w_up || !w_down || !dy || !y || !dlogits)
+        return R3_ERR_INVALID_ARG;
+    if (!workspace || !r3::aligned(workspace, 256) ||
+        ws_bytes < r3_replay_layer_workspace_bytes(shape))
+        return R3_ERR_WORKSPACE;
+    return r3::run_layer(shape, x, w_router, idx, w_gate, w_up, w_down, dy, nullptr, y, dlogits,
+                         gates_out, workspace, dev_status, stream, nullptr, nullptr, nullptr, true);
 }
 
 // ---- forward plus the backward to the layer input and the router weight ------------------------

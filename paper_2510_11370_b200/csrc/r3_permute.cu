@@ -498,6 +498,30 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
     }
 }
 
+r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_t* row_of_slot,
+                              void* xp, cudaStream_t cs) {
+    const int T = shape->T, K = shape->K;
+    const size_t row_bytes = (size_t)shape->d * act_bytes(shape);
+    if (row_bytes * kRowTokens <= 96 * 1024) {
+        const size_t smem = 128 + row_bytes * kRowTokens;
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaFuncSetAttribute(permute_rows_staged_kernel,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, 128 + 96 * 1024);
+            attr_set = true;
+        }
+        permute_rows_staged_kernel<<<(T + kRowTokens - 1) / kRowTokens, 32, smem, cs>>>(
+            static_cast<const uint8_t*>(x), row_of_slot, static_cast<uint8_t*>(xp), T, K,
+            (uint32_t)row_bytes);
+        return launch_status();
+    }
+    const int row_vecs = (int)(row_bytes / 16);
+    const int wpb = 8;
+    permute_rows_kernel<16><<<(T + wpb - 1) / wpb, wpb * 32, 0, cs>>>(
+        static_cast<const uint4*>(x), row_of_slot, static_cast<uint4*>(xp), T, K, row_vecs);
+    return launch_status();
+}
+
 }  // namespace r3
 
 extern "C" size_t r3_permute_workspace_bytes(const r3_shape* shape) {
@@ -610,26 +634,7 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
             static_cast<const IdxT*>(idx), chunk_counts, offsets, row_of_slot, slot_of_row,
             T, E, K, NB));
     }
-    if (x) {
-        const size_t row_bytes = (size_t)shape->d * r3::act_bytes(shape);
-        if (row_bytes * r3::kRowTokens <= 96 * 1024) {
-            const size_t smem = 128 + row_bytes * r3::kRowTokens;
-            static bool attr_set = false;
-            if (!attr_set) {
-                cudaFuncSetAttribute(r3::permute_rows_staged_kernel,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, 128 + 96 * 1024);
-                attr_set = true;
-            }
-            r3::permute_rows_staged_kernel<<<(T + r3::kRowTokens - 1) / r3::kRowTokens, 32, smem, cs>>>(
-                static_cast<const uint8_t*>(x), row_of_slot, static_cast<uint8_t*>(xp), T, K,
-                (uint32_t)row_bytes);
-            return r3::launch_status();
-        }
-        const int row_vecs = (int)(row_bytes / 16);
-        const int wpb = 8;
-        r3::permute_rows_kernel<16><<<(T + wpb - 1) / wpb, wpb * 32, 0, cs>>>(
-            static_cast<const uint4*>(x), row_of_slot, static_cast<uint4*>(xp), T, K, row_vecs);
-    }
+    if (x) return r3::launch_permute_rows(shape, x, row_of_slot, xp, cs);
     return r3::launch_status();
 }
 

@@ -207,11 +207,20 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const void* 
     if (shape->act_dtype == R3_BF16)
         return launch_grouped_swiglu_tc(shape, xp, x, slot_of_row, offsets, w_gate, w_up, w_down,
                                         h, o, tiles, dev_status, phases, cs, pre_gate, pre_up);
-    if (up) {
+    if (up && !(phases & kPhaseKeepLists)) {
         st = launch_build_tiles(offsets, shape->E, SBM, tiles, cs);
         if (st != R3_OK) return st;
     }
     return launch_grouped_swiglu_f32(shape, xp, tiles, w_gate, w_up, w_down, h, o, phases, cs);
+}
+
+r3_status grouped_swiglu_keep_lists(const r3_shape* shape, const void* xp, const int32_t* offsets,
+                                    const void* w_gate, const void* w_up, const void* w_down,
+                                    void* o, void* pre_gate, void* pre_up, void* workspace,
+                                    size_t ws_bytes, int32_t* dev_status, void* stream) {
+    return run_experts(shape, xp, nullptr, nullptr, offsets, w_gate, w_up, w_down, o, workspace,
+                       ws_bytes, dev_status, kPhaseUp | kPhaseDown | kPhaseKeepLists, stream,
+                       pre_gate, pre_up);
 }
 }  // namespace r3
 

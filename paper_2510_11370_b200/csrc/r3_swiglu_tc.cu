@@ -740,7 +740,8 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
                                                 list_bytes(R, s->E, nf0));
     static TokenMapCache cache_xp, cache_h;
     if (phases & kPhaseUp) {
-        build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1, pairs);
+        if (!(phases & kPhaseKeepLists))
+            build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1, pairs);
         PairMaps m;
         if (!make_map_3d(&m.a0, w_gate, s->E, s->F, s->d, BMF / 2) ||
             !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2))

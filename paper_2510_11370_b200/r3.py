@@ -37,6 +37,7 @@ EXPORTS = [
     "r3_replay_layer_workspace_bytes",
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host", "r3_replay_layer_host_enqueue",
+    "r3_replay_layer_same_record",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
     "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
     "r3_grouped_swiglu_bwd", "r3_grouped_swiglu_train", "r3_scale_rows", "r3_input_grad_finish",
@@ -101,6 +102,7 @@ lib.r3_replay_stack.argtypes = [_SP, ctypes.c_int32] + [_P] * 10 + [ctypes.c_siz
 lib.r3_combine_bwd_gates.argtypes = [_SP, _P, _P, _P, _P, _P]
 lib.r3_replay_finish.argtypes = [_SP] + [_P] * 11
 lib.r3_replay_layer.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
+lib.r3_replay_layer_same_record.argtypes = [_SP] + [_P] * 11 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_layer_host.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 lib.r3_replay_layer_host_enqueue.argtypes = [_SP] + [_P] * 10 + [ctypes.c_size_t, _P, _P]
 lib.r3_prob_discrepancy_workspace_bytes.restype = ctypes.c_size_t
@@ -443,6 +445,24 @@ def replay_layer(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, y=None
                                _ptr(w_up), _ptr(w_down), _ptr(dy), _ptr(y), _ptr(dlogits),
                                _ptr(gates), _ptr(ws), ws.numel(), _ptr(dev_status),
                                _stream(stream)))
+    return y, dlogits, gates
+
+
+def replay_layer_same_record(s: Shape, x, w_router, idx, w_gate, w_up, w_down, dy, *, ws, y=None,
+                             dlogits=None, gates=None, dev_status=None, stream=None):
+    """replay_layer for another pass over the record of the preceding replay_layer call on `ws`:
+    the dispatch and the expert work lists left there are used again."""
+    dev = _dev(x)
+    if y is None:
+        y = torch.empty((s.T, s.d), dtype=_act_dtype(s), device=dev)
+    if dlogits is None:
+        dlogits = torch.empty((s.T, s.E), dtype=torch.float32, device=dev)
+    if gates is None:
+        gates = torch.empty((s.T, s.K), dtype=torch.float32, device=dev)
+    _check(lib.r3_replay_layer_same_record(ctypes.byref(s), _ptr(x), _ptr(w_router), _ptr(idx),
+                                           _ptr(w_gate), _ptr(w_up), _ptr(w_down), _ptr(dy),
+                                           _ptr(y), _ptr(dlogits), _ptr(gates), _ptr(ws),
+                                           ws.numel(), _ptr(dev_status), _stream(stream)))
     return y, dlogits, gates
 
 

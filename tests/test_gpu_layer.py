@@ -266,3 +266,32 @@ def test_host_buffer_layer_and_two_batches_in_flight(r3):
         for b, (y, ds) in zip(bufs, alone):
             assert torch.equal(b["y"], y) and torch.equal(b["ds"], ds)
     assert st.item() == 0
+
+
+@pytest.mark.parametrize("name,T", [("c1_tiny_fp32", 512), ("c2_layer_bf16", 1500)])
+def test_second_pass_over_the_same_record(r3, name, T):
+    """r3_replay_layer_same_record uses the dispatch and the work lists that r3_replay_layer left
+    in the workspace: with new activations, new upstream gradient and scaled weights (the Update
+    stage after the Recompute stage) it gives the bits of a fresh r3_replay_layer call."""
+    w = synth.scaled(synth.WORKLOADS[name], T=T)
+    case = Case(w, device="cuda")
+    s = r3.shape_of(w)
+    c = case.cuda()
+    st = r3.new_status("cuda")
+    ws = r3.workspace(r3.replay_layer_workspace_bytes(s), "cuda")
+    first = r3.replay_layer(s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"], c["w_down"],
+                            c["dy"], ws=ws, dev_status=st)
+    x2 = (c["x"].flip(1) * 0.5).contiguous()
+    dy2 = c["dy"].flip(0).contiguous()
+    wd2 = (c["w_down"] * 1.25).contiguous()
+    for _ in range(2):
+        again = r3.replay_layer_same_record(s, x2, c["w_r"], c["idx"], c["w_gate"], c["w_up"], wd2,
+                                            dy2, ws=ws, dev_status=st)
+        torch.cuda.synchronize()
+        fresh = r3.replay_layer(s, x2, c["w_r"], c["idx"], c["w_gate"], c["w_up"], wd2, dy2,
+                                dev_status=st)
+        torch.cuda.synchronize()
+        for a, b in zip(again, fresh):
+            assert torch.equal(a, b)
+    assert st.item() == 0
+    assert not torch.equal(first[0], again[0])
