@@ -30,7 +30,13 @@ METRIC = "replayed-MoE-layer tokens/s (fwd+router bwd)"
 UNIT = "tokens/s"
 # kernel launches of one r3_replay_layer call: router-weight split 1, logits 1, permute 4
 # (count, scan, rank), GEMM work lists 1, expert GEMMs 2, finish (gate + combine + dgates + dlogits) 1
-LAUNCHES_PER_STEP = 8   # split_router_weight, router_tc, permute_maps_coop, permute_rows, build_work, two GEMMs, finish
+# split_router_weight, router_tc, dispatch maps, permute_rows, build_work, two GEMMs, finish; up
+# to 4096 tokens the one-cluster dispatch builds the work lists itself (no build_work launch)
+LAUNCHES_PER_STEP = 8
+
+
+def launches_per_step(T: int) -> int:
+    return LAUNCHES_PER_STEP - (1 if T <= 4096 else 0)
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
 # from the ncu capture summarised in profiles/grouped_gemm_pair_c2_layer_bf16.md.
 GEMM_UP_DRAM_TRAFFIC_BYTES = 990.4e6   # 942.9 MB read + 47.5 MB written
@@ -407,7 +413,7 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     assert torch.equal(y, y_first), "second pass over the record disagrees with the first"
     same_record = {"ms_per_step": round(ev0.elapsed_time(ev1) / sr_steps, 5), "steps": sr_steps,
-                   "launches_per_step": LAUNCHES_PER_STEP - 2,
+                   "launches_per_step": LAUNCHES_PER_STEP - 2,   # no dispatch maps, no build_work
                    "note": "r3_replay_layer_same_record: dispatch maps and work lists of the "
                            "preceding r3_replay_layer call used again; not the headline step"}
 
@@ -493,7 +499,7 @@ def run_ours(args, w):
                        "l2": "inputs larger than L2: %.2f GB of expert weights stream through "
                              "the 126 MB L2 every step" % (synth.layer_bytes(wk) / 1e9)},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
-            "gpu_launches": LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
+            "gpu_launches": launches_per_step(T) * args.steps, "clocks": clocks,
             "per_step": per_step, "inputs": inputs, "kernels": kernels, "same_record_pass": same_record, "peaks": peaks,
         }
         print(json.dumps(line), flush=True)

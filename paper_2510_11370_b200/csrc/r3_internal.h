@@ -69,6 +69,24 @@ size_t router_tc_workspace_bytes(const r3_shape* shape, int L);
 r3_status launch_router_tc(const r3_shape* shape, int L, const void* x, const void* w_router,
                            void* idx_out, float* logits_out, void* workspace, cudaStream_t stream);
 
+// Where the up phase of the bf16 experts expects its two work lists inside a
+// r3_grouped_swiglu workspace, and their parameters (feature tiles per list, resident clusters).
+// false: this shape does not use such lists (float32), or the device query failed.
+struct WorkListSpec {
+    int32_t* list0;
+    int32_t* list1;
+    int nf0, nf1, pairs;
+};
+bool grouped_swiglu_list_spec(const r3_shape* shape, void* workspace, WorkListSpec* spec);
+bool tc_work_lists(const r3_shape* shape, void* work, WorkListSpec* spec);
+
+// r3_permute; with `lists` the one-cluster form of the dispatch also builds the expert GEMMs'
+// work lists (then *lists_built = true and the experts run with kPhaseKeepLists).
+r3_status permute_impl(const r3_shape* shape, const void* idx, const void* x, int32_t* counts,
+                       int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* xp,
+                       void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream,
+                       const WorkListSpec* lists, bool* lists_built);
+
 // r3_grouped_swiglu (with pre_gate / pre_up: r3_grouped_swiglu_train) on a workspace whose work
 // lists an earlier call built from the same offsets.
 r3_status grouped_swiglu_keep_lists(const r3_shape* shape, const void* xp, const int32_t* offsets,

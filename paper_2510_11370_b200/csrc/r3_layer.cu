@@ -134,14 +134,25 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
         st = grouped_swiglu_keep_lists(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, pre_gate,
                                        pre_up, w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
     } else {
-        if ((st = r3_permute(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row,
-                             w.xp, w.permute_ws, w.permute_bytes, dev_status, stream)) != R3_OK)
+        // a small batch is dispatched by one cluster launch, which then builds the experts' work
+        // lists as well (one launch fewer in front of the GEMMs)
+        WorkListSpec lists;
+        const bool want = grouped_swiglu_list_spec(shape, w.swiglu_ws, &lists);
+        bool built = false;
+        if ((st = permute_impl(shape, idx, x, w.counts, w.offsets, w.row_of_slot, w.slot_of_row,
+                               w.xp, w.permute_ws, w.permute_bytes, dev_status, stream,
+                               want ? &lists : nullptr, &built)) != R3_OK)
             return st;
-        st = pre_gate ? r3_grouped_swiglu_train(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
-                                                pre_gate, pre_up, w.swiglu_ws, w.swiglu_bytes,
-                                                dev_status, stream)
-                      : r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
-                                          w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
+        if (built)
+            st = grouped_swiglu_keep_lists(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
+                                           pre_gate, pre_up, w.swiglu_ws, w.swiglu_bytes,
+                                           dev_status, stream);
+        else
+            st = pre_gate ? r3_grouped_swiglu_train(shape, w.xp, w.offsets, w_gate, w_up, w_down,
+                                                    w.o, pre_gate, pre_up, w.swiglu_ws,
+                                                    w.swiglu_bytes, dev_status, stream)
+                          : r3_grouped_swiglu(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o,
+                                              w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
     }
     if (st != R3_OK) return st;
     if (fused && side && cudaStreamWaitEvent(cs, side->join, 0) != cudaSuccess) return R3_ERR_CUDA;

@@ -13,6 +13,7 @@
 #include "r3_common.cuh"
 #include "r3_internal.h"
 #include "r3_tc.cuh"
+#include "r3_worklist.cuh"
 
 namespace r3 {
 
@@ -296,12 +297,14 @@ __global__ void __launch_bounds__(kChunk)
 permute_maps_cluster_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ counts,
                             int32_t* __restrict__ offsets, int32_t* __restrict__ row_of_slot,
                             int32_t* __restrict__ slot_of_row, int T, int E, int K,
-                            int32_t* dev_status) {
+                            int32_t* dev_status, WorkListSpec lists) {
     extern __shared__ int32_t sm[];
     int32_t* hist = sm;                                       // [E] this chunk's counts
     int32_t* total = sm + E;                                  // [E] all chunks
     int32_t* first = sm + 2 * E;                              // [E] first row of (expert, chunk)
     uint32_t* bits = reinterpret_cast<uint32_t*>(sm + 3 * E); // [E][kWords]
+    int32_t* eoff = sm + (3 + kWords) * E;                    // [E + 1] expert offsets
+    int32_t* s_items = eoff + E + 1;                          // [E + 1] scratch of the list builder
     __shared__ int32_t warp_sum[kChunk / 32];
     const int lt = threadIdx.x, lane = lt & 31, warp = lt >> 5;
     const int nb = gridDim.x, b = blockIdx.x;                 // one cluster: rank = blockIdx.x
@@ -373,6 +376,8 @@ permute_maps_cluster_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ 
         if (e < E) {
             const int32_t cnt = total[e];
             first[e] += run;                               // expert offset + rows of earlier chunks
+            eoff[e] = run;
+            if (e == E - 1) eoff[E] = run + cnt;
             if (b == 0) {
                 offsets[e] = run;
                 counts[e] = cnt;
@@ -406,6 +411,13 @@ permute_maps_cluster_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ 
                 }
             }
         }
+    }
+    // The work lists of the expert GEMMs, when the caller wants them from this launch: the last
+    // CTA builds the up-projection list, the one before it (if there is one) the other.
+    if (lists.list0) {
+        if (b == nb - 1) tc::build_work_list(eoff, E, lists.nf0, lists.list0, lists.pairs, s_items);
+        if (b == (nb >= 2 ? nb - 2 : 0))
+            tc::build_work_list(eoff, E, lists.nf1, lists.list1, lists.pairs, s_items);
     }
 }
 
@@ -530,10 +542,13 @@ extern "C" size_t r3_permute_workspace_bytes(const r3_shape* shape) {
     return r3::round_up((size_t)shape->E * (NB ? NB : 1) * sizeof(int32_t), 256);
 }
 
-extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const void* x,
-                                int32_t* counts, int32_t* offsets, int32_t* row_of_slot,
-                                int32_t* slot_of_row, void* xp, void* workspace, size_t ws_bytes,
-                                int32_t* dev_status, void* stream) {
+// `lists` (may be null): the expert GEMMs' work lists are wanted from the dispatch launch itself;
+// *lists_built tells whether this call could do that (only the one-cluster form does).
+r3_status r3::permute_impl(const r3_shape* shape, const void* idx, const void* x, int32_t* counts,
+                           int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* xp,
+                           void* workspace, size_t ws_bytes, int32_t* dev_status, void* stream,
+                           const WorkListSpec* lists, bool* lists_built) {
+    if (lists_built) *lists_built = false;
     r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
     if (shape->E > r3::kMaxExpertsPermute) return R3_ERR_UNSUPPORTED;
@@ -560,7 +575,7 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
     if (NB <= r3::kClusterMax) {
         int cl = 1;
         while (cl < NB) cl <<= 1;
-        const size_t smem = (size_t)E * (3 + r3::kWords) * sizeof(int32_t);
+        const size_t smem = ((size_t)E * (5 + r3::kWords) + 2) * sizeof(int32_t);
         static int usable[2][r3::kClusterMax + 1] = {};        // per index type and cluster size
         const int ti = shape->idx_type == R3_IDX_U8 ? 0 : 1;   // 0 = untested, 1 = ok, -1 = no
         cudaLaunchConfig_t cfg = {};
@@ -594,12 +609,15 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
             }
         }
         if (usable[ti][cl] == 1) {
+            r3::WorkListSpec wl = {nullptr, nullptr, 0, 0, 0};
+            if (lists && E <= 1024) wl = *lists;
             cudaError_t le = cudaErrorUnknown;
             R3_DISPATCH_IDX(shape, IdxT, le = cudaLaunchKernelEx(
                 &cfg, r3::permute_maps_cluster_kernel<IdxT>, static_cast<const IdxT*>(idx), counts,
-                offsets, row_of_slot, slot_of_row, T, E, K, dev_status));
+                offsets, row_of_slot, slot_of_row, T, E, K, dev_status, wl));
             if (le != cudaSuccess) return R3_ERR_CUDA;
             coop_done = true;
+            if (lists_built && wl.list0) *lists_built = true;
         }
     }
     // one cooperative launch when all the chunk CTAs can be resident together
@@ -636,6 +654,14 @@ extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const vo
     }
     if (x) return r3::launch_permute_rows(shape, x, row_of_slot, xp, cs);
     return r3::launch_status();
+}
+
+extern "C" r3_status r3_permute(const r3_shape* shape, const void* idx, const void* x,
+                                int32_t* counts, int32_t* offsets, int32_t* row_of_slot,
+                                int32_t* slot_of_row, void* xp, void* workspace, size_t ws_bytes,
+                                int32_t* dev_status, void* stream) {
+    return r3::permute_impl(shape, idx, x, counts, offsets, row_of_slot, slot_of_row, xp, workspace,
+                            ws_bytes, dev_status, stream, nullptr, nullptr);
 }
 
 // ---------------------------------------------------------------------------------------------

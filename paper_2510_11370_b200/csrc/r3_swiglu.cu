@@ -214,6 +214,11 @@ static r3_status run_experts(const r3_shape* shape, const void* xp, const void* 
     return launch_grouped_swiglu_f32(shape, xp, tiles, w_gate, w_up, w_down, h, o, phases, cs);
 }
 
+bool grouped_swiglu_list_spec(const r3_shape* shape, void* workspace, WorkListSpec* spec) {
+    if (shape->act_dtype != R3_BF16 || shape->E > 1024 || !workspace) return false;
+    return tc_work_lists(shape, static_cast<char*>(workspace) + h_bytes(shape), spec);
+}
+
 r3_status grouped_swiglu_keep_lists(const r3_shape* shape, const void* xp, const int32_t* offsets,
                                     const void* w_gate, const void* w_up, const void* w_down,
                                     void* o, void* pre_gate, void* pre_up, void* workspace,

@@ -44,12 +44,12 @@
 #include "r3_common.cuh"
 #include "r3_internal.h"
 #include "r3_tc.cuh"
+#include "r3_worklist.cuh"
 
 namespace r3 {
 namespace tc {
 
 constexpr int BMF = 128;           // weight rows (output features) per CTA; UMMA M = 2 * BMF
-constexpr int BNT = 256;           // most token rows per item (UMMA N)
 constexpr int BK = 64;             // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int UK = 16;             // k per tcgen05.mma (bf16)
 constexpr int STAGES = 6;
@@ -64,7 +64,6 @@ constexpr int EPI_BYTES = 28 * 1024;             // transpose / exchange buffers
 constexpr int BAR_BYTES = 256;
 constexpr int RING = 16;                         // item descriptors / claims in flight per CTA
 constexpr int SCHED_BYTES = RING * 32 + RING * 8;
-constexpr int STATIC_ITEMS = 3;                  // items per cluster taken by position
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + SCHED_BYTES + 1024;
 constexpr int FEAT0 = BMF;         // h features per item in MODE 0 (64 per CTA, gate + up rows)
 constexpr int FEAT1 = 2 * BMF;     // o features per item in MODE 1
@@ -76,73 +75,14 @@ struct alignas(64) PairMaps {
     CUtensorMap g;                 // gather form: the un-permuted activations, box 64 x 1
 };
 
-// ---- work list -------------------------------------------------------------------------------
-// Per list: int32 header[kHeaderInts] = {number of items, claim counter, clusters finished, 0},
-// then one int4 per item =
-// {expert | feature tile << 16, first row, N (multiple of 16), valid rows}, ordered
-// (expert, feature tile, token tile).  An expert with cnt rows is cut into nt = ceil(cnt / 256)
-// token tiles of equal size q (rounded up to 16; the last one holds what is left).
-constexpr int kHeaderInts = 4;
-
-__host__ __device__ inline int split_tiles(int cnt) { return (cnt + BNT - 1) / BNT; }
-__host__ __device__ inline int split_rows(int cnt, int nt) {      // rows per tile, multiple of 16
-    return (((cnt + nt - 1) / nt) + 15) & ~15;
-}
-
+// ---- work list (layout and builder: r3_worklist.cuh) ------------------------------------------
 // One CTA per list (blockIdx.x = 0: up projection with nf0 feature tiles, 1: down with nf1).
 __global__ void __launch_bounds__(1024)
 build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
                   int32_t* __restrict__ list0, int32_t* __restrict__ list1, int pairs) {
     __shared__ int32_t s_items[1025];
-    __shared__ int32_t w_items[32];
-    const int nf = blockIdx.x == 0 ? nf0 : nf1;
-    int32_t* list = blockIdx.x == 0 ? list0 : list1;
-    int4* items = reinterpret_cast<int4*>(list + kHeaderInts);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    const int32_t my_items = tid < E ? split_tiles(offsets[tid + 1] - offsets[tid]) * nf : 0;
-    int32_t ii = my_items;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int32_t a = __shfl_up_sync(0xffffffffu, ii, o);
-        if (lane >= o) ii += a;
-    }
-    if (lane == 31) w_items[warp] = ii;
-    __syncthreads();
-    if (warp == 0) {
-        const int32_t a0 = w_items[lane];
-        int32_t a = a0;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int32_t x = __shfl_up_sync(0xffffffffu, a, o);
-            if (lane >= o) a += x;
-        }
-        w_items[lane] = a - a0;
-    }
-    __syncthreads();
-    s_items[tid] = w_items[warp] + ii - my_items;      // exclusive prefix
-    if (tid == 1023) s_items[1024] = w_items[warp] + ii;
-    __syncthreads();
-    const int32_t I = s_items[1024];
-    if (tid == 0) {
-        list[0] = I;
-        list[1] = STATIC_ITEMS * pairs;          // first item handed out by the counter
-        list[2] = 0;
-    }
-    for (int32_t i = tid; i < I; i += 1024) {
-        int lo = 0, hi = E;                      // last e with s_items[e] <= i
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (s_items[mid] <= i) lo = mid; else hi = mid;
-        }
-        const int e = lo;
-        const int row_lo = offsets[e], cnt = offsets[e + 1] - row_lo;
-        const int nt = split_tiles(cnt), q = split_rows(cnt, nt);
-        const int k = i - s_items[e];
-        const int f = k / nt, j = k - f * nt;
-        const int valid = min(q, cnt - j * q);
-        items[i] = make_int4(e | (f << 16), row_lo + j * q, (valid + 15) & ~15, valid);
-    }
+    build_work_list(offsets, E, blockIdx.x == 0 ? nf0 : nf1, blockIdx.x == 0 ? list0 : list1, pairs,
+                    s_items);
 }
 
 // ---- item hand-over inside a CTA pair ---------------------------------------------------------
@@ -713,14 +653,8 @@ size_t tc_work_bytes(const r3_shape* s) {
     return list_bytes(R, s->E, feat_tiles_up(s)) + list_bytes(R, s->E, feat_tiles_down(s));
 }
 
-r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void* x,
-                                   const int32_t* slot_of_row, const int32_t* offsets,
-                                   const void* w_gate, const void* w_up, const void* w_down,
-                                   void* h, void* o, void* work, int32_t* dev_status, int phases,
-                                   cudaStream_t cs, void* pre_gate, void* pre_up) {
+static bool forward_attrs() {
     using namespace tc;
-    const long long R = (long long)s->T * s->K;
-    if (R == 0) return R3_OK;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<0, false>,
@@ -729,9 +663,35 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-            return R3_ERR_CUDA;
+            return false;
         attr_set = true;
     }
+    return true;
+}
+
+bool tc_work_lists(const r3_shape* s, void* work, WorkListSpec* spec) {
+    using namespace tc;
+    if (!forward_attrs()) return false;
+    const int pairs = resident_pairs(grouped_gemm_pair_kernel<0, false>);
+    if (pairs <= 0) return false;
+    const long long R = (long long)s->T * s->K;
+    spec->nf0 = feat_tiles_up(s);
+    spec->nf1 = feat_tiles_down(s);
+    spec->pairs = pairs;
+    spec->list0 = static_cast<int32_t*>(work);
+    spec->list1 = reinterpret_cast<int32_t*>(static_cast<char*>(work) + list_bytes(R, s->E, spec->nf0));
+    return true;
+}
+
+r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void* x,
+                                   const int32_t* slot_of_row, const int32_t* offsets,
+                                   const void* w_gate, const void* w_up, const void* w_down,
+                                   void* h, void* o, void* work, int32_t* dev_status, int phases,
+                                   cudaStream_t cs, void* pre_gate, void* pre_up) {
+    using namespace tc;
+    const long long R = (long long)s->T * s->K;
+    if (R == 0) return R3_OK;
+    if (!forward_attrs()) return R3_ERR_CUDA;
     const int pairs = resident_pairs(grouped_gemm_pair_kernel<0, false>);
     if (pairs <= 0) return R3_ERR_CUDA;
     const int nf0 = feat_tiles_up(s), nf1 = feat_tiles_down(s);
