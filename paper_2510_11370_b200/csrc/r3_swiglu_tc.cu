@@ -11,9 +11,11 @@
 //
 // Orientation.  The WEIGHT rows are the M side of the MMA and the TOKEN rows are the N side, so
 // the accumulator holds out^T: tensor-memory lane = output feature, column = token.  M is fixed
-// by the hardware (256 per CTA pair) while N may be any multiple of 16 up to 256, so an expert
-// with an awkward number of rows costs MMA time in proportion to its rows (padding to 16), not
-// to the next multiple of a fixed row tile.
+// by the hardware (256 per CTA pair) while N may be any multiple of 16 up to 256, so the token
+// rows of a tile are padded to 16, not to a fixed row tile: a short tile copies and stores fewer
+// rows.  (Its MMAs do not get shorter: one 256 x N x 16 MMA was measured to occupy the tensor pipe
+// for about the same time whatever its N, so a launch costs its NUMBER of MMAs, ceil(rows / 256)
+// token tiles per expert.)
 //
 // A work item is (expert, token tile of N <= 256 rows, feature tile).  The two CTAs of a cluster
 // share it (tcgen05 cta_group::2, UMMA 256 x N x 16): each CTA loads 128 weight rows and N/2
@@ -34,9 +36,10 @@
 // memory, so nobody waits on a claim.  The last cluster to finish re-arms the counter.
 //
 // Roles (192 threads per CTA): warp 0 lane 0 = TMA producer (both CTAs, into a 6-stage ring of
-// 128B-swizzled tiles), warp 1 of the leader CTA = MMA issuer (one elected lane) (two accumulator stages of
-// 256 columns, so the epilogue of an item overlaps the main loop of the next), warps 2..5 =
-// epilogue (tcgen05.ld -> transpose through shared memory -> 16-byte global stores).
+// 128B-swizzled tiles), warp 1 of the leader CTA = MMA issuer (the warp walks the barriers, one
+// elected lane issues; two accumulator stages of 256 columns, so the epilogue of an item overlaps
+// the main loop of the next), warps 2..5 = epilogue (tcgen05.ld -> transpose through shared
+// memory -> 16-byte global stores).
 //
 // Every mbarrier wait is bounded by a clock limit; when a wait runs out the CTA raises a shared
 // abort flag, reports R3_DEV_TIMEOUT, lets the other roles drain (they keep their barrier
