@@ -13,9 +13,8 @@
 // the accumulator holds out^T: tensor-memory lane = output feature, column = token.  M is fixed
 // by the hardware (256 per CTA pair) while N may be any multiple of 16 up to 256, so the token
 // rows of a tile are padded to 16, not to a fixed row tile: a short tile copies and stores fewer
-// rows.  (Its MMAs do not get shorter: one 256 x N x 16 MMA was measured to occupy the tensor pipe
-// for about the same time whatever its N, so a launch costs its NUMBER of MMAs, ceil(rows / 256)
-// token tiles per expert.)
+// rows and its MMAs are shorter (a 256 x N x 16 MMA measures max(58, N/2) clocks).  The weight
+// tile is copied once per token tile whatever its N.
 //
 // A work item is (expert, token tile of N <= 256 rows, feature tile).  The two CTAs of a cluster
 // share it (tcgen05 cta_group::2, UMMA 256 x N x 16): each CTA loads 128 weight rows and N/2
