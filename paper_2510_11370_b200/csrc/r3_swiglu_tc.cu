@@ -457,15 +457,27 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
 #pragma unroll
                     for (int i = 0; i < 16; ++i) send[i * 32 + lane] = gate ? v[16 + i] : v[i];
                     named_bar_sync(1 + p, 64);
+                    // all loads first, then the arithmetic, then the stores: written as one loop
+                    // the stores to hb may alias the loads from recv as far as the compiler knows,
+                    // and the 16 load - exp - divide - store chains run one after the other
+                    // (measured: 2000 of the 2700 clocks of a chunk)
+                    float other[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) other[i] = recv[i * 32 + lane];
+                    float hv[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const float other = recv[i * 32 + lane];
-                        const float g = gate ? v[i] : other;
-                        const float u = gate ? other : v[16 + i];
-                        hb[i * 32 + lane] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
-                        if (keep) {
-                            gb[i * 32 + lane] = __float2bfloat16_rn(g);
-                            ub[i * 32 + lane] = __float2bfloat16_rn(u);
+                        const float g = gate ? v[i] : other[i];
+                        const float u = gate ? other[i] : v[16 + i];
+                        hv[i] = __fdividef(g, 1.f + __expf(-g)) * u;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) hb[i * 32 + lane] = __float2bfloat16_rn(hv[i]);
+                    if (keep) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            gb[i * 32 + lane] = __float2bfloat16_rn(gate ? v[i] : other[i]);
+                            ub[i * 32 + lane] = __float2bfloat16_rn(gate ? other[i] : v[16 + i]);
                         }
                     }
                     __syncwarp();
