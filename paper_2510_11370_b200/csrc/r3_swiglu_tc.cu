@@ -481,20 +481,26 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
                         }
                     }
                     __syncwarp();
+                    uint4 hq[2], gq[2], uq[2];         // all reads before the first store
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const int in_tile = ((lane >> 2) + 8 * rr) * 32 + (lane & 3) * 8;
+                        hq[rr] = *reinterpret_cast<const uint4*>(hb + in_tile);
+                        if (keep) {
+                            gq[rr] = *reinterpret_cast<const uint4*>(gb + in_tile);
+                            uq[rr] = *reinterpret_cast<const uint4*>(ub + in_tile);
+                        }
+                    }
 #pragma unroll
                     for (int rr = 0; rr < 2; ++rr) {
                         const int tl = (lane >> 2) + 8 * rr;
                         const int tok = c + own + tl;
                         if (alive && tok < valid && feat + 8 <= Nout) {
                             const size_t at = (size_t)(row0 + tok) * Nout + feat;
-                            const int in_tile = tl * 32 + (lane & 3) * 8;
-                            *reinterpret_cast<uint4*>(out + at) =
-                                *reinterpret_cast<const uint4*>(hb + in_tile);
+                            *reinterpret_cast<uint4*>(out + at) = hq[rr];
                             if (keep) {
-                                *reinterpret_cast<uint4*>(pre_gate + at) =
-                                    *reinterpret_cast<const uint4*>(gb + in_tile);
-                                *reinterpret_cast<uint4*>(pre_up + at) =
-                                    *reinterpret_cast<const uint4*>(ub + in_tile);
+                                *reinterpret_cast<uint4*>(pre_gate + at) = gq[rr];
+                                *reinterpret_cast<uint4*>(pre_up + at) = uq[rr];
                             }
                         }
                     }
@@ -512,15 +518,18 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
 #pragma unroll
                         for (int i = 0; i < 32; ++i) tbuf[i * 32 + lane] = __float2bfloat16_rn(v[i]);
                         __syncwarp();
+                        uint4 val[4];                  // all reads before the first store
+#pragma unroll
+                        for (int rr = 0; rr < 4; ++rr)
+                            val[rr] = *reinterpret_cast<const uint4*>(
+                                tbuf + ((lane >> 2) + 8 * rr) * 32 + (lane & 3) * 8);
 #pragma unroll
                         for (int rr = 0; rr < 4; ++rr) {
                             const int tok = (lane >> 2) + 8 * rr;
-                            const uint4 val = *reinterpret_cast<const uint4*>(
-                                tbuf + tok * 32 + (lane & 3) * 8);
                             const int feat = feat0 + (lane & 3) * 8;
                             if (c + tok < valid && feat + 8 <= Nout)
                                 *reinterpret_cast<uint4*>(out + (size_t)(row0 + c + tok) * Nout +
-                                                          feat) = val;
+                                                          feat) = val[rr];
                         }
                         __syncwarp();
                     }

@@ -231,13 +231,18 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
                     tbuf[lane * 8 + (j ^ (lane & 7))] =
                         make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                 __syncwarp();
+                float4 val[8];                     // all reads before the first store (the
+#pragma unroll                                     // stores might alias them for the compiler)
+                for (int rr = 0; rr < 8; ++rr) {
+                    const int r = rr * 4 + (lane >> 3), j = lane & 7;
+                    val[rr] = tbuf[r * 8 + (j ^ (r & 7))];
+                }
 #pragma unroll
                 for (int rr = 0; rr < 8; ++rr) {
                     const int r = rr * 4 + (lane >> 3), j = lane & 7;
-                    const float4 val = tbuf[r * 8 + (j ^ (r & 7))];
                     const int m = it.m0 + q * 32 + r, n = it.n0 + c + 4 * j;
                     if (m < M && n + 4 <= N)
-                        *reinterpret_cast<float4*>(out + (size_t)m * N + n) = val;
+                        *reinterpret_cast<float4*>(out + (size_t)m * N + n) = val[rr];
                 }
                 __syncwarp();
             }
