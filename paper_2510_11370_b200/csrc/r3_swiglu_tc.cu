@@ -34,8 +34,9 @@
 // publish each item's descriptor to the other warps of their CTA through a tagged ring in shared
 // memory, so nobody waits on a claim.  The last cluster to finish re-arms the counter.
 //
-// Roles (192 threads per CTA): warp 0 lane 0 = TMA producer (both CTAs, into a 6-stage ring of
-// 128B-swizzled tiles), warp 1 of the leader CTA = MMA issuer (the warp walks the barriers, one
+// Roles (224 threads per CTA): warp 0 lane 0 = TMA producer of the weight boxes and warp 6 lane 0
+// = TMA producer of the token box (both CTAs, into a 6-stage ring of 128B-swizzled tiles; two
+// issuing threads per stage), warp 1 of the leader CTA = MMA issuer (the warp walks the barriers, one
 // elected lane issues; two accumulator stages of 256 columns, so the epilogue of an item overlaps
 // the main loop of the next), warps 2..5 = epilogue (tcgen05.ld -> transpose through shared
 // memory -> 16-byte global stores).
@@ -61,7 +62,7 @@ constexpr int A_BYTES = BMF * BK * 2;            // 16 KB of weights per CTA and
 constexpr int B_BYTES = (BNT / 2) * BK * 2;      // up to 16 KB of tokens per CTA and stage
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int EPI_WARPS = 4;
-constexpr int THREADS = (2 + EPI_WARPS) * 32;
+constexpr int THREADS = (3 + EPI_WARPS) * 32;    // + warp 6: token-tile copies
 constexpr int EPI_BYTES = 28 * 1024;             // transpose / exchange buffers of the epilogue
 constexpr int BAR_BYTES = 256;
 constexpr int RING = 16;                         // item descriptors / claims in flight per CTA
@@ -306,14 +307,13 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
                 }
                 idx_cur = idx_next;
                 ++seq;
-                const int e = it.x & 0xffff, f = it.x >> 16, n = it.z, half = n >> 1;
-                const CUtensorMap* bmap = &maps.b[(half >> 3) - 1];
+                const int e = it.x & 0xffff, f = it.x >> 16, n = it.z;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) {
                         ok = false;
                         break;
                     }
-                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint32_t sa = base + stage * STAGE_BYTES;
                     const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
                     if (rank == 0)                      // bytes of both CTAs: 2 x (A + n/2 rows)
                         mbar_expect_tx(full_bar(stage), (uint32_t)(2 * A_BYTES + n * BK * 2));
@@ -333,11 +333,6 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
                         tma_load_3d_pair(sa, amap, m0, kk * BK, e, lead_full);
                         tma_load_3d_pair(sa + A_BYTES / 2, amap, m0 + 64, kk * BK, e, lead_full);
                     }
-                    if (MODE == 3)
-                        tma_load_3d_pair(sb, bmap, (kb >> 1) * BK, it.y + (int)rank * half, kb & 1,
-                                         lead_full);
-                    else
-                        tma_load_2d_pair(sb, bmap, kb * BK, it.y + (int)rank * half, lead_full);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -405,6 +400,39 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
                 if (elect_one()) tc_commit_pair(tfull_bar(acc), 3);   // accumulator complete, both CTAs
                 __syncwarp();
                 if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else if (warp == 6) {
+        // ------------------------------ token-tile copies (each CTA its own half) --------------
+        // A second issuing thread: the weight boxes and the token box of a stage are asked for
+        // by two threads at once.  It follows the items through the descriptor ring and walks
+        // the same stages as warp 0; its bytes may land before warp 0 has told the barrier how
+        // many to expect (the pending arrival keeps the phase open).  The gather form copies the
+        // token rows in warp 0.
+        if (lane == 0 && !GATHER) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int seq = 0; ok; ++seq) {
+                int4 it;
+                if (!desc_get(desc_ring, seq, &it, abort_flag, dev_status)) break;
+                const int n = it.z, half = n >> 1;
+                if (n == 0) break;
+                const CUtensorMap* bmap = &maps.b[(half >> 3) - 1];
+                const int brow = it.y + (int)rank * half;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, dev_status)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sb = base + stage * STAGE_BYTES + A_BYTES;
+                    const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
+                    if (MODE == 3)
+                        tma_load_3d_pair(sb, bmap, (kb >> 1) * BK, brow, kb & 1, lead_full);
+                    else
+                        tma_load_2d_pair(sb, bmap, kb * BK, brow, lead_full);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
             }
         }
     } else {
