@@ -68,12 +68,14 @@ __device__ __forceinline__ void finish_tokens(const float* tile, int LD, const i
                                               IdxT* idx_out, float* logits_out,
                                               uint32_t peer_tile) {
     uint32_t key[NT][SLOTS];
+    float val[NT][SLOTS];
+    // all reads of the tile(s) first: the global stores below might alias them for the compiler
 #pragma unroll
     for (int a = 0; a < NT; ++a) {
 #pragma unroll
         for (int sl = 0; sl < SLOTS; ++sl) {
             const int e = lane + 32 * sl;
-            key[a][sl] = 0u;                             // 0 = no candidate (below every real key)
+            val[a][sl] = 0.f;
             if (a < n_rows && e < E) {
                 float v = tile[(size_t)rows[a] * LD + e];
                 if (peer_tile) {                         // the other half of the contraction
@@ -82,6 +84,18 @@ __device__ __forceinline__ void finish_tokens(const float* tile, int LD, const i
                                  : "=f"(w) : "r"(peer_tile + 4u * (uint32_t)(rows[a] * LD + e)));
                     v += w;
                 }
+                val[a][sl] = v;
+            }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < NT; ++a) {
+#pragma unroll
+        for (int sl = 0; sl < SLOTS; ++sl) {
+            const int e = lane + 32 * sl;
+            key[a][sl] = 0u;                             // 0 = no candidate (below every real key)
+            if (a < n_rows && e < E) {
+                const float v = val[a][sl];
                 if (logits_out) logits_out[(out_row0 + rows[a]) * E + e] = v;
                 const uint32_t u = __float_as_uint(v);
                 const uint32_t k2 = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
