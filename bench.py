@@ -39,7 +39,7 @@ def launches_per_step(T: int) -> int:
     return LAUNCHES_PER_STEP - (1 if T <= 4096 else 0)
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel on the bench workload,
 # from the ncu capture summarised in profiles/grouped_gemm_pair_c2_layer_bf16.md.
-GEMM_UP_DRAM_TRAFFIC_BYTES = 988.8e6   # 940.5 MB read + 48.3 MB written
+GEMM_UP_DRAM_TRAFFIC_BYTES = 988.8e6   # 940.8 MB read + 48.0 MB written
 
 
 def load_peaks():
