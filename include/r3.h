@@ -121,7 +121,8 @@ r3_status r3_replay_gate_fwd(const r3_shape* shape, const float* logits, const v
 
 /* Gradient through Eq. (replay_gate) with the mask held constant:
  *   c = sum_j g[t,j] dg[t,j];  dlogits[t,e_j] = g[t,j] (dg[t,j] - c);  dlogits[t,i] = 0 elsewhere.
- * gates, dgates [T,K] f32; idx [T,K]; dlogits [T,E] f32, every element written. */
+ * gates, dgates [T,K] f32; idx [T,K]; dlogits [T,E] f32, every element written; a dlogits that is
+ * not 16-byte aligned returns R3_ERR_INVALID_ARG. */
 r3_status r3_replay_gate_bwd(const r3_shape* shape, const float* gates, const float* dgates,
                              const void* idx, float* dlogits, void* stream);
 
@@ -448,11 +449,15 @@ r3_status r3_ep_move_rows(const void* src, void* dst, const int32_t* perm, int32
  * rank's own experts).  n_ranks <= 64.
  * r3_ep_dispatch_rows: copies x[t] to its K places; idx, row_of_slot and my_offsets (= offsets) are
  * those of this rank's r3_permute (called without x); peer_buffers_host [n_ranks] is a HOST array
- * of device addresses, entry q = base of rank q's receive buffer [rows_q, d].  The owners must
- * not read the buffers before every rank's call has completed (a barrier of the job's own).
+ * of device addresses, entry q = base of rank q's receive buffer [capacity_rows, d] (the same
+ * capacity on every rank).  A row whose place lies at or beyond capacity_rows is NOT stored and
+ * dev_status (optional) receives R3_DEV_BAD_INDEX: a peer's memory is never written out of
+ * bounds.  The owners must not read the buffers before every rank's call has completed (a barrier
+ * of the job's own).
  * r3_ep_slot_rows: row_ptr [T, K] (device, 64-bit addresses) = where the expert-output row of each
- * (token, slot) pair will stand in the owners' OUTPUT buffers (peer_buffers_host: their bases);
- * 0 for a pair that r3_permute dropped.
+ * (token, slot) pair will stand in the owners' OUTPUT buffers (peer_buffers_host: their bases,
+ * capacity_rows as above); 0 for a pair that r3_permute dropped or whose place is beyond the
+ * capacity (then dev_status receives R3_DEV_BAD_INDEX).
  * r3_replay_finish_rows: r3_replay_finish with the rows given by address (row_ptr) instead of
  * (o, row_of_slot).  K <= 8 and the rows of one token must fit in shared memory
  * ((K + 2) d elements, else R3_ERR_UNSUPPORTED). */
@@ -461,11 +466,13 @@ r3_status r3_ep_dest_table(const int32_t* counts_all, int32_t n_ranks, int32_t E
 r3_status r3_ep_dispatch_rows(const r3_shape* shape, int32_t n_ranks, const void* x,
                               const void* idx, const int32_t* row_of_slot,
                               const int32_t* my_offsets, const int32_t* dst_base,
-                              const unsigned long long* peer_buffers_host, void* stream);
+                              const unsigned long long* peer_buffers_host, int64_t capacity_rows,
+                              int32_t* dev_status, void* stream);
 r3_status r3_ep_slot_rows(const r3_shape* shape, int32_t n_ranks, const void* idx,
                           const int32_t* row_of_slot, const int32_t* my_offsets,
                           const int32_t* dst_base, const unsigned long long* peer_buffers_host,
-                          unsigned long long* row_ptr, void* stream);
+                          int64_t capacity_rows, unsigned long long* row_ptr, int32_t* dev_status,
+                          void* stream);
 r3_status r3_replay_finish_rows(const r3_shape* shape, const float* logits, const void* idx,
                                 const unsigned long long* row_ptr, const void* dy,
                                 const void* residual, void* y, float* gates_out, float* dlogits,
@@ -551,6 +558,22 @@ r3_status r3_pagepool_alloc(r3_pagepool* pool, int32_t n, int32_t* pages_out);
 r3_status r3_pagepool_publish(r3_pagepool* pool, const int32_t* token_ids, int32_t n_tokens,
                               const int32_t* table, int32_t n_table);
 r3_status r3_pagepool_release(r3_pagepool* pool, const int32_t* table, int32_t n);
+
+/* ---- self-test of the error path (the paper has no counterpart) ---------------------------------
+ *
+ * The tensor-core kernels wait on shared-memory barriers for their copies and MMAs; every such
+ * wait is bounded, and a wait that runs out raises an abort flag in its CTA, writes
+ * R3_DEV_TIMEOUT to dev_status and lets the kernel drain and return (see "General rules").  In a
+ * healthy run that path never executes.  r3_selftest_bounded_wait runs it on purpose in a
+ * harmless form: one 32-thread CTA waits, with the library's own wait routine and a limit of
+ * `limit_clocks` SM clocks (1 .. 2e9, else R3_ERR_INVALID_ARG), on a barrier of its own that nothing
+ * signals - no copy is in flight and no tensor memory is held.  Afterwards dev_status (optional)
+ * holds R3_DEV_TIMEOUT and out [4] int32 (device) = {the wait's return value (0 = gave up), the
+ * abort flag (1), clocks spent waiting (saturated), the return value of a second wait entered
+ * while the CTA was already aborting (0)}.  The context stays usable: the next call is an
+ * ordinary one. */
+r3_status r3_selftest_bounded_wait(int64_t limit_clocks, int32_t* dev_status, int32_t* out,
+                                   void* stream);
 
 #ifdef __cplusplus
 }

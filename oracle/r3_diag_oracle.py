@@ -41,14 +41,18 @@ def kl_k3(p_train, p_infer) -> float:
     return float(np.sum(r - 1.0 - np.log(r)) / pt.size)
 
 
+def extreme_ratio(p_train, p_infer) -> np.ndarray:
+    """max(r_t, 1 / r_t) per token, r_t = p_train[t] / p_infer[t], in float64 (Eq. (etdf) is
+    stated on real ratios; the stored probabilities are widened exactly)."""
+    pt = np.asarray(p_train, dtype=F64).reshape(-1)
+    pi = np.asarray(p_infer, dtype=F64).reshape(-1)
+    return np.maximum(pt / pi, pi / pt)
+
+
 def extreme_counts(p_train, p_infer, taus) -> np.ndarray:
-    """Number of tokens with max(r, 1/r) > tau, one count per tau (Eq. (etdf) times |T|).
-    The ratio is formed in float32, the precision of the stored probabilities, because the
-    count is an integer decision; both sides of a comparison take it in that precision."""
-    pt = np.asarray(p_train, dtype=np.float32).reshape(-1)
-    pi = np.asarray(p_infer, dtype=np.float32).reshape(-1)
-    big = np.maximum(pt / pi, pi / pt)
-    return np.array([int(np.count_nonzero(big > np.float32(t))) for t in taus], dtype=np.int64)
+    """Number of tokens with max(r, 1/r) > tau, one count per tau (Eq. (etdf) times |T|)."""
+    big = extreme_ratio(p_train, p_infer)
+    return np.array([int(np.count_nonzero(big > F64(t))) for t in taus], dtype=np.int64)
 
 
 def extreme_fraction(p_train, p_infer, taus) -> np.ndarray:

@@ -111,7 +111,8 @@ ep_dispatch_rows_kernel(const uint4* __restrict__ x, const IdxT* __restrict__ id
                         const int32_t* __restrict__ row_of_slot,
                         const int32_t* __restrict__ my_offsets,
                         const int32_t* __restrict__ dst_base, const __grid_constant__ EpPeers peers,
-                        int T, int E, int K, int el, int row_vecs) {
+                        int T, int E, int K, int el, int row_vecs, long long capacity_rows,
+                        int32_t* dev_status) {
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (t >= T) return;
@@ -121,6 +122,10 @@ ep_dispatch_rows_kernel(const uint4* __restrict__ x, const IdxT* __restrict__ id
         if (r < 0) continue;
         const int e = idx_to_int(idx[(size_t)t * K + j]);
         const size_t row = (size_t)dst_base[e] + (size_t)(r - my_offsets[e]);
+        if ((long long)row >= capacity_rows) {        // beyond the owner's buffer: never stored
+            if (lane == 0) report(dev_status, R3_DEV_BAD_INDEX);
+            continue;
+        }
         uint4* dst = reinterpret_cast<uint4*>(peers.base[e / el]) + row * row_vecs;
         for (int c = lane; c < row_vecs; c += 32) dst[c] = src[c];
     }
@@ -132,14 +137,19 @@ __global__ void __launch_bounds__(256)
 ep_slot_rows_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ row_of_slot,
                     const int32_t* __restrict__ my_offsets, const int32_t* __restrict__ dst_base,
                     const __grid_constant__ EpPeers peers, unsigned long long* __restrict__ row_ptr,
-                    long long pairs, int el, unsigned long long row_bytes) {
+                    long long pairs, int el, unsigned long long row_bytes, long long capacity_rows,
+                    int32_t* dev_status) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= pairs) return;
     const int32_t r = row_of_slot[i];
     unsigned long long p = 0;
     if (r >= 0) {
         const int e = idx_to_int(idx[i]);
-        p = peers.base[e / el] + ((unsigned long long)dst_base[e] + (r - my_offsets[e])) * row_bytes;
+        const unsigned long long row = (unsigned long long)dst_base[e] + (r - my_offsets[e]);
+        if ((long long)row < capacity_rows)
+            p = peers.base[e / el] + row * row_bytes;
+        else
+            report(dev_status, R3_DEV_BAD_INDEX);     // beyond the owner's buffer: no address
     }
     row_ptr[i] = p;
 }
@@ -161,10 +171,12 @@ extern "C" r3_status r3_ep_dispatch_rows(const r3_shape* shape, int32_t n_ranks,
                                          const void* idx, const int32_t* row_of_slot,
                                          const int32_t* my_offsets, const int32_t* dst_base,
                                          const unsigned long long* peer_buffers_host,
+                                         int64_t capacity_rows, int32_t* dev_status,
                                          void* stream) {
     r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
-    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || shape->E % n_ranks) return R3_ERR_INVALID_ARG;
+    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || shape->E % n_ranks || capacity_rows < 0)
+        return R3_ERR_INVALID_ARG;
     if (shape->T == 0) return R3_OK;
     if (!x || !idx || !row_of_slot || !my_offsets || !dst_base || !peer_buffers_host ||
         !r3::aligned(x, 16))
@@ -180,7 +192,8 @@ extern "C" r3_status r3_ep_dispatch_rows(const r3_shape* shape, int32_t n_ranks,
     R3_DISPATCH_IDX(shape, IdxT,
         r3::ep_dispatch_rows_kernel<IdxT><<<(shape->T + wpb - 1) / wpb, wpb * 32, 0, cs>>>(
             static_cast<const uint4*>(x), static_cast<const IdxT*>(idx), row_of_slot, my_offsets,
-            dst_base, peers, shape->T, shape->E, shape->K, shape->E / n_ranks, row_vecs));
+            dst_base, peers, shape->T, shape->E, shape->K, shape->E / n_ranks, row_vecs,
+            (long long)capacity_rows, dev_status));
     return r3::launch_status();
 }
 
@@ -188,10 +201,12 @@ extern "C" r3_status r3_ep_slot_rows(const r3_shape* shape, int32_t n_ranks, con
                                      const int32_t* row_of_slot, const int32_t* my_offsets,
                                      const int32_t* dst_base,
                                      const unsigned long long* peer_buffers_host,
-                                     unsigned long long* row_ptr, void* stream) {
+                                     int64_t capacity_rows, unsigned long long* row_ptr,
+                                     int32_t* dev_status, void* stream) {
     r3_status st = r3::check_shape(shape);
     if (st != R3_OK) return st;
-    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || shape->E % n_ranks) return R3_ERR_INVALID_ARG;
+    if (n_ranks <= 0 || n_ranks > r3::kEpMaxRanks || shape->E % n_ranks || capacity_rows < 0)
+        return R3_ERR_INVALID_ARG;
     if (shape->T == 0) return R3_OK;
     if (!idx || !row_of_slot || !my_offsets || !dst_base || !peer_buffers_host || !row_ptr)
         return R3_ERR_INVALID_ARG;
@@ -205,7 +220,8 @@ extern "C" r3_status r3_ep_slot_rows(const r3_shape* shape, int32_t n_ranks, con
     R3_DISPATCH_IDX(shape, IdxT,
         r3::ep_slot_rows_kernel<IdxT><<<(unsigned)((pairs + 255) / 256), 256, 0, cs>>>(
             static_cast<const IdxT*>(idx), row_of_slot, my_offsets, dst_base, peers, row_ptr, pairs,
-            shape->E / n_ranks, (unsigned long long)shape->d * r3::act_bytes(shape)));
+            shape->E / n_ranks, (unsigned long long)shape->d * r3::act_bytes(shape),
+            (long long)capacity_rows, dev_status));
     return r3::launch_status();
 }
 

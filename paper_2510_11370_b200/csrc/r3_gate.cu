@@ -259,14 +259,15 @@ extern "C" r3_status r3_replay_gate_bwd(const r3_shape* shape, const float* gate
     if (st != R3_OK) return st;
     if (shape->T == 0) return R3_OK;
     if (!gates || !dgates || !idx || !dlogits) return R3_ERR_INVALID_ARG;
+    // rows are written in 16-byte pieces whenever E is a multiple of 4
+    if (!r3::aligned(dlogits, 16)) return R3_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int wpb = 8;
     const int tpb = wpb * r3::kGateBwdTokens;               // tokens per block
     const unsigned grid = (unsigned)((shape->T + tpb - 1) / tpb);
     // rows staged in shared memory when they are 16-byte pieces and a block's rows fit 32 KB
     const size_t stage_bytes = (size_t)tpb * shape->E * sizeof(float);
-    const bool staged = shape->K <= 32 && (shape->E & 3) == 0 && stage_bytes <= 32 * 1024 &&
-                        (reinterpret_cast<uintptr_t>(dlogits) & 15) == 0;
+    const bool staged = shape->K <= 32 && (shape->E & 3) == 0 && stage_bytes <= 32 * 1024;
     R3_DISPATCH_IDX(shape, IdxT,
         r3::replay_gate_bwd_kernel<IdxT><<<grid, wpb * 32, staged ? stage_bytes : 0, cs>>>(
             gates, dgates, static_cast<const IdxT*>(idx), dlogits, shape->T, shape->E, shape->K,

@@ -97,7 +97,9 @@ __device__ __forceinline__ void finish_tokens(const float* tile, int LD, const i
             if (a < n_rows && e < E) {
                 const float v = val[a][sl];
                 if (logits_out) logits_out[(out_row0 + rows[a]) * E + e] = v;
-                const uint32_t u = __float_as_uint(v);
+                // order-preserving key; -0.0 and +0.0 are one value (a tie: lower expert wins)
+                uint32_t u = __float_as_uint(v);
+                if (u == 0x80000000u) u = 0u;
                 const uint32_t k2 = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
                 key[a][sl] = k2 ? k2 : 1u;
             }

@@ -36,9 +36,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out after
+// `limit` clocks; then the abort flag is raised and R3_DEV_TIMEOUT reported).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* dev_status) {
+                                          int32_t* dev_status, long long limit = WAIT_CLOCKS) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -46,7 +47,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_CLOCKS) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             report(dev_status, R3_DEV_TIMEOUT);
             return false;

@@ -8,6 +8,9 @@ collective; torch.distributed is used only for the start barrier and to reduce t
 from __future__ import annotations
 
 import os
+import socket
+import subprocess
+import sys
 
 import torch
 import torch.distributed as dist
@@ -53,3 +56,34 @@ def sum_over_ranks(value: float, device="cpu") -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return float(t.item())
+
+
+def free_port() -> int:
+    """A TCP port of the loopback interface that is free right now."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_command(n_ranks: int, script: str, argv, port: int) -> list:
+    """Command line that runs `script argv...` as n_ranks processes of one node under
+    torch.distributed.run, rendezvous on the loopback interface (one process per GPU: every rank
+    reads RANK / LOCAL_RANK / WORLD_SIZE from its environment)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+            f"--nproc-per-node={n_ranks}", "--master-addr", "127.0.0.1", "--master-port",
+            str(port), script, *argv]
+
+
+def run_ranks(n_ranks: int, script: str, argv, env=None) -> int:
+    """Starts the n_ranks processes of a job whose caller gave only a rank count (no launcher
+    environment), waits for them and returns the launcher's exit code.  The ranks inherit the
+    caller's standard output, so rank 0's one line is the job's line."""
+    full_env = dict(os.environ)
+    # NCCL's communicator log (rings, NVLS, transports) of every rank, kept out of the job's
+    # standard output
+    full_env.setdefault("NCCL_DEBUG", "INFO")
+    full_env.setdefault("NCCL_DEBUG_FILE", os.path.join(
+        os.environ.get("TMPDIR", "/tmp"), "r3_nccl_%h_%p.log"))
+    if env:
+        full_env.update(env)
+    return subprocess.call(launch_command(n_ranks, script, list(argv), free_port()), env=full_env)

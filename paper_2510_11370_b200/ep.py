@@ -30,6 +30,26 @@ def split_sizes(send_counts, recv_counts):
     return [int(v) for v in both[0]], [int(v) for v in both[1]]
 
 
+def owner_totals(counts_all, world: int):
+    """Rows every rank will RECEIVE in the direct-write form, from the all-gathered [N, E] count
+    table (the same table on every rank, so every rank computes the same list): entry q is the
+    number of rows routed to the experts of rank q by all ranks together.  One device-to-host copy
+    when the table lives on a GPU."""
+    n, e_total = counts_all.shape
+    el = e_total // world
+    totals = counts_all.reshape(n, world, el).sum(dim=(0, 2)).cpu()
+    return [int(v) for v in totals]
+
+
+def check_capacity(totals, capacity_rows: int):
+    """Raises on EVERY rank (the totals are identical everywhere) when some owner's buffer cannot
+    take the rows routed to it - before any rank has stored a row into a peer's memory."""
+    worst = max(totals)
+    if worst > capacity_rows:
+        raise ValueError(f"receive buffers of {capacity_rows} rows are too small: rank "
+                         f"{totals.index(worst)} is sent {worst} rows")
+
+
 def exchange_counts(send_counts, group=None):
     """All-to-all of the [N, E/N] count table: row q goes to rank q; row s of the result is what
     rank s sends here."""
@@ -129,17 +149,18 @@ class EpDirectRank:
         return self.counts
 
     def plan(self, counts_all):
-        """counts_all [N, E] (all-gathered).  Returns the rows this rank will receive."""
+        """counts_all [N, E] (all-gathered).  Returns the rows this rank will receive; the rows
+        every rank will receive are kept in `owner_rows` (identical on all ranks)."""
         self.dst_base, self.offsets_local = r3.ep_dest_table(counts_all.contiguous(), self.rank)
-        el = self.e_local
-        mine = counts_all[:, self.rank * el:(self.rank + 1) * el]
-        self.recv_rows = int(mine.sum().item())
+        self.owner_rows = owner_totals(counts_all, self.world)
+        self.recv_rows = self.owner_rows[self.rank]
         return self.recv_rows
 
-    def send(self, receive_buffers):
-        """receive_buffers: base addresses of every rank's [rows, d] receive buffer."""
+    def send(self, receive_buffers, capacity_rows: int):
+        """receive_buffers: base addresses of every rank's [capacity_rows, d] receive buffer."""
         r3.ep_dispatch_rows(self.shape, self.world, self.x, self.idx, self.row_of_slot,
-                            self.offsets, self.dst_base, receive_buffers)
+                            self.offsets, self.dst_base, receive_buffers, capacity_rows,
+                            dev_status=self.status)
 
     def experts(self, received, w_gate, w_up, w_down, out):
         """This rank's experts on its receive buffer (already in expert-major order)."""
@@ -149,10 +170,11 @@ class EpDirectRank:
                               dev_status=self.status)
         return out
 
-    def finish(self, output_buffers, dy):
-        """output_buffers: base addresses of every rank's expert-output buffer."""
+    def finish(self, output_buffers, dy, capacity_rows: int):
+        """output_buffers: base addresses of every rank's [capacity_rows, d] output buffer."""
         row_ptr = r3.ep_slot_rows(self.shape, self.world, self.idx, self.row_of_slot, self.offsets,
-                                  self.dst_base, output_buffers)
+                                  self.dst_base, output_buffers, capacity_rows,
+                                  dev_status=self.status)
         y, gates, dlogits = r3.replay_finish_rows(self.shape, self.logits, self.idx, row_ptr, dy,
                                                   dev_status=self.status)
         return y, dlogits, gates
@@ -164,6 +186,7 @@ class PeerBuffers:
 
     def __init__(self, received, outputs, receive_addresses, output_addresses, barrier):
         self.received, self.outputs = received, outputs
+        self.capacity_rows = int(received.shape[0])      # the same on every rank
         self.receive_addresses, self.output_addresses = receive_addresses, output_addresses
         self.barrier = barrier
 
@@ -203,14 +226,15 @@ def ep_replay_layer_direct(state: "EpDirectRank", buffers: PeerBuffers, x, w_rou
         dist.all_gather_into_tensor(counts_all, counts, group=group)
     else:
         counts_all = counts.view(1, -1)
-    rows = state.plan(counts_all)
-    if rows > buffers.received.shape[0]:
-        raise ValueError("receive buffer too small for the rows routed to this rank")
-    state.send(buffers.receive_addresses)
+    state.plan(counts_all)
+    # every rank sees the same totals: all of them stop here together, before anybody has
+    # written into a peer's memory (the kernels also refuse to store beyond the capacity)
+    check_capacity(state.owner_rows, buffers.capacity_rows)
+    state.send(buffers.receive_addresses, buffers.capacity_rows)
     buffers.barrier()                       # every rank's rows have landed everywhere
     state.experts(buffers.received, w_gate, w_up, w_down, buffers.outputs)
     buffers.barrier()                       # every owner's outputs are complete
-    result = state.finish(buffers.output_addresses, dy)
+    result = state.finish(buffers.output_addresses, dy, buffers.capacity_rows)
     buffers.barrier()                       # nobody overwrites a buffer that is still being read
     return result
 

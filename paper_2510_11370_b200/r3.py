@@ -48,6 +48,7 @@ EXPORTS = [
     "r3_record_page_bytes", "r3_record_append", "r3_record_gather",
     "r3_pagepool_create", "r3_pagepool_destroy", "r3_pagepool_free_pages", "r3_pagepool_match",
     "r3_pagepool_alloc", "r3_pagepool_publish", "r3_pagepool_release",
+    "r3_selftest_bounded_wait",
 ]
 
 
@@ -71,8 +72,9 @@ lib.r3_replay_stack_train_workspace_bytes.argtypes = [_SP, ctypes.c_int32]
 lib.r3_replay_stack_train.argtypes = [_SP, ctypes.c_int32] + [_P] * 15 + [ctypes.c_size_t, _P, _P]
 lib.r3_ep_regroup_map.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _P, _P, _P, _P]
 lib.r3_ep_dest_table.argtypes = [_P, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _P, _P, _P]
-lib.r3_ep_dispatch_rows.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, _P]
-lib.r3_ep_slot_rows.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, _P]
+lib.r3_ep_dispatch_rows.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, _P, ctypes.c_int64,
+                                    _P, _P]
+lib.r3_ep_slot_rows.argtypes = [_SP, ctypes.c_int32, _P, _P, _P, _P, _P, ctypes.c_int64, _P, _P, _P]
 lib.r3_replay_finish_rows.argtypes = [_SP] + [_P] * 10
 lib.r3_ep_move_rows.argtypes = [_P, _P, _P, ctypes.c_int32, ctypes.c_size_t, ctypes.c_int32, _P]
 lib.r3_grouped_swiglu_bwd.argtypes = [_SP] + [_P] * 13 + [ctypes.c_size_t, _P, _P]
@@ -125,6 +127,7 @@ lib.r3_pagepool_match.argtypes = [_P, _P, _I32, _P, _I32]
 lib.r3_pagepool_alloc.argtypes = [_P, _I32, _P]
 lib.r3_pagepool_publish.argtypes = [_P, _P, _I32, _P, _I32]
 lib.r3_pagepool_release.argtypes = [_P, _P, _I32]
+lib.r3_selftest_bounded_wait.argtypes = [ctypes.c_int64, _P, _P, _P]
 _NOT_STATUS = ("r3_status_string", "r3_pagepool_create", "r3_pagepool_destroy")
 for _n in EXPORTS:
     if _n not in _NOT_STATUS and not _n.endswith("_bytes"):
@@ -744,21 +747,23 @@ def ep_dest_table(counts_all, rank: int, *, stream=None):
 
 
 def ep_dispatch_rows(s: Shape, n_ranks: int, x, idx, row_of_slot, my_offsets, dst_base,
-                     peer_addresses, *, stream=None):
-    """x[t] straight into the owners' receive buffers (peer_addresses: their base addresses)."""
+                     peer_addresses, capacity_rows: int, *, dev_status=None, stream=None):
+    """x[t] straight into the owners' receive buffers (peer_addresses: their base addresses,
+    capacity_rows rows each; a row beyond the capacity is dropped and flagged)."""
     arr = _peer_array(peer_addresses)
     _check(lib.r3_ep_dispatch_rows(ctypes.byref(s), n_ranks, _ptr(x), _ptr(idx), _ptr(row_of_slot),
-                                   _ptr(my_offsets), _ptr(dst_base), arr, _stream(stream)))
+                                   _ptr(my_offsets), _ptr(dst_base), arr, int(capacity_rows),
+                                   _ptr(dev_status), _stream(stream)))
 
 
 def ep_slot_rows(s: Shape, n_ranks: int, idx, row_of_slot, my_offsets, dst_base, peer_addresses,
-                 *, stream=None):
+                 capacity_rows: int, *, dev_status=None, stream=None):
     """[T, K] addresses of the pairs' expert-output rows in the owners' output buffers."""
     row_ptr = torch.empty((s.T, s.K), dtype=torch.int64, device=_dev(idx))
     arr = _peer_array(peer_addresses)
     _check(lib.r3_ep_slot_rows(ctypes.byref(s), n_ranks, _ptr(idx), _ptr(row_of_slot),
-                               _ptr(my_offsets), _ptr(dst_base), arr, _ptr(row_ptr),
-                               _stream(stream)))
+                               _ptr(my_offsets), _ptr(dst_base), arr, int(capacity_rows),
+                               _ptr(row_ptr), _ptr(dev_status), _stream(stream)))
     return row_ptr
 
 
@@ -799,3 +804,12 @@ def grouped_swiglu_bwd_input(s: Shape, dout, pre_gate, pre_up, offsets, w_gate, 
                                            _ptr(w_down), _ptr(dxp), _ptr(ws), ws.numel(),
                                            _ptr(dev_status), _stream(stream)))
     return dxp
+
+
+def selftest_bounded_wait(limit_clocks: int, *, dev_status=None, device="cuda", stream=None):
+    """Makes the library's bounded barrier wait run out on purpose (a barrier nothing signals).
+    Returns out [4] int32: (wait result, abort flag, clocks waited, result of a second wait)."""
+    out = torch.full((4,), -1, dtype=torch.int32, device=device)
+    _check(lib.r3_selftest_bounded_wait(int(limit_clocks), _ptr(dev_status), _ptr(out),
+                                        _stream(stream)))
+    return out

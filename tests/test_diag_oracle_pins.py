@@ -27,6 +27,9 @@ def test_k3_and_extreme_counts_match_the_hand_derived_values():
     assert D.extreme_counts(g["p_train"], g["p_infer"], g["taus"]).tolist() == [int(c) for c in g["counts"]]
     assert np.allclose(D.extreme_fraction(g["p_train"], g["p_infer"], g["taus"]),
                        np.array(g["counts"]) / 4)
+    # ratios one part in a million either side of a threshold fall on the right side of it
+    assert D.extreme_counts(g["near_p_train"], g["near_p_infer"], g["near_taus"]).tolist() == \
+        [int(c) for c in g["near_counts"]]
 
 
 def test_k3_special_cases():
@@ -51,9 +54,8 @@ def test_extreme_fraction_properties():
     assert np.all(np.diff(f) <= 0)                                   # non-increasing in tau
     assert np.array_equal(D.extreme_counts(p, q, taus), D.extreme_counts(q, p, taus))   # symmetric
     assert D.extreme_counts(p, p, [1.0])[0] == 0                     # strict inequality
-    p32, q32 = p.astype(np.float32), q.astype(np.float32)            # brute force, float32 ratios
-    brute = [sum(1 for a, b in zip(p32, q32) if max(a / b, b / a) > np.float32(t)) for t in taus]
-    assert D.extreme_counts(p, q, taus).tolist() == brute
+    brute = [sum(1 for a, b in zip(p.tolist(), q.tolist()) if max(a / b, b / a) > t) for t in taus]
+    assert D.extreme_counts(p, q, taus).tolist() == brute            # brute force, Python floats
 
 
 def test_router_level_diff_against_sets_and_special_cases():

@@ -1,5 +1,8 @@
 """Discrepancy measures of Sections 3.1-3.2 on the GPU against the oracle: integer outputs bit for
-bit, the k3 estimate within 1e-5 relative (terms formed in float32, summed in float64)."""
+bit, the k3 estimate within 1e-5 relative (terms formed in float32, summed in float64).  The
+extreme-token counts are integer decisions that the kernel takes on float32 ratios and the oracle
+on exact (float64) ones: they may differ only by tokens whose exact ratio lies within one float32
+ulp of the threshold, and those tokens are counted."""
 import numpy as np
 import pytest
 import torch
@@ -25,6 +28,39 @@ def probs(n, seed, spread):
     return pt.float(), pi.float()
 
 
+def check_extreme_counts(got, pt, pi, taus):
+    """got[i] against the oracle's count for taus[i] (the float32 value the kernel is given).  A
+    correctly rounded float32 ratio is within half an ulp of the exact one, so only a token whose
+    exact ratio is within tau * 2^-23 of tau may be decided the other way."""
+    big = D.extreme_ratio(pt, pi)
+    near_total = 0
+    for c, t in zip(got, taus):
+        t = float(np.float32(t))
+        lo = int(np.count_nonzero(big > t * (1 + 2.0 ** -23)))
+        hi = int(np.count_nonzero(big > t * (1 - 2.0 ** -23)))
+        near_total += hi - lo
+        assert lo <= c <= hi, (t, c, lo, hi)
+        if hi == lo:
+            assert c == int(D.extreme_counts(pt, pi, [t])[0])
+    return near_total
+
+
+def test_extreme_counts_just_either_side_of_a_threshold(r3):
+    """The hand-derived tokens of tests/golden/k3_and_etdf_closed_form.txt whose ratios sit one
+    part in a million above and below tau = 2 (all values exact in float32)."""
+    import os
+    g = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "k3_and_etdf_closed_form.txt")):
+        if line.strip() and not line.startswith("#"):
+            k, *v = line.split()
+            g[k] = [float(x) for x in v]
+    pt = torch.tensor(g["near_p_train"], dtype=torch.float32)
+    pi = torch.tensor(g["near_p_infer"], dtype=torch.float32)
+    assert pt.double().tolist() == g["near_p_train"]             # stored exactly
+    _, counts = r3.prob_discrepancy(pt.cuda(), pi.cuda(), g["near_taus"])
+    assert counts.cpu().tolist() == [int(c) for c in g["near_counts"]]
+
+
 @pytest.mark.parametrize("n,spread", [(1, 0.1), (1000, 0.05), (300_001, 0.3), (5_000_000, 0.1)])
 def test_k3_and_extreme_counts(r3, n, spread):
     pt, pi = probs(n, n, spread)
@@ -33,7 +69,7 @@ def test_k3_and_extreme_counts(r3, n, spread):
     ref_kl = D.kl_k3(pt.numpy(), pi.numpy())
     # float32 terms (relative error below 1e-5 each), float64 sum
     assert abs(kl.item() - ref_kl) <= 1e-5 * abs(ref_kl) + 1e-12
-    assert counts.cpu().tolist() == D.extreme_counts(pt.numpy(), pi.numpy(), taus).tolist()
+    check_extreme_counts(counts.cpu().tolist(), pt.numpy(), pi.numpy(), taus)
     kl2, counts2 = r3.prob_discrepancy(pt.cuda(), pi.cuda(), taus)
     assert kl2.item() == kl.item() and torch.equal(counts, counts2)      # reproducible
 

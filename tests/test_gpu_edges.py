@@ -196,3 +196,56 @@ def test_backward_entry_points_reject_float32_and_accept_no_tokens(r3):
         r3.replay_layer_train(s, c["x"], c["w_r"], c["idx"], c["w_gate"], c["w_up"], c["w_down"],
                               c["dy"], ws=ws)
     assert err.value.code == r3.R3_ERR_UNSUPPORTED
+
+
+def test_a_bounded_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable(r3):
+    """The pipelines of the tensor-core kernels never spin for ever: a barrier wait gives up
+    after its clock limit, raises the abort flag and reports R3_DEV_TIMEOUT.  The self-test entry
+    point makes exactly that happen (a barrier nothing signals, 200 000 clocks = about 0.1 ms)."""
+    st = r3.new_status("cuda")
+    out = r3.selftest_bounded_wait(200_000, dev_status=st)
+    torch.cuda.synchronize()
+    waited, second = int(out[2]), int(out[3])
+    assert int(out[0]) == 0 and int(out[1]) == 1          # gave up, abort flag raised
+    assert 200_000 <= waited < 50_000_000                 # after the limit, and not much later
+    assert second == 0                                    # a later wait in the aborting CTA returns at once
+    assert st.item() == r3.DEV_TIMEOUT
+    # first error wins: a second run does not overwrite the word; a fresh word is set again
+    r3.selftest_bounded_wait(1000, dev_status=st)
+    assert st.item() == r3.DEV_TIMEOUT
+    with pytest.raises(r3.R3Error):
+        r3.selftest_bounded_wait(0)
+    with pytest.raises(r3.R3Error):
+        r3.selftest_bounded_wait(3_000_000_000)
+    # the context is intact: an ordinary tensor-core call right after is clean and correct
+    T, d, E, K = 300, 256, 32, 4
+    x = torch.randn(T, d).to(torch.bfloat16).cuda()
+    w = (torch.randn(E, d) * 0.1).to(torch.bfloat16).cuda()
+    s = r3.make_shape(T, d, E, K, 8, router=torch.bfloat16)
+    idx, logits = r3.capture_topk(s, x, w, want_logits=True)
+    torch.cuda.synchronize()
+    ref = x.float() @ w.float().T
+    assert torch.allclose(logits, ref, atol=1e-2) and idx.shape == (T, K)
+
+
+def test_gate_bwd_refuses_a_misaligned_dlogits_instead_of_faulting(r3):
+    """dlogits rows are written in 16-byte pieces; a view that starts 4 bytes into an allocation
+    is refused on the host (R3_ERR_INVALID_ARG), nothing is launched."""
+    T, E, K = 64, 128, 8
+    rng = np.random.default_rng(1)
+    idx = random_record(rng, T, E, K, torch.uint8).cuda()
+    g = torch.softmax(torch.randn(T, K), dim=1).cuda()
+    dg = torch.randn(T, K).cuda()
+    s = r3.make_shape(T, 8, E, K, 8)
+    backing = torch.full((T * E + 4,), 7.0, dtype=torch.float32, device="cuda")
+    view = backing[1:1 + T * E].view(T, E)
+    assert view.data_ptr() % 16 == 4 and view.is_contiguous()
+    with pytest.raises(r3.R3Error) as err:
+        r3.replay_gate_bwd(s, g, dg, idx, dlogits=view)
+    assert err.value.code == r3.R3_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert torch.all(backing == 7.0)
+    ok = backing[4:4 + T * E].view(T, E)
+    ds = r3.replay_gate_bwd(s, g, dg, idx, dlogits=ok)
+    ref = O.replay_gate_bwd(g.cpu().numpy(), dg.cpu().numpy(), idx.cpu().to(torch.int64).numpy(), E)
+    assert rel_err(ds.cpu().numpy(), ref) < TOL_F32

@@ -161,11 +161,12 @@ def test_direct_write_ranks_equal_the_single_gpu_layer(r3, world):
     ranks = [EpDirectRank(q, world, Tl, d, E, K, F) for q in range(world)]
     counts_all = torch.stack([rk.route(xs[tok(q)], w_r_d, idxs[tok(q)])
                               for q, rk in enumerate(ranks)])           # the all-gather
-    recv = [torch.full((max(rk.plan(counts_all), 1), d), float("nan"), dtype=torch.bfloat16,
-                       device=dev) for rk in ranks]
+    cap = max(max(rk.plan(counts_all) for rk in ranks), 1)               # one capacity for all
+    assert all(rk.owner_rows == ranks[0].owner_rows for rk in ranks)
+    recv = [torch.full((cap, d), float("nan"), dtype=torch.bfloat16, device=dev) for rk in ranks]
     outs = [torch.empty_like(b) for b in recv]
     for rk in ranks:
-        rk.send([b.data_ptr() for b in recv])
+        rk.send([b.data_ptr() for b in recv], cap)
     torch.cuda.synchronize()                                             # barrier 1
     assert sum(rk.recv_rows for rk in ranks) == T * K
     for q, rk in enumerate(ranks):
@@ -175,11 +176,41 @@ def test_direct_write_ranks_equal_the_single_gpu_layer(r3, world):
                    outs[q])
     torch.cuda.synchronize()                                             # barrier 2
     for q, rk in enumerate(ranks):
-        y, dlogits, gates = rk.finish([b.data_ptr() for b in outs], dys[tok(q)])
+        y, dlogits, gates = rk.finish([b.data_ptr() for b in outs], dys[tok(q)], cap)
         torch.cuda.synchronize()
         assert rk.status.item() == 0
         assert torch.equal(y, y_ref[tok(q)]) and torch.equal(dlogits, ds_ref[tok(q)])
         assert torch.equal(gates, g_ref[tok(q)])
+
+
+def test_direct_form_refuses_buffers_that_are_too_small(r3):
+    """A receive buffer smaller than the rows routed to its owner: the driver raises before any
+    row is stored, and the kernels themselves never write beyond the capacity they are given (a
+    canary behind the buffer stays intact, the status word reports the dropped rows)."""
+    from paper_2510_11370_b200.ep import EpDirectRank, PeerBuffers, ep_replay_layer_direct
+    T, d, E, K, F = 300, 256, 16, 4, 128
+    w, x, dy, w_r, wg, wu, wd, idx = _case(T, d, E, K, F)
+    c = [t.cuda() for t in (x, w_r, idx, wg, wu, wd, dy)]
+    small = PeerBuffers.single(T * K - 100, d, torch.bfloat16, "cuda")
+    with pytest.raises(ValueError, match="too small"):
+        ep_replay_layer_direct(EpDirectRank(0, 1, T, d, E, K, F), small, *c)
+    # the kernels alone, with the host check bypassed
+    rk = EpDirectRank(0, 1, T, d, E, K, F)
+    counts = rk.route(c[0], c[1], c[2])
+    rk.plan(counts.view(1, -1))
+    cap = T * K - 100
+    buf = torch.zeros((T * K, d), dtype=torch.bfloat16, device="cuda")   # canary: rows >= cap
+    rk.send([buf.data_ptr()], cap)
+    torch.cuda.synchronize()
+    assert rk.status.item() == r3.DEV_BAD_INDEX
+    assert not buf[cap:].any() and buf[:cap].any()
+    rk.status.zero_()
+    row_ptr = r3.ep_slot_rows(rk.shape, 1, rk.idx, rk.row_of_slot, rk.offsets, rk.dst_base,
+                              [buf.data_ptr()], cap, dev_status=rk.status)
+    torch.cuda.synchronize()
+    assert rk.status.item() == r3.DEV_BAD_INDEX
+    beyond = (rk.row_of_slot.reshape(-1) >= cap)                         # one rank: place = row
+    assert torch.all(row_ptr.reshape(-1)[beyond] == 0) and torch.all(row_ptr.reshape(-1)[~beyond] != 0)
 
 
 def test_direct_form_driver_with_one_rank(r3):

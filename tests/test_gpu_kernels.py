@@ -206,6 +206,19 @@ def test_replay_finish_flags_bad_records_and_rejects_wide_k(r3):
 
 
 # ------------------------------------------------------------------ capture: logits + TopKMask
+def plant_signed_zeros(x, w):
+    """Logits that are zero with either sign.  Token 7 is all +0 and token 9 all -0, expert 3 has
+    only negative and expert 1 only positive weights, so the products of those tokens are zeros of
+    both signs and a sum of them may come out as -0.0 or +0.0 depending on the order and the unit
+    that adds them.  TopKMask orders VALUES: -0.0 and +0.0 are the same logit, a tie, and the
+    lower expert index wins (for tokens 7 and 9 the record is 0, 1, ..., K-1)."""
+    x[7] = 0.0
+    x[9] = -0.0
+    w[3] = -1.0
+    w[1] = 1.0
+    w[11] = -2.0
+
+
 @pytest.mark.parametrize("act,rw", [(torch.float32, torch.float32), (torch.bfloat16, torch.float32),
                                     (torch.bfloat16, torch.bfloat16)])
 def test_capture_exact_arithmetic_with_planted_ties(r3, act, rw):
@@ -217,6 +230,7 @@ def test_capture_exact_arithmetic_with_planted_ties(r3, act, rw):
     w = torch.from_numpy(rng.integers(-2, 3, (E, d)).astype(np.float32)).to(rw)
     w[5] = w[2]
     w[17] = w[2]                                       # three experts always tie
+    plant_signed_zeros(x, w)
     s = r3.make_shape(T, d, E, K, 8, act=act, router=rw)
     idx, logits = r3.capture_topk(s, x.cuda(), w.cuda(), want_logits=True)
     ref_s = O.router_logits(f64(x), f64(w))
@@ -236,6 +250,7 @@ def test_capture_tensor_core_exact_arithmetic_with_planted_ties(r3, rw, T, d, E,
     w[5] = w[2]
     w[17] = w[2]
     w[E - 1] = w[0]
+    plant_signed_zeros(x, w)
     s = r3.make_shape(T, d, E, K, 8, router=rw)
     idx, logits = r3.capture_topk_ws(s, 1, x.cuda(), w.cuda(), want_logits=True)
     ref_s = O.router_logits(f64(x), f64(w))

@@ -100,15 +100,71 @@ def test_config2_bf16_layer_full(r3):
 
 
 def sampled_check(case, got, n_samples, tol, seed=0):
-    """Tokens the oracle evaluates one at a time straight from the equations."""
+    """Sampled tokens through the oracle's layer (every token's result depends on that token
+    alone, so the oracle is run on the sampled rows as a batch of their own): y and dlogits of
+    those tokens, and - when the run kept them - the expert outputs o of their K rows."""
     w = case.w
     rng = np.random.default_rng(seed)
     sel = np.sort(rng.choice(w.T, size=n_samples, replace=False))
-    y_ref, ds_ref = O.layer_tokens(f64(case.x[sel]), f64(case.w_r), case.idx_np()[sel],
-                                   case.w_gate, case.w_up, case.w_down, f64(case.dy[sel]))
-    y_all, ds_all = f64(got["y"]), f64(got["ds"])
-    assert np.abs(y_all[sel] - y_ref).max() / np.abs(y_ref).max() < tol
-    assert np.abs(ds_all[sel] - ds_ref).max() / np.abs(ds_ref).max() < tol
+    ref = O.layer_fwd_bwd(f64(case.x[sel]), f64(case.w_r), case.idx_np()[sel], case.w_gate,
+                          case.w_up, case.w_down, f64(case.dy[sel]))
+    tsel = torch.from_numpy(sel)
+    err_y = rel_err(f64(got["y"].cpu()[tsel]), ref["y"])
+    err_ds = rel_err(f64(got["ds"].cpu()[tsel]), ref["ds"])
+    assert err_y < tol and err_ds < tol, (err_y, err_ds)
+    errs = dict(y=err_y, ds=err_ds)
+    if "o" in got:
+        rows = got["ros"].cpu()[tsel].to(torch.int64)                 # [n, K] grouped rows
+        o_rows = f64(got["o"].cpu()[rows.reshape(-1)]).reshape(n_samples, w.K, w.d)
+        errs["o"] = rel_err(o_rows, ref["eo"])
+        assert errs["o"] < tol, errs
+    return errs
+
+
+def expert_rows_check(case, got, experts, tol):
+    """ALL rows of the given experts: o[offsets[e] : offsets[e+1]] against the oracle's expert
+    network on the rows the oracle's own dispatch gives that expert (the dispatch itself is
+    compared bit for bit elsewhere in the same test).  Returns {expert: (rows, error)}."""
+    w = case.w
+    _, offsets, _, sor = O.permutation(case.idx_np(), w.E)
+    o = got["o"]
+    out = {}
+    for e in experts:
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi == lo:
+            out[int(e)] = (0, 0.0)
+            continue
+        tokens = torch.from_numpy(sor[lo:hi].astype(np.int64) // w.K)
+        ref = O.swiglu_expert(f64(case.x[tokens]), case.w_gate[e], case.w_up[e], case.w_down[e])
+        err = rel_err(f64(o[lo:hi].cpu()), ref)
+        assert err < tol, (int(e), hi - lo, err)
+        out[int(e)] = (hi - lo, err)
+    return out
+
+
+def pick_experts(counts):
+    """Experts whose row counts exercise the tile schedule: the largest, one just over one
+    256-row tile (closest to 257..272), one whose count is not a multiple of 16, the smallest
+    non-empty one, and every empty one's two neighbours."""
+    counts = np.asarray(counts)
+    chosen = [int(np.argmax(counts))]
+    over = np.where(counts > 256)[0]
+    if over.size:
+        chosen.append(int(over[np.argmin(np.abs(counts[over] - 264))]))
+    ragged = np.where((counts % 16 != 0) & (counts > 0))[0]
+    if ragged.size:
+        chosen.append(int(ragged[np.argmin(counts[ragged])]))          # the smallest ragged one
+        chosen.append(int(ragged[np.argmax(counts[ragged] % 16)]))
+    nonempty = np.where(counts > 0)[0]
+    chosen.append(int(nonempty[np.argmin(counts[nonempty])]))
+    for e in np.where(counts == 0)[0]:
+        chosen += [int(x) for x in (e - 1, e + 1) if 0 <= x < counts.size and counts[x] > 0]
+    seen, out = set(), []
+    for e in chosen:
+        if e not in seen:
+            seen.add(e)
+            out.append(e)
+    return out
 
 
 class LazyWeights:
@@ -152,10 +208,10 @@ def run_big(r3, case, raw):
     assert torch.equal(y, y2) and torch.equal(g, g2)
     assert (ds - ds2).abs().max().item() <= 1e-5 * ds.abs().max().item()
     return dict(y=y, ds=ds, g=g, logits=logits, counts=counts, offsets=offsets, ros=ros, sor=sor,
-                xp=xp)
+                xp=xp, o=o)
 
 
-def check_big(case, got, tol, n_samples=48):
+def check_big(case, got, tol, n_samples=256):
     w = case.w
     counts, offsets, ros, sor = O.permutation(case.idx_np(), w.E)
     assert np.array_equal(got["counts"].cpu().numpy(), counts)
@@ -165,7 +221,10 @@ def check_big(case, got, tol, n_samples=48):
     assert torch.equal(got["xp"].cpu(), case.x[torch.from_numpy(sor.astype(np.int64)) // w.K])
     assert rel_err(got["logits"].cpu().numpy(), case.s) < 1e-5
     assert rel_err(f64(got["g"]), O.replay_gate(case.s, case.idx_np())) < 1e-5
-    sampled_check(case, got, n_samples, tol)
+    errs = sampled_check(case, got, n_samples, tol)
+    rows = expert_rows_check(case, got, pick_experts(counts), tol)
+    print(f"{w.name}: {n_samples} sampled tokens {errs}; all rows of experts "
+          f"{ {e: (n, round(err, 5)) for e, (n, err) in rows.items()} }")
     return counts
 
 
@@ -179,6 +238,8 @@ def test_config3_skewed_routing_full_size(r3):
     # the Zipf bias really skews the load: a few experts take most rows, some take (almost) none
     assert counts.max() > 20 * max(1, np.median(counts)) or counts.max() > w.T // 2
     assert counts.min() < w.T * w.K // w.E // 4
+    # the largest expert spans over a hundred 256-row token tiles, and ragged tails exist
+    assert counts.max() > 100 * 256 and np.any(counts % 16 != 0)
 
 
 def test_config4_capture_then_replay_round_trip(r3):
@@ -218,11 +279,20 @@ def test_config4_capture_then_replay_round_trip(r3):
     assert st.item() == 0
     assert np.allclose(g.cpu().numpy().sum(axis=1), 1.0, atol=1e-5)
     rng = np.random.default_rng(1)
-    sel = np.sort(rng.choice(np.nonzero(same)[0], size=32, replace=False))
-    y_ref, ds_ref = O.layer_tokens(f64(case.x[sel]), f64(case.w_r), oracle_rec[sel],
-                                   case.w_gate, case.w_up, case.w_down, f64(case.dy[sel]))
-    assert np.abs(f64(y)[sel] - y_ref).max() / np.abs(y_ref).max() < TOL_BF16
-    assert np.abs(f64(ds)[sel] - ds_ref).max() / np.abs(ds_ref).max() < TOL_BF16
+    sel = np.sort(rng.choice(np.nonzero(same)[0], size=256, replace=False))
+    ref = O.layer_fwd_bwd(f64(case.x[sel]), f64(case.w_r), oracle_rec[sel], case.w_gate,
+                          case.w_up, case.w_down, f64(case.dy[sel]))
+    tsel = torch.from_numpy(sel)
+    err_y, err_ds = rel_err(f64(y.cpu()[tsel]), ref["y"]), rel_err(f64(ds.cpu()[tsel]), ref["ds"])
+    print(f"c4 round trip: 256 sampled tokens y {err_y:.2e} dlogits {err_ds:.2e}")
+    assert err_y < TOL_BF16 and err_ds < TOL_BF16
+    del y, ds, g
+
+    # the same batch replayed from the ORACLE's record (an input that does not come from the
+    # library): dispatch bit for bit, all rows of chosen experts, 256 sampled tokens
+    case.idx = torch.from_numpy(oracle_rec).to(torch.uint8)
+    got = run_big(r3, case, raw)
+    check_big(case, got, TOL_BF16)
 
 
 def test_host_buffer_layer_and_two_batches_in_flight(r3):
