@@ -9,19 +9,37 @@
 // the same fp32 TMEM accumulator: x is exact in bf16, so the logits keep float32-level accuracy
 // while the contraction runs on the tensor pipe.
 //
-// When the tiles are few (a single layer's decode batch, or the training logits of a few thousand
-// tokens: at most half as many tiles as SMs), two CTAs of a cluster share a tile: each contracts
-// half of the k blocks into its own accumulator and finishes half of the tile's tokens, reading
-// the other CTA's partial logits through distributed shared memory (the sum of the two partials is
-// the same number in both CTAs).
+// Orientation.  The EXPERT rows of W_r are the M side of the MMA (128 per M tile, up to two M
+// tiles) and the TOKENS are the N side (a tile of up to 256 tokens, any multiple of 16), so the
+// accumulator holds s^T: tensor-memory lane = expert, column = token.  A whole decode batch of a
+// layer (256 tokens) is then ONE tile whose router weights are fetched once.
 //
-// One CTA of 12 warps per 128-token tile: warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA
-// issuer, warps 2-5 read the finished accumulator out of TMEM into a [128][E + 1] float tile in
-// shared memory (the copy ring is free by then).  All 12 warps then finish tokens out of that
-// tile, four at a time per warp: the lanes write the token's logits out coalesced and pick the K
-// largest with K rounds of warp reductions on order-preserving integer keys (exact ties go to the
-// lower expert).  A per-thread sorted insertion list, one thread per token, took 12 us of
-// dependent compare-and-swaps per tile; this takes about a third of that.
+// K split.  The kernel is bound by bytes (4 KB of x per token for 0.5 MFLOP), so the bytes of a
+// tile are spread over several SMs whenever the tiles are fewer than the SMs: the CTAs of a
+// cluster share a tile, each contracting its own range of the k blocks into its own accumulator,
+// and each finishes its share of the tile's tokens.  The partial logits travel between the CTAs
+// in one of two ways:
+//   two CTAs   every CTA moves its whole accumulator into its own shared memory [token][experts+1]
+//              and PUSHES the rows of the other CTA's tokens to it with one bulk asynchronous copy
+//              (shared memory to the peer's shared memory, completion on the peer's barrier); no
+//              cluster barrier is needed after the start;
+//   3..8 CTAs  (one layer's decode batch) every CTA stores each token's values straight into the
+//              shared memory of the CTA that finishes the token (st.shared::cluster, 32 consecutive
+//              words per instruction) into the slot of its own rank, between two cluster barriers.
+// Measured on one layer's decode batch split 8 ways: reading the partials with ld.shared::cluster
+// cost about 1.6 us per dependent round trip (13 us of 21), the remote stores cost 6 us.  The
+// partial sums are added in rank order (a fixed order: reproducible).
+//
+// One CTA of 12 warps per (tile, k range): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA
+// issuer; then all 12 warps move the finished accumulator out of TMEM (transposed on the way:
+// tensor-memory lane = expert, but a token's experts must lie next to each other), and TopKMask
+// is taken by FOUR lanes per token on packed candidates in registers (thread_topk below), with a
+// warp-wide exact selection for the few tokens that the packed form cannot decide.  The earlier
+// form, K rounds of two warp reductions per token, cost 9.6 us for the 128 tokens of a CTA.
+//
+// The kernel is launched with programmatic stream serialisation: everything up to its first
+// access to global memory (barrier set-up, tensor-memory allocation) may run while the previous
+// kernel of the stream drains, and it lets its own successor do the same once its copies are done.
 #include "r3_common.cuh"
 #include "r3_internal.h"
 #include "r3_tc.cuh"
@@ -31,15 +49,17 @@ namespace rt {
 
 using namespace tc;
 
-constexpr int BM = 128;
+constexpr int BME = 128;                 // expert rows per M tile (UMMA M)
 constexpr int BK = 64;
 constexpr int UK = 16;
-constexpr int A_BYTES = BM * BK * 2;
-constexpr int THREADS = 12 * 32;           // producer, MMA issuer, 4 TMEM readers; all 12 pick top-K
+constexpr int A_BYTES = BME * BK * 2;    // one M tile of one weight plane per stage
+constexpr int THREADS = 12 * 32;         // producer, MMA issuer, 4 TMEM readers; all 12 pick top-K
 constexpr int BAR_BYTES = 256;
 constexpr int MAX_STAGES = 7;
-constexpr int KMAX = 16;                 // longest record the register top-K list supports
+constexpr int KMAX = 16;                 // longest record the warp top-K supports (one lane per slot)
 constexpr int SMEM_LIMIT = 227 * 1024;
+constexpr int MAX_SPLIT = 8;             // portable cluster size
+constexpr int GROUP = 4;                 // lanes that share a token in the TopKMask
 
 __global__ void __launch_bounds__(256)
 split_router_weight_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ planes,
@@ -58,119 +78,266 @@ split_router_weight_kernel(const float* __restrict__ w, __nv_bfloat16* __restric
     base[2 * per_layer] = lo;
 }
 
-// One warp finishes NT tokens at a time out of the shared-memory logits tile: lane l holds the
-// logits of experts l + 32 s (slot s), writes them out (coalesced) and, if a record is wanted,
-// picks the K largest by K rounds of warp reductions on order-preserving integer keys; exact ties
-// go to the lower expert.  NT tokens are interleaved so that their reduction chains overlap.
-template <typename IdxT, int SLOTS, int NT>
-__device__ __forceinline__ void finish_tokens(const float* tile, int LD, const int* rows, int n_rows,
-                                              int lane, int E, int K, size_t out_row0,
-                                              IdxT* idx_out, float* logits_out,
-                                              uint32_t peer_tile) {
-    uint32_t key[NT][SLOTS];
-    float val[NT][SLOTS];
-    // all reads of the tile(s) first: the global stores below might alias them for the compiler
-#pragma unroll
-    for (int a = 0; a < NT; ++a) {
-#pragma unroll
-        for (int sl = 0; sl < SLOTS; ++sl) {
-            const int e = lane + 32 * sl;
-            val[a][sl] = 0.f;
-            if (a < n_rows && e < E) {
-                float v = tile[(size_t)rows[a] * LD + e];
-                if (peer_tile) {                         // the other half of the contraction
-                    float w;
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];"
-                                 : "=f"(w) : "r"(peer_tile + 4u * (uint32_t)(rows[a] * LD + e)));
-                    v += w;
-                }
-                val[a][sl] = v;
-            }
-        }
-    }
-#pragma unroll
-    for (int a = 0; a < NT; ++a) {
-#pragma unroll
-        for (int sl = 0; sl < SLOTS; ++sl) {
-            const int e = lane + 32 * sl;
-            key[a][sl] = 0u;                             // 0 = no candidate (below every real key)
-            if (a < n_rows && e < E) {
-                const float v = val[a][sl];
-                if (logits_out) logits_out[(out_row0 + rows[a]) * E + e] = v;
-                // order-preserving key; -0.0 and +0.0 are one value (a tie: lower expert wins)
-                uint32_t u = __float_as_uint(v);
-                if (u == 0x80000000u) u = 0u;
-                const uint32_t k2 = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-                key[a][sl] = k2 ? k2 : 1u;
-            }
-        }
-    }
-    if (!idx_out) return;
-    int mine[NT];
-#pragma unroll
-    for (int a = 0; a < NT; ++a) mine[a] = 0;
-    for (int j = 0; j < K; ++j) {
-#pragma unroll
-        for (int a = 0; a < NT; ++a) {
-            uint32_t best = 0u;
-#pragma unroll
-            for (int sl = 0; sl < SLOTS; ++sl) best = max(best, key[a][sl]);
-            const uint32_t top = __reduce_max_sync(0xffffffffu, best);
-            uint32_t cand = 0xffffffffu;                 // lowest expert of this lane with that key
-#pragma unroll
-            for (int sl = SLOTS - 1; sl >= 0; --sl)
-                if (key[a][sl] == top) cand = (uint32_t)(lane + 32 * sl);
-            const uint32_t win = __reduce_min_sync(0xffffffffu, cand);
-#pragma unroll
-            for (int sl = 0; sl < SLOTS; ++sl)
-                if (win == (uint32_t)(lane + 32 * sl)) key[a][sl] = 0u;
-            if (lane == j) mine[a] = (int)win;
-        }
-    }
-#pragma unroll
-    for (int a = 0; a < NT; ++a)
-        if (a < n_rows && lane < K) idx_out[(out_row0 + rows[a]) * K + lane] = (IdxT)mine[a];
+// Order-preserving integer key of a logit: a < b as floats  <=>  key(a) < key(b) as unsigned.
+// -0.0 and +0.0 are one value (a tie); 0 is reserved for "no candidate".
+__device__ __forceinline__ uint32_t logit_key(float v) {
+    const uint32_t u = __float_as_uint(v + 0.0f);        // -0.0 + 0.0 = +0.0
+    // negative: all bits flipped; positive: sign bit set
+    const uint32_t k = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+    return k ? k : 1u;
 }
 
+// Where the partial logits of the tokens a CTA finishes lie in its shared memory: the value of
+// (row, expert) is the sum over the ranks r = 0 .. n - 1, in that order, of the words at
+// p0 (rank 0), p1 (rank 1), p1 + stride (rank 2), ..., each at offset row * LD + e.
+struct Partials {
+    const float* p0;
+    const float* p1;
+    int stride, n;
+    // CNT values at offsets off + i * STEP: all loads of a rank are issued together (a loop over
+    // the ranks inside a loop over the values made every load wait for the one before it)
+    template <int CNT, int STEP>
+    __device__ __forceinline__ void sum(int off, float* v) const {
+#pragma unroll
+        for (int i = 0; i < CNT; ++i) v[i] = p0[off + i * STEP];
+        if (n > 1) {
+#pragma unroll
+            for (int i = 0; i < CNT; ++i) v[i] += p1[off + i * STEP];
+            for (int r = 2; r < n; ++r) {
+                const float* q = p1 + (r - 1) * stride;
+#pragma unroll
+                for (int i = 0; i < CNT; ++i) v[i] += q[off + i * STEP];
+            }
+        }
+    }
+};
+
+// Exact TopKMask of one token by the whole warp: lane l holds the keys of experts l + 32 s; K
+// rounds of two warp reductions pick the largest key and, among equal keys, the lowest expert.
+// About 30 instructions per round and token: used only for the few tokens the packed selection
+// below cannot decide.
+template <typename IdxT, int SLOTS>
+__device__ __forceinline__ void warp_topk_exact(const Partials& ps, int LD, int row, int lane, int E,
+                                                int K, IdxT* out) {
+    uint32_t key[SLOTS];
+    float v[SLOTS];
+    ps.sum<SLOTS, 32>(row * LD + lane, v);               // 32 * SLOTS < LD: inside the row
+#pragma unroll
+    for (int sl = 0; sl < SLOTS; ++sl) key[sl] = lane + 32 * sl < E ? logit_key(v[sl]) : 0u;
+    int mine = 0;
+    for (int j = 0; j < K; ++j) {
+        uint32_t best = 0u;
+#pragma unroll
+        for (int sl = 0; sl < SLOTS; ++sl) best = max(best, key[sl]);
+        const uint32_t top = __reduce_max_sync(0xffffffffu, best);
+        uint32_t cand = 0xffffffffu;                     // lowest expert of this lane with that key
+#pragma unroll
+        for (int sl = SLOTS - 1; sl >= 0; --sl)
+            if (key[sl] == top) cand = (uint32_t)(lane + 32 * sl);
+        const uint32_t win = __reduce_min_sync(0xffffffffu, cand);
+#pragma unroll
+        for (int sl = 0; sl < SLOTS; ++sl)
+            if (win == (uint32_t)(lane + 32 * sl)) key[sl] = 0u;
+        if (lane == j) mine = (int)win;
+    }
+    if (lane < K) out[lane] = (IdxT)mine;
+}
+
+// A packed candidate is the logit itself (a float, after -0.0 -> +0.0) with its low 8 mantissa
+// bits replaced by a tag of the expert e (E <= 256): 255 - e for a positive logit, e for a
+// negative one.  Compared as FLOATS, a larger candidate has the larger logit truncated to 24 bits
+// (sign, exponent, 15 mantissa bits) and, among equal truncated logits, the LOWER expert (for a
+// negative number a smaller tag means a smaller magnitude, i.e. a larger value).  A
+// compare-exchange is one fminf and one fmaxf.  -inf = no candidate.
+__device__ __forceinline__ float pack_candidate(float v, int e) {
+    const uint32_t u = __float_as_uint(v + 0.0f);                       // -0.0 + 0.0 = +0.0
+    const uint32_t tag = (uint32_t)(255 - e) ^ ((uint32_t)((int32_t)u >> 31) & 255u);
+    return __uint_as_float((u & 0xffffff00u) | tag);
+}
+__device__ __forceinline__ int candidate_expert(float c) {
+    const uint32_t u = __float_as_uint(c);
+    return (int)(((u & 255u) ^ ((uint32_t)((int32_t)u >> 31) & 255u)) ^ 255u);
+}
+__device__ __forceinline__ void ce_desc(float& a, float& b) {           // a keeps the larger
+    const float hi = fmaxf(a, b), lo = fminf(a, b);
+    a = hi;
+    b = lo;
+}
+constexpr float kNoCandidate = -__builtin_huge_valf();
+
+// Sorts KM candidates in descending order: the 19-comparator network for 8, a bitonic network
+// for 16.
+template <int KM>
+__device__ __forceinline__ void sort_desc(float* c) {
+    if (KM == 8) {
+        ce_desc(c[0], c[2]); ce_desc(c[1], c[3]); ce_desc(c[4], c[6]); ce_desc(c[5], c[7]);
+        ce_desc(c[0], c[4]); ce_desc(c[1], c[5]); ce_desc(c[2], c[6]); ce_desc(c[3], c[7]);
+        ce_desc(c[0], c[1]); ce_desc(c[2], c[3]); ce_desc(c[4], c[5]); ce_desc(c[6], c[7]);
+        ce_desc(c[2], c[4]); ce_desc(c[3], c[5]);
+        ce_desc(c[1], c[4]); ce_desc(c[3], c[6]);
+        ce_desc(c[1], c[2]); ce_desc(c[3], c[4]); ce_desc(c[5], c[6]);
+    } else {
+#pragma unroll
+        for (int k = 2; k <= KM; k <<= 1) {
+#pragma unroll
+            for (int j = k >> 1; j > 0; j >>= 1) {
+#pragma unroll
+                for (int i = 0; i < KM; ++i) {
+                    const int l = i ^ j;
+                    if (l > i) {
+                        if ((i & k) == 0) ce_desc(c[i], c[l]); else ce_desc(c[l], c[i]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+// A sorted list of the KM largest candidates seen so far, plus the largest one dropped
+// (`runner` = the (KM+1)-th largest).
+template <int KM>
+struct TopList {
+    float top[KM];
+    float runner;
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int i = 0; i < KM; ++i) top[i] = kNoCandidate;
+        runner = kNoCandidate;
+    }
+    // Merges a list sorted in descending order (and its runner) into this one: max(a_i, b_{KM-1-i})
+    // are the KM largest of both (a bitonic sequence), a bitonic merge sorts them again.
+    __device__ __forceinline__ void merge(const float* b, float b_runner) {
+        float dropped[KM];
+#pragma unroll
+        for (int i = 0; i < KM; ++i) {
+            const float x = top[i], y = b[KM - 1 - i];
+            top[i] = fmaxf(x, y);
+            dropped[i] = fminf(x, y);
+        }
+#pragma unroll
+        for (int w = KM >> 1; w > 0; w >>= 1)                // a tree, not a chain
+#pragma unroll
+            for (int i = 0; i < w; ++i) dropped[i] = fmaxf(dropped[i], dropped[i + w]);
+        runner = fmaxf(fmaxf(runner, b_runner), dropped[0]);
+#pragma unroll
+        for (int j = KM >> 1; j > 0; j >>= 1) {
+#pragma unroll
+            for (int i = 0; i < KM; ++i) {
+                const int l = i ^ j;
+                if (l > i) ce_desc(top[i], top[l]);
+            }
+        }
+    }
+};
+
+// TopKMask of the tokens of one warp task: GROUP lanes share a token (lane = GROUP * token +
+// part); each takes every GROUP-th block of KM experts, sorts the block with a sorting network
+// and merges it into its list; the GROUP lists of a token are then merged through shuffles.  The
+// result is exact unless two candidates next to each other in the final order (down to the first
+// one left out) share their 24 leading bits while the full logits might differ; such a token is
+// flagged and repeated with warp_topk_exact (random logits: a few tokens in a thousand; planted
+// exact ties: every such token, still correct).  Returns the flags of the warp's tokens (bit =
+// lane of the token's first lane).
 template <typename IdxT, int KM>
+__device__ __forceinline__ uint32_t group_topk(const Partials& ps, int LD, int row, bool valid,
+                                               int part, int E, int K, IdxT* out) {
+    TopList<KM> list;
+    list.clear();
+    if (valid) {
+        for (int e0 = part * KM; e0 < E; e0 += GROUP * KM) {
+            float c[KM];
+            ps.sum<KM, 1>(row * LD + e0, c);
+#pragma unroll
+            for (int i = 0; i < KM; ++i) c[i] = pack_candidate(c[i], e0 + i);
+            sort_desc<KM>(c);
+            list.merge(c, kNoCandidate);
+        }
+    }
+    // the lists of the GROUP lanes of a token, merged pairwise (every lane ends with the result)
+#pragma unroll
+    for (int m = 1; m < GROUP; m <<= 1) {
+        float other[KM];
+#pragma unroll
+        for (int i = 0; i < KM; ++i) other[i] = __shfl_xor_sync(0xffffffffu, list.top[i], m);
+        const float other_runner = __shfl_xor_sync(0xffffffffu, list.runner, m);
+        list.merge(other, other_runner);
+    }
+    bool sure = true;
+    if (valid && part == 0) {
+#pragma unroll
+        for (int j = 0; j < KM; ++j) {
+            const float next = j + 1 < KM ? list.top[j + 1 < KM ? j + 1 : j] : list.runner;
+            if (j < K) {
+                if ((__float_as_uint(list.top[j]) >> 8) == (__float_as_uint(next) >> 8)) sure = false;
+                out[j] = (IdxT)candidate_expert(list.top[j]);
+            }
+        }
+    }
+    return __ballot_sync(0xffffffffu, !sure);
+}
+
+// grid = (token tiles of a layer * ksplit, L), cluster = (ksplit, 1, 1).  N = tokens per tile
+// (multiple of 16), MT = M tiles of 128 experts (1 or 2).  Shared memory: [ring_bytes: the copy
+// ring, later the logits of the accumulator / the slots of the partial logits and, from recv_off
+// on, the rows pushed by the other CTA of a pair][barriers].
+template <typename IdxT>
 __global__ void __launch_bounds__(THREADS, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                  IdxT* __restrict__ idx_out, float* __restrict__ logits_out, int T, int d, int E,
-                 int K, int planes, int stages, uint32_t tmem_cols, int ksplit) {
+                 int K, int planes, int stages, uint32_t tmem_cols, int ksplit, int N, int MT,
+                 int ring_bytes, int recv_off) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const int b_bytes = planes * E * BK * 2;
-    const int stage_bytes = A_BYTES + b_bytes;
-    const uint32_t bar0 = base + stages * stage_bytes;
+    const int a_bytes = planes * MT * A_BYTES;
+    const int stage_bytes = a_bytes + N * BK * 2;
+    const int LD = MT * BME + 1;                         // odd: rows start in different banks
+    const uint32_t recv0 = base + (uint32_t)recv_off;
+    const uint32_t bar0 = base + (uint32_t)ring_bytes;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
     const uint32_t acc_bar = bar0 + 8u * (2 * MAX_STAGES);
-    volatile uint32_t* tmem_slot =
-        reinterpret_cast<volatile uint32_t*>(base_ptr + stages * stage_bytes + 128);
-    volatile int* abort_flag =
-        reinterpret_cast<volatile int*>(base_ptr + stages * stage_bytes + 132);
+    const uint32_t push_bar = bar0 + 8u * (2 * MAX_STAGES + 1);
+    const uint32_t ready_bar = bar0 + 8u * (2 * MAX_STAGES + 2);
+    uint8_t* misc = base_ptr + ring_bytes + 128;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int layer = blockIdx.y;
-    // ksplit = 2: the two CTAs of a cluster (consecutive blockIdx.x) share a tile
-    const int rank = ksplit == 2 ? (int)cluster_ctarank() : 0;
-    const int t0 = (ksplit == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x) * BM;
+    const int rank = ksplit > 1 ? (int)cluster_ctarank() : 0;
+    const int t0 = (int)(blockIdx.x / (unsigned)ksplit) * N;
     const int kblocks = (d + BK - 1) / BK;
-    const int kb_per = (kblocks + ksplit - 1) / ksplit;
-    const int kb0 = rank * kb_per, kb1 = min(kblocks, kb0 + kb_per);    // this CTA's k blocks
+    // this CTA's k blocks (ranges differ by at most one block)
+    const int kb0 = (int)((long long)rank * kblocks / ksplit);
+    const int kb1 = (int)((long long)(rank + 1) * kblocks / ksplit);
+    // Token c of the tile is finished by CTA c / per as its row c % per; `per` is a multiple of 32,
+    // so the 32 tokens of one tensor-memory read go to one CTA.
+    const int n_all = max(0, min(N, T - t0));
+    const int per = ((n_all + ksplit - 1) / ksplit + 31) & ~31;
+    const int tok_lo = rank * per;
+    const int n_mine = max(0, min(per, n_all - tok_lo));
+    const bool pair = ksplit == 2;             // partial logits pushed with a bulk copy
+    const uint32_t push_bytes = (uint32_t)(per * LD * 4);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(acc_bar, 1);
+        mbar_init(push_bar, 1);
+        mbar_init(ready_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
+        // the rows the other CTA of the pair will push here
+        if (pair && n_mine > 0) mbar_expect_tx(push_bar, push_bytes);
     }
     if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), tmem_cols);
     tc_fence_before();
     __syncthreads();
+    if (ksplit > 1) cluster_sync_all();        // the peers' barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // nothing above touched global memory: it may have run beside the previous kernel of the stream
+    grid_dependency_wait();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -178,33 +345,37 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             uint32_t phase = 0;
             for (int kb = kb0; kb < kb1; ++kb) {
                 if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, nullptr)) break;
-                const uint32_t sa = base + stage * stage_bytes, sb = sa + A_BYTES;
+                const uint32_t sa = base + stage * stage_bytes, sb = sa + a_bytes;
                 mbar_expect_tx(full_bar(stage), (uint32_t)stage_bytes);
-                tma_load_2d(sa, &tmX, kb * BK, layer * T + t0, full_bar(stage));
+                tma_load_2d(sb, &tmX, kb * BK, layer * T + t0, full_bar(stage));
                 for (int p = 0; p < planes; ++p)
-                    tma_load_2d(sb + p * E * BK * 2, &tmW, kb * BK, (layer * planes + p) * E,
-                                full_bar(stage));
+                    for (int m = 0; m < MT; ++m)       // rows beyond E are filled with zeros
+                        tma_load_3d(sa + (p * MT + m) * A_BYTES, &tmW, kb * BK, m * BME,
+                                    layer * planes + p, full_bar(stage));
                 if (++stage == stages) { stage = 0; phase ^= 1u; }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(BM, E);
+            const uint32_t idesc = instr_desc_bf16(BME, N);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int kb = kb0; kb < kb1 && ok; ++kb) {
                 if (!mbar_wait(full_bar(stage), phase, abort_flag, nullptr)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t sa = base + stage * stage_bytes, sb = sa + A_BYTES;
-                const uint64_t da = smem_desc_sw128(sa);
-                for (int p = 0; p < planes; ++p) {
-                    const uint64_t db = smem_desc_sw128(sb + p * E * BK * 2);
+                const uint32_t sa = base + stage * stage_bytes, sb = sa + a_bytes;
+                const uint64_t db = smem_desc_sw128(sb);
+                for (int m = 0; m < MT; ++m) {
+                    for (int p = 0; p < planes; ++p) {
+                        const uint64_t da = smem_desc_sw128(sa + (p * MT + m) * A_BYTES);
 #pragma unroll
-                    for (int kk = 0; kk < BK / UK; ++kk)
-                        tc_mma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
-                                    idesc, ((kb - kb0) | p | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < BK / UK; ++kk)
+                            tc_mma_bf16(tmem_base + (uint32_t)(m * N), da + (uint64_t)(kk * 2),
+                                        db + (uint64_t)(kk * 2), idesc,
+                                        ((kb - kb0) | p | kk) != 0 ? 1u : 0u);
+                    }
                 }
                 tc_commit(empty_bar(stage));
                 if (++stage == stages) { stage = 0; phase ^= 1u; }
@@ -213,61 +384,143 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
         __syncwarp();
     } else if (warp < 6) {
-        // ------------------------------ epilogue, part 1 --------------------------------------
-        // every epilogue warp dumps its 32 tokens' logits from tensor memory into a [128][E + 1]
-        // float tile in shared memory (the copy ring is free once the accumulator is complete)
-        const int q = warp & 3;
-        float* tile = reinterpret_cast<float*>(base_ptr);
-        float* trow = tile + (size_t)(q * 32 + lane) * (E + 1);
-        if (kb1 <= kb0) {
-            for (int c = 0; c < E; ++c) trow[c] = 0.f;      // no k block fell to this CTA
-        } else if (__all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, nullptr))) {
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            for (int c = 0; c < E; c += 32) {
-                float v[32];
-                tc_ld32(taddr + c, v);
+        // the accumulator is complete: every copy has landed and every MMA has read its operands
+        if (kb1 > kb0) __all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, nullptr));
+    }
+    tc_fence_before();
+    __syncthreads();
+    // this grid has fetched its inputs: the next kernel of the stream may begin its set-up
+    grid_launch_dependents();
+    // a pair: this CTA has left its copy ring, the peer may push rows into it (the signal travels
+    // while the accumulator is moved out); 3..8 CTAs store into each other's rings right away:
+    // every CTA of the cluster must have left its ring first
+    if (pair && threadIdx.x == 0) mbar_arrive_cluster(mapa_shared(ready_bar, (uint32_t)(rank ^ 1)));
+    if (ksplit > 2) cluster_sync_all();
+
+    // ------------------------------ epilogue, part 1 ------------------------------------------
+    // Every warp moves 32 experts' partial logits of 32 tokens at a time out of tensor memory
+    // (one store instruction writes 32 consecutive words of a token's row):
+    //   one or two CTAs: into this CTA's own [token][LD] tile, all tokens of the tile;
+    //   more CTAs: into slot [this rank][row] of the CTA that finishes the token.
+    const int nchunk = (n_all + 31) >> 5;
+    auto store_chunks = [&](int chunk_lo, int chunk_hi) {
+        const int q = warp & 3;                // the tensor-memory lanes this warp may read
+        const int span = chunk_hi - chunk_lo;
+        // (M tile, 32-token chunk) pairs are dealt to the three warps of a lane quadrant
+        for (int p = warp >> 2; p < MT * span; p += 3) {
+            const int m = p / span, c = (chunk_lo + p - m * span) << 5;
+            float v[32];
+            if (kb1 > kb0) {
+                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(m * N + c), v);
                 tc_wait_ld();
+            } else {                                        // no k block fell to this CTA
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c + i < E) trow[c + i] = v[i];
+                for (int i = 0; i < 32; ++i) v[i] = 0.f;
+            }
+            const int e_off = m * BME + q * 32 + lane;
+            uint32_t dst;
+            if (ksplit <= 2) {
+                dst = base + 4u * (uint32_t)(c * LD + e_off);
+            } else {
+                const int owner = c / per, row0 = c - owner * per;
+                dst = mapa_shared(base + 4u * (uint32_t)((rank * per + row0) * LD + e_off),
+                                  (uint32_t)owner);
+            }
+            const int n_here = min(32, n_all - c);
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < n_here)
+                    asm volatile("st.shared::cluster.f32 [%0], %1;"
+                                 ::"r"(dst + 4u * (uint32_t)(i * LD)), "f"(v[i]) : "memory");
+        }
+    };
+    tc_fence_after();
+    if (pair) {
+        // the peer's tokens first: their rows leave with one bulk copy while this CTA's own rows
+        // are still being moved out of tensor memory
+        const int peer = rank ^ 1;
+        const int peer_lo = min(nchunk, (peer * per) >> 5), peer_hi = min(nchunk, ((peer + 1) * per) >> 5);
+        if (!*abort_flag) store_chunks(peer_lo, peer_hi);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (threadIdx.x == 0 && peer_hi > peer_lo && !*abort_flag &&
+            mbar_wait(ready_bar, 0u, abort_flag, nullptr)) {
+            asm volatile(
+                "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                ::"r"(mapa_shared(recv0, (uint32_t)peer)),
+                  "r"(base + (uint32_t)(peer * per) * (uint32_t)(LD * 4)), "r"(push_bytes),
+                  "r"(mapa_shared(push_bar, (uint32_t)peer)) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        const int own_lo = min(nchunk, tok_lo >> 5), own_hi = min(nchunk, (tok_lo + per) >> 5);
+        if (!*abort_flag) store_chunks(own_lo, own_hi);
+        tc_fence_before();
+        __syncthreads();
+        if (n_mine > 0) mbar_wait(push_bar, 0u, abort_flag, nullptr);
+    } else {
+        if (!*abort_flag) store_chunks(0, nchunk);
+        tc_fence_before();
+        __syncthreads();
+        if (ksplit > 2) cluster_sync_all();    // the partial logits of this CTA's tokens have landed
+    }
+
+    // ------------------------------ epilogue, part 2 --------------------------------------------
+    Partials ps;
+    {
+        const float* tile = reinterpret_cast<const float*>(base_ptr);
+        const float* recv = reinterpret_cast<const float*>(base_ptr + recv_off);
+        const float* own = tile + (size_t)tok_lo * LD;
+        ps.n = ksplit;
+        ps.stride = per * LD;
+        ps.p0 = tile;
+        ps.p1 = tile + (size_t)per * LD;
+        if (pair) {                            // rank order: the lower rank's partial first
+            ps.p0 = rank == 0 ? own : recv;
+            ps.p1 = rank == 0 ? recv : own;
+        }
+    }
+    const size_t out_row0 = (size_t)layer * T + t0 + tok_lo;
+    if (!*abort_flag && logits_out) {
+        // one warp per token, lane l writes the experts l, l + 32, ... (coalesced)
+        for (int row = warp; row < n_mine; row += THREADS / 32) {
+            float v[8];                                  // experts lane, lane + 32, ...
+            if (E <= 128) ps.sum<4, 32>(row * LD + lane, v); else ps.sum<8, 32>(row * LD + lane, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (lane + 32 * i < E) logits_out[(out_row0 + row) * E + lane + 32 * i] = v[i];
+        }
+    }
+    if (!*abort_flag && idx_out) {
+        // TopKMask: GROUP lanes per token, 32 / GROUP tokens per warp task
+        constexpr int TPW = 32 / GROUP;
+        for (int task = warp; task * TPW < n_mine; task += THREADS / 32) {
+            const int row = task * TPW + (lane / GROUP);
+            const bool valid = row < n_mine;
+            IdxT* out = idx_out + (out_row0 + (valid ? row : 0)) * K;
+            uint32_t redo = K <= 8
+                ? group_topk<IdxT, 8>(ps, LD, row, valid, lane % GROUP, E, K, out)
+                : group_topk<IdxT, 16>(ps, LD, row, valid, lane % GROUP, E, K, out);
+            while (redo) {
+                const int r2 = task * TPW + (__ffs(redo) - 1) / GROUP;
+                redo &= redo - 1;
+                if (E <= 128)
+                    warp_topk_exact<IdxT, 4>(ps, LD, r2, lane, E, K, idx_out + (out_row0 + r2) * K);
+                else
+                    warp_topk_exact<IdxT, 8>(ps, LD, r2, lane, E, K, idx_out + (out_row0 + r2) * K);
             }
         }
     }
-    // ------------------------------ epilogue, part 2: all twelve warps, a few tokens each -------
-    tc_fence_before();
-    __syncthreads();
-    if (ksplit == 2) cluster_sync_all();       // the other CTA's partial logits are in its tile
-    if (!*abort_flag) {
-        const float* tile = reinterpret_cast<const float*>(base_ptr);
-        const uint32_t peer_tile = ksplit == 2 ? mapa_shared(smem_u32(tile), (uint32_t)(rank ^ 1)) : 0u;
-        // with a shared tile each CTA finishes half of its tokens
-        const int n_all = min(BM, T - t0);
-        const int tok_lo = ksplit == 2 ? rank * (BM / 2) : 0;
-        const int n_tok = ksplit == 2 ? min(n_all, tok_lo + BM / 2) : n_all;
-        constexpr int NT = 4, NW = THREADS / 32;
-        for (int r0 = tok_lo + warp * NT; r0 < n_tok; r0 += NW * NT) {
-            int rows[NT];
-#pragma unroll
-            for (int a = 0; a < NT; ++a) rows[a] = min(r0 + a, n_tok - 1);
-            const int n_rows = min(NT, n_tok - r0);
-            const size_t out_row0 = (size_t)layer * T + t0;
-            if (E <= 128)
-                finish_tokens<IdxT, 4, NT>(tile, E + 1, rows, n_rows, lane, E, K, out_row0, idx_out,
-                                           logits_out, peer_tile);
-            else
-                finish_tokens<IdxT, 8, NT>(tile, E + 1, rows, n_rows, lane, E, K, out_row0, idx_out,
-                                           logits_out, peer_tile);
-        }
-    }
 
+    // ------------------------------ teardown ---------------------------------------------------
+    if (pair && threadIdx.x == 0)              // the peer has read the pushed rows out of this CTA
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         __syncthreads();
     }
-    if (ksplit == 2) cluster_sync_all();       // the other CTA may still be reading this tile
+    if (ksplit > 1) cluster_sync_all();        // no CTA leaves while a peer may still address it
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, tmem_cols);
@@ -286,6 +539,41 @@ size_t router_tc_workspace_bytes(const r3_shape* s, int L) {
     return round_up((size_t)L * 3 * s->E * s->d * sizeof(__nv_bfloat16), 256);
 }
 
+namespace rt {
+// Largest cluster size c <= want such that `units` clusters of c CTAs can all be resident at once
+// on the current device (a cluster lives inside one GPC, whose SM count need not be a multiple of
+// c: a B200 with 148 SMs holds 74 pairs but only 45 triples).  Cached per (device, c).
+template <typename Kern>
+static int usable_split(Kern kern, int want, long long units) {
+    static int max_clusters[64][MAX_SPLIT + 1] = {};        // 0 = not asked yet, -1 = failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    for (int c = want; c >= 2; --c) {
+        if (max_clusters[dev][c] == 0) {
+            cudaLaunchConfig_t cfg = {};
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)c;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.gridDim = dim3((unsigned)c * 64);
+            cfg.blockDim = dim3(THREADS);
+            cfg.dynamicSmemBytes = (size_t)SMEM_LIMIT;      // the most a CTA of this kernel asks for
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+                cudaGetLastError();
+                n = -1;
+            }
+            max_clusters[dev][c] = n;
+        }
+        if ((long long)max_clusters[dev][c] >= units) return c;
+    }
+    return 1;
+}
+}  // namespace rt
+
 r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* w_router,
                            void* idx_out, float* logits_out, void* workspace, cudaStream_t cs) {
     using namespace rt;
@@ -298,59 +586,80 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
             total);
         wplanes = workspace;
     }
-    const int stage_bytes = A_BYTES + planes * s->E * BK * 2;
-    const int tiles = (s->T + BM - 1) / BM;
+    // token tiles of a layer: as few as possible, of equal size (a multiple of 16); with two M
+    // tiles (E > 128) the logits of 256 tokens would not fit in shared memory
+    const int MT = (s->E + BME - 1) / BME;
+    const int n_max = MT == 1 ? 256 : 128;
+    const int tiles = (s->T + n_max - 1) / n_max;
+    const int N = (((s->T + tiles - 1) / tiles) + 15) & ~15;
     const int kblocks = (s->d + BK - 1) / BK;
-    // Few enough tiles that twice as many CTAs still get an SM each: two CTAs of a cluster share
-    // a tile (half of the k blocks and half of the tokens each).  With more tiles than that the
-    // shared form needs two CTAs per SM with half the ring each, which measured slower on the
-    // 48-layer decode batch (29.4 us against 24.7 us).
-    const int ksplit = ((long long)2 * tiles * L <= sm_count() && kblocks >= 2) ? 2 : 1;
-    int stages = (SMEM_LIMIT - BAR_BYTES - 1024) / stage_bytes;
-    if (stages > MAX_STAGES) stages = MAX_STAGES;
-    if (stages < 2) return R3_ERR_UNSUPPORTED;
-    const int tile_bytes = BM * (s->E + 1) * 4;        // the logits tile re-uses the ring
-    int ring = stages * stage_bytes;
-    if (ring < tile_bytes) ring = (tile_bytes + 1023) & ~1023;
-    if (ring + BAR_BYTES + 1024 > SMEM_LIMIT) return R3_ERR_UNSUPPORTED;
-    const int smem = ring + BAR_BYTES + 1024;
+    const int LD = MT * BME + 1;
+    const int stage_bytes = planes * MT * A_BYTES + N * BK * 2;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < s->E) tmem_cols <<= 1;
+    while ((int)tmem_cols < MT * N) tmem_cols <<= 1;
 
     CUtensorMap mx, mw;
-    if (!make_map_2d(&mx, x, (uint64_t)L * s->T, (uint64_t)s->d, BM) ||
-        !make_map_2d(&mw, wplanes, (uint64_t)L * planes * s->E, (uint64_t)s->d, (uint32_t)s->E))
+    if (!make_map_2d(&mx, x, (uint64_t)L * s->T, (uint64_t)s->d, (uint32_t)N) ||
+        !make_map_3d(&mw, wplanes, (uint64_t)L * planes, (uint64_t)s->E, (uint64_t)s->d, BME))
         return R3_ERR_CUDA;
+    const long long units = (long long)tiles * L;
+    // What a cluster of c CTAs keeps in the ring's place once the ring is free: per = tokens
+    // finished by one CTA (a multiple of 32).  c <= 2: the whole tile [c * per][LD] and, for
+    // c = 2, behind it the rows pushed by the peer [per][LD].  c > 2: the slots [c][per][LD].
+    auto per_of = [&](int c) { return (((N + c - 1) / c) + 31) & ~31; };
+    auto tile_of = [&](int c) { return (c * per_of(c) * LD * 4 + 127) & ~127; };
+    auto recv_of = [&](int c) { return c == 2 ? per_of(c) * LD * 4 : 0; };
+    const int fixed = BAR_BYTES + 1024;
+    auto fits = [&](int c) {
+        const int after = tile_of(c) + recv_of(c);
+        return (after > 2 * stage_bytes ? after : 2 * stage_bytes) + fixed <= SMEM_LIMIT;
+    };
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)ksplit;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.gridDim = dim3((unsigned)(tiles * ksplit), (unsigned)L);
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = cs;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-#define R3_RT(IDX, KM)                                                                          \
+    cfg.numAttrs = 2;
+#define R3_RT(IDX)                                                                              \
     do {                                                                                        \
-        auto kern = router_tc_kernel<IDX, KM>;                                                  \
-        static int attr_smem = 0;              /* largest size set so far, per instantiation */ \
-        if (smem > attr_smem) {                                                                 \
+        auto kern = router_tc_kernel<IDX>;                                                      \
+        static bool attr_set[64] = {};         /* per device */                                 \
+        int dev = 0;                                                                            \
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return R3_ERR_CUDA;     \
+        if (!attr_set[dev]) {                                                                   \
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
                                      SMEM_LIMIT) != cudaSuccess)                                \
                 return R3_ERR_CUDA;                                                             \
-            attr_smem = SMEM_LIMIT;                                                             \
+            attr_set[dev] = true;                                                               \
         }                                                                                       \
+        /* few tiles: the CTAs of a cluster share a tile's k blocks, as many as give every CTA  \
+           an SM of its own and at least two k blocks, and whose slots fit in shared memory */  \
+        int want = (int)(sm_count() / (units > 0 ? units : 1));                                 \
+        if (want > MAX_SPLIT) want = MAX_SPLIT;                                                 \
+        if (want > kblocks / 2) want = kblocks / 2;                                             \
+        while (want > 1 && !fits(want)) --want;                                                 \
+        int ksplit = want >= 2 ? usable_split(kern, want, units) : 1;                           \
+        while (ksplit > 1 && !fits(ksplit)) --ksplit;                                           \
+        if (!fits(ksplit)) return R3_ERR_UNSUPPORTED;                                           \
+        int stages = (SMEM_LIMIT - fixed) / stage_bytes;                                        \
+        if (stages > MAX_STAGES) stages = MAX_STAGES;                                           \
+        int ring = stages * stage_bytes;                                                        \
+        const int after = tile_of(ksplit) + recv_of(ksplit);                                    \
+        if (ring < after) ring = (after + 127) & ~127;                                          \
+        attr[0].val.clusterDim.x = (unsigned)ksplit;                                            \
+        cfg.gridDim = dim3((unsigned)(tiles * ksplit), (unsigned)L);                            \
+        cfg.dynamicSmemBytes = (size_t)(ring + fixed);                                          \
         if (cudaLaunchKernelEx(&cfg, kern, mx, mw, static_cast<IDX*>(idx_out), logits_out,      \
                                (int)s->T, (int)s->d, (int)s->E, (int)s->K, planes, stages,      \
-                               tmem_cols, ksplit) != cudaSuccess)                               \
+                               tmem_cols, ksplit, N, MT, ring, tile_of(ksplit)) != cudaSuccess) \
             return R3_ERR_CUDA;                                                                 \
     } while (0)
-    const bool u8 = s->idx_type == R3_IDX_U8;
-    if (s->K <= 8) { if (u8) R3_RT(uint8_t, 8); else R3_RT(int16_t, 8); }
-    else { if (u8) R3_RT(uint8_t, 16); else R3_RT(int16_t, 16); }
+    if (s->idx_type == R3_IDX_U8) R3_RT(uint8_t); else R3_RT(int16_t);
 #undef R3_RT
     return launch_status();
 }

@@ -103,6 +103,18 @@ __device__ __forceinline__ void tc_wait_ld() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Programmatic dependent launch.  A kernel launched with programmatic stream serialisation may
+// start while its predecessor in the stream is still running; grid_dependency_wait() returns once
+// the predecessor has completed and its memory is visible (every access to global memory comes
+// after it), grid_launch_dependents() lets the successor start its own prologue.  Both are no-ops
+// for a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- two-CTA (cta_group::2) forms ---------------------------------------------------------------
 // A CTA pair (the two CTAs of a 2x1x1 cluster) issues one MMA of M = 256: each CTA supplies its own
 // 128 rows of A and its own half of the N columns of B from the SAME shared-memory offsets, and

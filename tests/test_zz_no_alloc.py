@@ -46,10 +46,11 @@ def test_permute_static_matches_permute_on_two_calls_in_a_row():
         out = empty_outputs(T, E, K, d)
         st = r3.new_status("cuda")
         torch.cuda.synchronize()
-        held = torch.cuda.memory_allocated()
+        requests = torch.cuda.memory_stats()["allocation.all.allocated"]
         got = r3.permute_static(s, idx, x, *out, dev_status=st)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == held      # the caller's allocator saw nothing
+        # the caller's allocator was asked for nothing during the call
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == requests
         assert st.item() == 0
         for a, b in zip(got, want):
             assert torch.equal(a, b)              # integer maps and copied rows: bit-exact
