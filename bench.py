@@ -649,18 +649,18 @@ def measure_capture(torch, r3, synth, w, args, peaks, sampler, dev):
     (r3_capture_topk_batched), records packed as uint8; inputs rotate over more than L2."""
     L, T, d, E, K = w.layers, w.T, w.d, w.E, w.K
     s = r3.shape_of(w)
-    reps = 8                                  # rotate over > L2-sized input rings
+    reps = 8                                  # rotate over > L2-sized rings: activations AND weights
     xs = [torch.stack([synth.activations(w, dev, l + 100 * r) for l in range(L)]) for r in range(reps)]
-    wr = torch.stack([synth.router_weight(w, dev, l) for l in range(L)])
+    wrs = [torch.stack([synth.router_weight(w, dev, l + 100 * r) for l in range(L)]) for r in range(reps)]
     idx = torch.empty((L, T, K), dtype=w.idx_dtype, device=dev)
     one_idx = torch.empty((T, K), dtype=w.idx_dtype, device=dev)
     steps, warmup = max(args.steps, 20), max(args.warmup, 3)
 
     def batched(i):
-        r3.capture_topk_batched(s, L, xs[i % reps], wr, idx_out=idx)
+        r3.capture_topk_batched(s, L, xs[i % reps], wrs[i % reps], idx_out=idx)
 
     def one(i):
-        r3.capture_topk(s, xs[i % reps][i % L], wr[i % L], idx_out=one_idx)
+        r3.capture_topk(s, xs[i % reps][i % L], wrs[i % reps][i % L], idx_out=one_idx)
 
     for i in range(warmup):
         batched(i)
@@ -691,7 +691,8 @@ def measure_capture(torch, r3, synth, w, args, peaks, sampler, dev):
         "value": L * T / (ms_b * 1e-3), "unit": "layer-tokens/s", "steps": steps, "warmup": warmup,
         "ms_per_step": ms_b, "dtype": "bf16",
         "config": {"workload": w.name, "layers": L, "T": T, "d": d, "E": E, "K": K,
-                   "l2": f"inputs rotate over {reps} sets of {L * T * d * 2 / 1e6:.0f} MB (> L2 in all)"},
+                   "l2": f"activations and router weights rotate over {reps} sets of "
+                         f"{L * (T + E) * d * 2 / 1e6:.0f} MB (> L2 in all)"},
         "roofline": {"bound": "hbm", "kernel": "router_tc_kernel (48 layers in one launch)",
                      "achieved": round(bytes_b / ms_b / 1e6, 1), "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": round(bytes_b / ms_b / 1e6 / peaks["hbm_gbs"], 4),

@@ -33,13 +33,14 @@
 // One CTA of 12 warps per (tile, k range): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA
 // issuer; then all 12 warps move the finished accumulator out of TMEM (transposed on the way:
 // tensor-memory lane = expert, but a token's experts must lie next to each other), and TopKMask
-// is taken by FOUR lanes per token on packed candidates in registers (thread_topk below), with a
-// warp-wide exact selection for the few tokens that the packed form cannot decide.  The earlier
-// form, K rounds of two warp reductions per token, cost 9.6 us for the 128 tokens of a CTA.
+// is taken by two or four lanes per token on packed candidates in registers (group_topk below), with a
+// warp-wide exact selection for the few tokens that the packed form cannot decide.
 //
 // The kernel is launched with programmatic stream serialisation: everything up to its first
 // access to global memory (barrier set-up, tensor-memory allocation) may run while the previous
 // kernel of the stream drains, and it lets its own successor do the same once its copies are done.
+#include <type_traits>
+
 #include "r3_common.cuh"
 #include "r3_internal.h"
 #include "r3_tc.cuh"
@@ -59,7 +60,6 @@ constexpr int MAX_STAGES = 7;
 constexpr int KMAX = 16;                 // longest record the warp top-K supports (one lane per slot)
 constexpr int SMEM_LIMIT = 227 * 1024;
 constexpr int MAX_SPLIT = 8;             // portable cluster size
-constexpr int GROUP = 4;                 // lanes that share a token in the TopKMask
 
 __global__ void __launch_bounds__(256)
 split_router_weight_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ planes,
@@ -230,15 +230,20 @@ struct TopList {
     }
 };
 
-// TopKMask of the tokens of one warp task: GROUP lanes share a token (lane = GROUP * token +
-// part); each takes every GROUP-th block of KM experts, sorts the block with a sorting network
+// TopKMask of the tokens of one warp task: GROUP (2 or 4) lanes share a token (lane = GROUP *
+// token + part); each takes every GROUP-th block of KM experts, sorts the block with a sorting network
 // and merges it into its list; the GROUP lists of a token are then merged through shuffles.  The
 // result is exact unless two candidates next to each other in the final order (down to the first
 // one left out) share their 24 leading bits while the full logits might differ; such a token is
 // flagged and repeated with warp_topk_exact (random logits: a few tokens in a thousand; planted
 // exact ties: every such token, still correct).  Returns the flags of the warp's tokens (bit =
 // lane of the token's first lane).
-template <typename IdxT, int KM>
+// Measured for the 128 tokens that a CTA of the 48-layer decode batch finishes: K rounds of two
+// warp reductions per token 9.6 us; one reduction per round on packed candidates 6.3 us (a warp
+// reduction costs this SM about ten cycles whoever issues it); this form 4.2 us with four lanes
+// per token (16 warp tasks for 12 warps) and 3.3 us with two (8 tasks): about 1400 fminf / fmaxf
+// per token, which issue at half rate.  With few tokens per CTA four lanes are faster.
+template <typename IdxT, int KM, int GROUP>
 __device__ __forceinline__ uint32_t group_topk(const Partials& ps, int LD, int row, bool valid,
                                                int part, int E, int K, IdxT* out) {
     TopList<KM> list;
@@ -491,24 +496,29 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
     }
     if (!*abort_flag && idx_out) {
-        // TopKMask: GROUP lanes per token, 32 / GROUP tokens per warp task
-        constexpr int TPW = 32 / GROUP;
-        for (int task = warp; task * TPW < n_mine; task += THREADS / 32) {
-            const int row = task * TPW + (lane / GROUP);
-            const bool valid = row < n_mine;
-            IdxT* out = idx_out + (out_row0 + (valid ? row : 0)) * K;
-            uint32_t redo = K <= 8
-                ? group_topk<IdxT, 8>(ps, LD, row, valid, lane % GROUP, E, K, out)
-                : group_topk<IdxT, 16>(ps, LD, row, valid, lane % GROUP, E, K, out);
-            while (redo) {
-                const int r2 = task * TPW + (__ffs(redo) - 1) / GROUP;
-                redo &= redo - 1;
-                if (E <= 128)
-                    warp_topk_exact<IdxT, 4>(ps, LD, r2, lane, E, K, idx_out + (out_row0 + r2) * K);
-                else
-                    warp_topk_exact<IdxT, 8>(ps, LD, r2, lane, E, K, idx_out + (out_row0 + r2) * K);
+        // TopKMask: two lanes per token (16 tokens per warp task), four when the tokens are few
+        auto select = [&](auto group_tag) {
+            constexpr int GROUP = decltype(group_tag)::value;
+            constexpr int TPW = 32 / GROUP;
+            for (int task = warp; task * TPW < n_mine; task += THREADS / 32) {
+                const int row = task * TPW + (lane / GROUP);
+                const bool valid = row < n_mine;
+                IdxT* out = idx_out + (out_row0 + (valid ? row : 0)) * K;
+                uint32_t redo = K <= 8
+                    ? group_topk<IdxT, 8, GROUP>(ps, LD, row, valid, lane % GROUP, E, K, out)
+                    : group_topk<IdxT, 16, GROUP>(ps, LD, row, valid, lane % GROUP, E, K, out);
+                while (redo) {
+                    const int r2 = task * TPW + (__ffs(redo) - 1) / GROUP;
+                    redo &= redo - 1;
+                    if (E <= 128)
+                        warp_topk_exact<IdxT, 4>(ps, LD, r2, lane, E, K, idx_out + (out_row0 + r2) * K);
+                    else
+                        warp_topk_exact<IdxT, 8>(ps, LD, r2, lane, E, K, idx_out + (out_row0 + r2) * K);
+                }
             }
-        }
+        };
+        if (n_mine > 6 * (THREADS / 32)) select(std::integral_constant<int, 2>{});
+        else select(std::integral_constant<int, 4>{});
     }
 
     // ------------------------------ teardown ---------------------------------------------------
