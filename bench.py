@@ -1150,6 +1150,9 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=4096,
                     help="tokens of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tokens", type=int, default=None,
+                    help="with --workload: the same layer on this many tokens (profiling captures "
+                         "on a case of a few GB); the line then names the workload 'name@T'")
     ap.add_argument("--stack", action="store_true", help="kept for old command lines: a multi-layer "
                     "workload is always timed over all its blocks")
     ap.add_argument("--ep", action="store_true",
@@ -1167,6 +1170,8 @@ def main():
         return run_diag(args)
     name = HEADLINE if args.workload == "all" else args.workload
     w = synth.WORKLOADS[name]
+    if args.tokens:
+        w = synth.WORKLOADS[name] = synth.scaled(w, name=f"{name}@{args.tokens}", T=args.tokens)
     if args.impl == "reference":
         return run_reference(args, w)
     if args.ep or args.ep_direct:

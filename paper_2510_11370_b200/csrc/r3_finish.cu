@@ -236,6 +236,8 @@ replay_finish_staged_kernel(const float* __restrict__ logits, const IdxT* __rest
 
     int my_e = -1;
     float g = 0.f;
+    tc::grid_launch_dependents();
+    tc::grid_dependency_wait();            // everything this kernel reads may come from the one before
     if (warp == 0) {
         // ---- the token's record and row numbers first (independent loads), then the logit of
         // each recorded expert, so that only two memory latencies precede the copies ------------
@@ -437,10 +439,12 @@ static r3_status launch_finish(const r3_shape* s, const float* logits, const voi
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
             attr_set = true;
         }
-        kern<<<T, kTokThreads, smem, cs>>>(
-            logits, static_cast<const IdxT*>(idx), nullptr, nullptr, row_ptr,
-            static_cast<const ActT*>(dy), static_cast<const ActT*>(residual), static_cast<ActT*>(y),
-            gates_out, dlogits, E, K, d, W, dev_status);
+        if (tc::launch_dependent(kern, dim3(T), dim3(kTokThreads), smem, cs, logits,
+                                 static_cast<const IdxT*>(idx), nullptr, nullptr, row_ptr,
+                                 static_cast<const ActT*>(dy), static_cast<const ActT*>(residual),
+                                 static_cast<ActT*>(y), gates_out, dlogits, E, K, d, W,
+                                 dev_status) != cudaSuccess)
+            return R3_ERR_CUDA;
         return R3_OK;
     }
     if (row_ptr) return R3_ERR_UNSUPPORTED;    // rows by address need the staged kernel
@@ -451,10 +455,12 @@ static r3_status launch_finish(const r3_shape* s, const float* logits, const voi
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
             attr_set = true;
         }
-        kern<<<T, kTokThreads, smem, cs>>>(
-            logits, static_cast<const IdxT*>(idx), static_cast<const ActT*>(o), row_of_slot, nullptr,
-            static_cast<const ActT*>(dy), static_cast<const ActT*>(residual), static_cast<ActT*>(y),
-            gates_out, dlogits, E, K, d, W, dev_status);
+        if (tc::launch_dependent(kern, dim3(T), dim3(kTokThreads), smem, cs, logits,
+                                 static_cast<const IdxT*>(idx), static_cast<const ActT*>(o),
+                                 row_of_slot, nullptr, static_cast<const ActT*>(dy),
+                                 static_cast<const ActT*>(residual), static_cast<ActT*>(y),
+                                 gates_out, dlogits, E, K, d, W, dev_status) != cudaSuccess)
+            return R3_ERR_CUDA;
         return R3_OK;
     }
     const int tpt = pick_team_fused(d / Vec16<ActT>::N);

@@ -314,6 +314,8 @@ permute_maps_cluster_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ 
     for (int e = lt; e < E; e += kChunk) hist[e] = 0;
     for (int i = lt; i < E * kWords; i += kChunk) bits[i] = 0u;
     __syncthreads();
+    tc::grid_launch_dependents();
+    tc::grid_dependency_wait();                    // the record may come from the kernel before
     int kept[8];                                   // slots 0..7: the expert, or -1 for a dropped pair
 #pragma unroll
     for (int u = 0; u < 8; ++u) kept[u] = -1;
@@ -476,6 +478,8 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
         tc::mbar_expect_tx(bar, row_bytes * (uint32_t)nt);
     }
     __syncwarp();
+    tc::grid_launch_dependents();
+    tc::grid_dependency_wait();            // x and the maps may come from the kernel before
     if (lane < nt)
         asm volatile(
             "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -522,9 +526,10 @@ r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, 128 + 96 * 1024);
             attr_set = true;
         }
-        permute_rows_staged_kernel<<<(T + kRowTokens - 1) / kRowTokens, 32, smem, cs>>>(
-            static_cast<const uint8_t*>(x), row_of_slot, static_cast<uint8_t*>(xp), T, K,
-            (uint32_t)row_bytes);
+        if (tc::launch_dependent(permute_rows_staged_kernel, dim3((T + kRowTokens - 1) / kRowTokens),
+                                 dim3(32), smem, cs, static_cast<const uint8_t*>(x), row_of_slot,
+                                 static_cast<uint8_t*>(xp), T, K, (uint32_t)row_bytes) != cudaSuccess)
+            return R3_ERR_CUDA;
         return launch_status();
     }
     const int row_vecs = (int)(row_bytes / 16);
@@ -579,17 +584,19 @@ r3_status r3::permute_impl(const r3_shape* shape, const void* idx, const void* x
         static int usable[2][r3::kClusterMax + 1] = {};        // per index type and cluster size
         const int ti = shape->idx_type == R3_IDX_U8 ? 0 : 1;   // 0 = untested, 1 = ok, -1 = no
         cudaLaunchConfig_t cfg = {};
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)cl;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.gridDim = dim3((unsigned)cl);
         cfg.blockDim = dim3(r3::kChunk);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = cs;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         if (usable[ti][cl] == 0) {
             usable[ti][cl] = -1;
             if (smem <= 200 * 1024) {

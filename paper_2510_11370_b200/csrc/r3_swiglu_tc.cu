@@ -84,6 +84,8 @@ __global__ void __launch_bounds__(1024)
 build_work_kernel(const int32_t* __restrict__ offsets, int E, int nf0, int nf1,
                   int32_t* __restrict__ list0, int32_t* __restrict__ list1, int pairs) {
     __shared__ int32_t s_items[1025];
+    grid_launch_dependents();
+    grid_dependency_wait();                // the offsets come from the dispatch before
     build_work_list(offsets, E, blockIdx.x == 0 ? nf0 : nf1, blockIdx.x == 0 ? list0 : list1, pairs,
                     s_items);
 }
@@ -179,7 +181,6 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
     const uint32_t rank = cluster_ctarank();          // 0 = leader of the CTA pair
     const int pair = blockIdx.x >> 1;
     const int w_step = gridDim.x >> 1;
-    const int w_begin = pair, w_end = list[0];
     const int4* __restrict__ items = reinterpret_cast<const int4*>(list + kHeaderInts);
     const int4 kNone = make_int4(0, 0, 0, 0);          // n = 0 ends the item stream
     // MODE 3 walks the k blocks of both weight matrices alternately
@@ -201,6 +202,11 @@ grouped_gemm_pair_kernel(const __grid_constant__ PairMaps maps, int32_t* list,
     cluster_sync_all();            // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Nothing above touched global memory: it may have run while the kernel before this one in
+    // the stream was draining.  The work list, the operands and the outputs come after the wait.
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int w_begin = pair, w_end = list[0];
 
     if (warp == 0 && GATHER) {
         // ------------------------------ TMA producer, gather form (the whole warp) -------------
@@ -639,17 +645,19 @@ static r3_status launch_pair(const PairMaps& maps, int pairs, int32_t* list,
                              int32_t* dev_status, cudaStream_t cs, void* pre_gate = nullptr,
                              void* pre_up = nullptr) {
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.gridDim = dim3(2 * pairs);
     cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = cs;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<MODE, GATHER>, maps, list, slot_of_row, K,
                               static_cast<__nv_bfloat16*>(out), static_cast<__nv_bfloat16*>(pre_gate),
                               static_cast<__nv_bfloat16*>(pre_up), Kdim, Nout,
@@ -752,7 +760,8 @@ r3_status launch_grouped_swiglu_tc(const r3_shape* s, const void* xp, const void
     static TokenMapCache cache_xp, cache_h;
     if (phases & kPhaseUp) {
         if (!(phases & kPhaseKeepLists))
-            build_work_kernel<<<2, 1024, 0, cs>>>(offsets, s->E, nf0, nf1, list0, list1, pairs);
+            launch_dependent(build_work_kernel, dim3(2), dim3(1024), 0, cs, offsets, (int)s->E, nf0,
+                             nf1, list0, list1, pairs);
         PairMaps m;
         if (!make_map_3d(&m.a0, w_gate, s->E, s->F, s->d, BMF / 2) ||
             !make_map_3d(&m.a1, w_up, s->E, s->F, s->d, BMF / 2))

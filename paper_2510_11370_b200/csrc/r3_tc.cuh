@@ -115,6 +115,24 @@ __device__ __forceinline__ void grid_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Launches `kern` on `cs` with programmatic stream serialisation (see above): for kernels that
+// call grid_dependency_wait() before their first access to global memory.
+template <typename... Params, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(Params...), dim3 grid, dim3 block, size_t smem,
+                                    cudaStream_t cs, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = cs;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<Params>(args)...);
+}
+
 // ---- two-CTA (cta_group::2) forms ---------------------------------------------------------------
 // A CTA pair (the two CTAs of a 2x1x1 cluster) issues one MMA of M = 256: each CTA supplies its own
 // 128 rows of A and its own half of the N columns of B from the SAME shared-memory offsets, and
