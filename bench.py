@@ -382,9 +382,9 @@ def measure_layer(torch, r3, r3dist, inp, args, peaks, sampler, world=1, dev=Non
            "clocks": sampler.window(t_wall0, t_wall1) if sampler else None}
 
     # ---- the same step for at least SUSTAINED_SECONDS (power-capped clocks) ---------------------
-    sus = sustained_region(torch, sampler, step, ms_per_step, T)
+    if not args.no_sustained:
+        rec["sustained"] = sustained_region(torch, sampler, step, ms_per_step, T)
     assert st.item() == 0
-    rec["sustained"] = sus
     if not detail:
         return rec
 
@@ -670,7 +670,7 @@ def measure_capture(torch, r3, synth, w, args, peaks, sampler, dev):
     ms_b = event_time(torch, batched, steps)
     t1 = time.time()
     ms_1 = event_time(torch, one, steps)
-    n_sus = int(math.ceil(SUSTAINED_SECONDS * 1e3 / ms_b))
+    n_sus = 3 if args.no_sustained else int(math.ceil(SUSTAINED_SECONDS * 1e3 / ms_b))
     ts0 = time.time()
     ms_sus = event_time(torch, batched, n_sus)
     ts1 = time.time()
@@ -1150,6 +1150,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=4096,
                     help="tokens of the workload the CPU oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true",
+                    help="skip the regions of at least 0.6 s (for runs under a profiler)")
     ap.add_argument("--tokens", type=int, default=None,
                     help="with --workload: the same layer on this many tokens (profiling captures "
                          "on a case of a few GB); the line then names the workload 'name@T'")
