@@ -41,7 +41,8 @@ NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel, from the ncu captures
 # summarised under profiles/ (a constant taken from the profile, not re-measured by a run)
-GEMM_UP_DRAM_TRAFFIC_BYTES = {"c2_layer_bf16": 988.8e6}
+GEMM_UP_DRAM_TRAFFIC_BYTES = {"c2_layer_bf16": 988.8e6,     # 940.8 MB read + 48.0 MB written
+                              "c4_replay": 3.742e9}         # 2.95 GB read + 791.8 MB written
 
 
 def launches_per_step(w) -> int:

@@ -203,7 +203,11 @@ r3_status r3_expert_down(const r3_shape* shape, const void* w_down, void* o, voi
                          size_t ws_bytes, int32_t* dev_status, void* stream);
 
 /* Eq. (replay_output): y[t] = sum_{j=0..K-1} gates[t,j] * o[row_of_slot[t,j]], added in slot
- * order in fp32 (no atomics), rounded once to act_dtype.  o [R,d]; y [T,d]. */
+ * order in fp32 (no atomics), rounded once to act_dtype.  o [R,d]; y [T,d].
+ * r3_combine, r3_combine_residual and r3_combine_bwd_gates take no dev_status word: should one of
+ * their internal bounded waits ever run out, the affected token's output is left unwritten without
+ * a report.  r3_replay_finish (what the layer runs) computes the same values and reports
+ * R3_DEV_TIMEOUT. */
 r3_status r3_combine(const r3_shape* shape, const void* o, const int32_t* row_of_slot,
                      const float* gates, void* y, void* stream);
 

@@ -280,10 +280,14 @@ static bool launch_staged(const r3_shape* s, const void* o, const int32_t* row_o
     const size_t smem = kStageHeader + (size_t)rows * s->d * sizeof(ActT);
     if (smem > (size_t)kStageSmemLimit) return false;
     auto kern = gather_staged_kernel<ActT, DO_Y, DO_DG>;
-    static bool attr_set = false;              // one flag per instantiation
-    if (!attr_set) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kStageSmemLimit);
-        attr_set = true;
+    static PerDevice attr_set;                 // one set of flags per instantiation
+    if (!attr_set.done()) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kStageSmemLimit) != cudaSuccess) {
+            cudaGetLastError();
+            return false;                      // the register kernel takes over
+        }
+        attr_set.mark();
     }
     kern<<<s->T, kStageThreads, smem, cs>>>(
         static_cast<const ActT*>(o), row_of_slot, gates, static_cast<const ActT*>(residual),

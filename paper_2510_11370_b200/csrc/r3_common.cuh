@@ -32,6 +32,19 @@ inline r3_status check_shape(const r3_shape* s) {
     return R3_OK;
 }
 
+// Per-device "already done" flags for host-side set-up that CUDA keeps per device (function
+// attributes, occupancy answers): a process that drives several devices repeats the set-up on
+// each of them.  done() is false until mark() has been called with the same device current.
+struct PerDevice {
+    bool flag[64] = {};
+    static int current() {
+        int dev = 0;
+        return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) ? dev : 0;
+    }
+    bool done() const { return flag[current()]; }
+    void mark() { flag[current()] = true; }
+};
+
 inline r3_status launch_status() {
     return cudaGetLastError() == cudaSuccess ? R3_OK : R3_ERR_CUDA;
 }

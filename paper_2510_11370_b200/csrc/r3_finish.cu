@@ -434,10 +434,12 @@ static r3_status launch_finish(const r3_shape* s, const float* logits, const voi
     const size_t smem = kTokHeader + 128 + (size_t)(K + 1 + (residual ? 1 : 0)) * d * sizeof(ActT);
     if (smem <= (size_t)kTokSmemLimit / 2 && row_ptr) {
         auto kern = replay_finish_staged_kernel<ActT, IdxT, true>;
-        static bool attr_set = false;          // one flag per instantiation
-        if (!attr_set) {
-            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
-            attr_set = true;
+        static PerDevice attr_set;             // one set of flags per instantiation
+        if (!attr_set.done()) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kTokSmemLimit / 2) != cudaSuccess)
+                return R3_ERR_CUDA;
+            attr_set.mark();
         }
         if (tc::launch_dependent(kern, dim3(T), dim3(kTokThreads), smem, cs, logits,
                                  static_cast<const IdxT*>(idx), nullptr, nullptr, row_ptr,
@@ -450,10 +452,12 @@ static r3_status launch_finish(const r3_shape* s, const float* logits, const voi
     if (row_ptr) return R3_ERR_UNSUPPORTED;    // rows by address need the staged kernel
     if (smem <= (size_t)kTokSmemLimit / 2) {
         auto kern = replay_finish_staged_kernel<ActT, IdxT, false>;
-        static bool attr_set = false;          // one flag per instantiation
-        if (!attr_set) {
-            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kTokSmemLimit / 2);
-            attr_set = true;
+        static PerDevice attr_set;             // one set of flags per instantiation
+        if (!attr_set.done()) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kTokSmemLimit / 2) != cudaSuccess)
+                return R3_ERR_CUDA;
+            attr_set.mark();
         }
         if (tc::launch_dependent(kern, dim3(T), dim3(kTokThreads), smem, cs, logits,
                                  static_cast<const IdxT*>(idx), static_cast<const ActT*>(o),

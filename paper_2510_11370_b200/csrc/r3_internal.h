@@ -96,7 +96,7 @@ r3_status grouped_swiglu_keep_lists(const r3_shape* shape, const void* xp, const
 
 // The row copy of the dispatch alone: xp[row_of_slot[t, j]] = x[t] (maps from an earlier r3_permute).
 r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_t* row_of_slot,
-                              void* xp, cudaStream_t stream);
+                              void* xp, cudaStream_t stream, int32_t* dev_status);
 
 // Number of SMs of the current device (cached).
 int sm_count();

@@ -130,7 +130,7 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
     if (same_record) {
         // the maps and the GEMM work lists of the previous call on this workspace still hold:
         // only the rows are copied again
-        if ((st = launch_permute_rows(shape, x, w.row_of_slot, w.xp, cs)) != R3_OK) return st;
+        if ((st = launch_permute_rows(shape, x, w.row_of_slot, w.xp, cs, dev_status)) != R3_OK) return st;
         st = grouped_swiglu_keep_lists(shape, w.xp, w.offsets, w_gate, w_up, w_down, w.o, pre_gate,
                                        pre_up, w.swiglu_ws, w.swiglu_bytes, dev_status, stream);
     } else {

@@ -463,7 +463,8 @@ constexpr int kRowTokens = 8;
 
 __global__ void __launch_bounds__(32)
 permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_slot,
-                           uint8_t* __restrict__ xp, int T, int K, uint32_t row_bytes) {
+                           uint8_t* __restrict__ xp, int T, int K, uint32_t row_bytes,
+                           int32_t* dev_status) {
     extern __shared__ __align__(128) uint8_t smem_p[];
     const uint32_t bar = tc::smem_u32(smem_p);
     volatile int* flags = reinterpret_cast<volatile int*>(smem_p + 8);
@@ -490,7 +491,8 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
     const int32_t* rows = row_of_slot + (size_t)(t0 + (lane < nt ? lane : 0)) * K;
 #pragma unroll
     for (int u = 0; u < 8; ++u) r[u] = (lane < nt && u < K) ? rows[u] : -1;
-    const bool ok = __all_sync(0xffffffffu, tc::mbar_wait(bar, 0u, flags, nullptr));
+    // a wait that runs out leaves these tokens' rows unwritten and says so in dev_status
+    const bool ok = __all_sync(0xffffffffu, tc::mbar_wait(bar, 0u, flags, dev_status));
     if (ok && lane < nt) {
         for (int j0 = 0; j0 < K; j0 += 8) {
             if (j0 > 0) {
@@ -515,20 +517,23 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
 }
 
 r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_t* row_of_slot,
-                              void* xp, cudaStream_t cs) {
+                              void* xp, cudaStream_t cs, int32_t* dev_status) {
     const int T = shape->T, K = shape->K;
     const size_t row_bytes = (size_t)shape->d * act_bytes(shape);
     if (row_bytes * kRowTokens <= 96 * 1024) {
         const size_t smem = 128 + row_bytes * kRowTokens;
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaFuncSetAttribute(permute_rows_staged_kernel,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, 128 + 96 * 1024);
-            attr_set = true;
+        static PerDevice attr_set;
+        if (!attr_set.done()) {
+            if (cudaFuncSetAttribute(permute_rows_staged_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     128 + 96 * 1024) != cudaSuccess)
+                return R3_ERR_CUDA;
+            attr_set.mark();
         }
         if (tc::launch_dependent(permute_rows_staged_kernel, dim3((T + kRowTokens - 1) / kRowTokens),
                                  dim3(32), smem, cs, static_cast<const uint8_t*>(x), row_of_slot,
-                                 static_cast<uint8_t*>(xp), T, K, (uint32_t)row_bytes) != cudaSuccess)
+                                 static_cast<uint8_t*>(xp), T, K, (uint32_t)row_bytes,
+                                 dev_status) != cudaSuccess)
             return R3_ERR_CUDA;
         return launch_status();
     }
@@ -581,8 +586,10 @@ r3_status r3::permute_impl(const r3_shape* shape, const void* idx, const void* x
         int cl = 1;
         while (cl < NB) cl <<= 1;
         const size_t smem = ((size_t)E * (5 + r3::kWords) + 2) * sizeof(int32_t);
-        static int usable[2][r3::kClusterMax + 1] = {};        // per index type and cluster size
-        const int ti = shape->idx_type == R3_IDX_U8 ? 0 : 1;   // 0 = untested, 1 = ok, -1 = no
+        // per device, index type and cluster size: 0 = untested, 1 = ok, -1 = no
+        static int usable_dev[64][2][r3::kClusterMax + 1] = {};
+        int (*usable)[r3::kClusterMax + 1] = usable_dev[r3::PerDevice::current()];
+        const int ti = shape->idx_type == R3_IDX_U8 ? 0 : 1;
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -659,7 +666,7 @@ r3_status r3::permute_impl(const r3_shape* shape, const void* idx, const void* x
             static_cast<const IdxT*>(idx), chunk_counts, offsets, row_of_slot, slot_of_row,
             T, E, K, NB));
     }
-    if (x) return r3::launch_permute_rows(shape, x, row_of_slot, xp, cs);
+    if (x) return r3::launch_permute_rows(shape, x, row_of_slot, xp, cs, dev_status);
     return r3::launch_status();
 }
 

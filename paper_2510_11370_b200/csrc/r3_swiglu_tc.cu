@@ -714,8 +714,8 @@ size_t tc_work_bytes(const r3_shape* s) {
 
 static bool forward_attrs() {
     using namespace tc;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDevice attr_set;
+    if (!attr_set.done()) {
         if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<0, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(grouped_gemm_pair_kernel<0, true>,
@@ -723,7 +723,7 @@ static bool forward_attrs() {
             cudaFuncSetAttribute(grouped_gemm_pair_kernel<1, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return false;
-        attr_set = true;
+        attr_set.mark();
     }
     return true;
 }
@@ -811,14 +811,14 @@ r3_status launch_grouped_swiglu_bwd_tc(const r3_shape* s, const void* dout, cons
     using namespace tc;
     const long long R = (long long)s->T * s->K;
     if (R == 0) return R3_OK;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDevice attr_set;
+    if (!attr_set.done()) {
         if (cudaFuncSetAttribute(grouped_gemm_pair_kernel<2, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(grouped_gemm_pair_kernel<3, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
             return R3_ERR_CUDA;
-        attr_set = true;
+        attr_set.mark();
     }
     const int pairs = resident_pairs(grouped_gemm_pair_kernel<2, false>);
     if (pairs <= 0) return R3_ERR_CUDA;

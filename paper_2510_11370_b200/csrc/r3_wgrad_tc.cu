@@ -280,12 +280,12 @@ r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, c
     using namespace wg;
     const uint64_t R = (uint64_t)s->T * s->K;
     if (R == 0) return R3_OK;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDevice attr_set;
+    if (!attr_set.done()) {
         if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SMEM_BYTES) != cudaSuccess)
             return R3_ERR_CUDA;
-        attr_set = true;
+        attr_set.mark();
     }
     Params P;
     const void* a_ptr[3] = {dout, da, db};
