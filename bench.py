@@ -382,11 +382,9 @@ def measure_layer(torch, r3, r3dist, inp, args, peaks, sampler, world=1, dev=Non
            "config": layer_config(wk), "gpu_launches": launches_per_step(wk) * steps,
            "clocks": sampler.window(t_wall0, t_wall1) if sampler else None}
 
-    # ---- the same step for at least SUSTAINED_SECONDS (power-capped clocks) ---------------------
-    if not args.no_sustained:
-        rec["sustained"] = sustained_region(torch, sampler, step, ms_per_step, T)
-    assert st.item() == 0
     if not detail:
+        if not args.no_sustained:
+            rec["sustained"] = sustained_region(torch, sampler, step, ms_per_step, T)
         return rec
 
     # ---- the same step timed one by one: best and median ---------------------------------------
@@ -557,6 +555,12 @@ def measure_layer(torch, r3, r3dist, inp, args, peaks, sampler, world=1, dev=Non
                            "peak_kind": "fp32 FMA: 148 SMs x 128 lanes x 2 x max SM clock",
                            "traffic": None}
     del o, pout, logits
+    # ---- the same step for at least SUSTAINED_SECONDS (power-capped clocks).  It comes after the
+    # per-kernel timings, so that those, like the K timed steps, are taken before the long region
+    # has driven the GPU into its power cap (their peak is the burst figure) ----------------------
+    if not args.no_sustained:
+        rec["sustained"] = sustained_region(torch, sampler, step, ms_per_step, T)
+    assert st.item() == 0
     if not e2e:
         return rec
 

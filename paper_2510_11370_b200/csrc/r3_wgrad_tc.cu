@@ -3,9 +3,16 @@
 //   dW_down[e] [d,F] = dout_e^T h_e      dW_gate[e] [F,d] = da_e^T xp_e      dW_up[e] [F,d] = db_e^T xp_e
 // Every product contracts over the expert's token rows, so both operands are read "MN-major": a
 // TMA box of 64 consecutive columns x 64 token rows lands as 64 swizzled 128-byte rows, and the
-// tcgen05 descriptors walk the rows as the k dimension.  One CTA per SM (cta_group::1), tiles of
-// 128 x 256 outputs, float32 accumulators in tensor memory (two stages, so a tile's epilogue runs
-// under the next tile's MMAs), items (expert, problem, m tile, n tile) dealt round-robin.
+// tcgen05 descriptors walk the rows as the k dimension.  One CTA per SM (cta_group::1), float32
+// accumulators in tensor memory, items (expert, problem, m tile, n tile) dealt round-robin.  Two
+// tile shapes:
+//   MT = 1: 128 x 256 outputs, two accumulator stages (a tile's epilogue runs under the next tile's
+//           MMAs), 4 ring stages of 48 KB.  For few rows per expert, where the float32 result
+//           written to HBM is the bound and the epilogue must never wait.
+//   MT = 2: 256 x 256 outputs as two 128-row MMAs that share the B boxes, one accumulator stage
+//           (all 512 columns), 3 ring stages of 64 KB.  For many rows per expert, where the bound
+//           is the operand bytes each SM can draw from L2: 32 KB per SM and 64 token rows for
+//           2 x 128 x 256 x 64 products, against 48 KB for half of that with MT = 1.
 //
 // The token count of an expert is ragged.  Rows of the last 64-row block that belong to the next
 // expert must not contribute: whole 16-row MMA steps beyond the expert's end are not issued, and
@@ -23,19 +30,26 @@ constexpr int WM = 128;                 // output rows per tile (MMA M)
 constexpr int WN = 256;                 // output columns per tile (MMA N)
 constexpr int WK = 64;                  // token rows per pipeline stage
 constexpr int UK = 16;                  // token rows per MMA
-constexpr int STAGES = 4;
-constexpr int ACC_STAGES = 2;
 constexpr int BOX_BYTES = 64 * WK * 2;  // one TMA box: 64 columns x 64 rows of bf16
-constexpr int A_BYTES = (WM / 64) * BOX_BYTES;
-constexpr int B_BYTES = (WN / 64) * BOX_BYTES;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 48 KB
-constexpr int EPI_WARPS = 4;
+constexpr int EPI_WARPS = 8;                            // two per TMEM lane quadrant
+constexpr int EPI_PER_Q = EPI_WARPS / 4;
 constexpr int EPI_BYTES = EPI_WARPS * 32 * 32 * 4;      // a 32 x 32 float block per warp
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
-constexpr int TMEM_COLS = ACC_STAGES * WN;              // 512
-constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 256;
+constexpr int TMEM_COLS = 512;
+constexpr int MAX_STAGES = 4;
+template <int MT>
+struct Shape {
+    static constexpr int TILE_M = MT * WM;
+    static constexpr int STAGES = MT == 1 ? 4 : 3;
+    static constexpr int ACC_STAGES = 2 / MT;
+    static constexpr int A_BYTES = (TILE_M / 64) * BOX_BYTES;
+    static constexpr int B_BYTES = (WN / 64) * BOX_BYTES;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 48 KB / 64 KB
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 256;
+};
 constexpr uint32_t kInstrDescBothMN = (1u << 15) | (1u << 16);
 constexpr int MAX_PROBLEMS = 3;
+constexpr int TALL_TILE_MIN_ROWS = 1024;   // average rows per expert from which MT = 2 is used
 
 struct Problem {
     CUtensorMap a;      // [R, M] bf16, box 64 x 64
@@ -58,6 +72,7 @@ struct Item {
 // Items run expert by expert (all tiles of all problems of an expert are neighbours, so the CTAs
 // that run at the same time share that expert's operand rows in L2), then problem, m tile, n tile
 // (neighbouring CTAs write neighbouring 1 KB pieces of the same gradient rows).
+template <int MT>
 __device__ __forceinline__ Item decode(const Params& P, int i) {
     const int e = i / P.tiles_per_expert, t = i - e * P.tiles_per_expert;
     int q = 0;
@@ -66,12 +81,16 @@ __device__ __forceinline__ Item decode(const Params& P, int i) {
         if (k < P.n_problems && t >= P.p[k].tile0) q = k;
     const int rem = t - P.p[q].tile0;
     const int m = rem / P.p[q].nt, n = rem - m * P.p[q].nt;     // n fastest: neighbours fill a row
-    return Item{q, e, m * WM, n * WN};
+    return Item{q, e, m * (MT * WM), n * WN};
 }
 
+template <int MT>
 __global__ void __launch_bounds__(THREADS, 1)
 wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offsets,
              int32_t* dev_status) {
+    using S = Shape<MT>;
+    constexpr int STAGES = S::STAGES, ACC_STAGES = S::ACC_STAGES, STAGE_BYTES = S::STAGE_BYTES;
+    constexpr int A_BYTES = S::A_BYTES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -79,8 +98,8 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
     const uint32_t bar0 = base + STAGES * STAGE_BYTES + EPI_BYTES;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + ACC_STAGES + a); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * MAX_STAGES + 2 + a); };
     uint8_t* misc = epi_ptr + EPI_BYTES + 128;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
@@ -110,7 +129,7 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
             uint32_t phase = 0;
             bool ok = true;
             for (int w = w_begin; ok && w < w_end; w += w_step) {
-                const Item it = decode(P, w);
+                const Item it = decode<MT>(P, w);
                 const CUtensorMap* amap = &P.p[it.q].a;
                 const CUtensorMap* bmap = &P.p[it.q].b;
                 const int lo = offsets[it.e], hi = offsets[it.e + 1];
@@ -122,7 +141,7 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
                     const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_BYTES;
                     mbar_expect_tx(full_bar(stage), (uint32_t)STAGE_BYTES);
 #pragma unroll
-                    for (int bx = 0; bx < WM / 64; ++bx)
+                    for (int bx = 0; bx < S::TILE_M / 64; ++bx)
                         tma_load_2d(sa + bx * BOX_BYTES, amap, it.m0 + 64 * bx, row,
                                     full_bar(stage));
 #pragma unroll
@@ -144,15 +163,16 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
         uint32_t phase = 0, acc_phase = 0;
         bool ok = true;
         constexpr uint32_t idesc = instr_desc_bf16(WM, WN) | kInstrDescBothMN;
+        constexpr int HALF_A = (WM / 64) * BOX_BYTES;     // the A boxes of one 128-row half
         for (int w = w_begin; ok && w < w_end; w += w_step) {
-            const Item it = decode(P, w);
+            const Item it = decode<MT>(P, w);
             const int lo = offsets[it.e], hi = offsets[it.e + 1];
             int go = 1;
             if (lane == 0)
                 go = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, dev_status) ? 1 : 0;
             if (!__shfl_sync(0xffffffffu, go, 0)) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * WN);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * MT * WN);
             for (int row = lo; row < hi; row += WK) {
                 if (lane == 0)
                     go = mbar_wait(full_bar(stage), phase, abort_flag, dev_status) ? 1 : 0;
@@ -165,7 +185,7 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
                 const int valid = min(WK, hi - row);
                 const int ksteps = (valid + UK - 1) / UK;
                 if (valid < ksteps * UK) {
-                    // rows valid .. ksteps*16-1 of all six boxes: 8 x 16 bytes per row and box
+                    // rows valid .. ksteps*16-1 of every box: 8 x 16 bytes per row and box
                     uint8_t* tile = base_ptr + stage * STAGE_BYTES;
                     const int n_rows = ksteps * UK - valid;
                     const int n_vec = n_rows * (STAGE_BYTES / BOX_BYTES) * 8;
@@ -179,12 +199,16 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    const uint64_t da = smem_desc_mn_sw128(sa, BOX_BYTES);
                     const uint64_t db = smem_desc_mn_sw128(sb, BOX_BYTES);
-                    for (int kk = 0; kk < ksteps; ++kk)
-                        tc_mma_bf16(d_tmem, da + (uint64_t)(kk * (2048 >> 4)),
-                                    db + (uint64_t)(kk * (2048 >> 4)), idesc,
-                                    (row != lo || kk != 0) ? 1u : 0u);
+#pragma unroll
+                    for (int half = 0; half < MT; ++half) {
+                        const uint64_t da = smem_desc_mn_sw128(sa + half * HALF_A, BOX_BYTES);
+                        for (int kk = 0; kk < ksteps; ++kk)
+                            tc_mma_bf16(d_tmem + (uint32_t)(half * WN),
+                                        da + (uint64_t)(kk * (2048 >> 4)),
+                                        db + (uint64_t)(kk * (2048 >> 4)), idesc,
+                                        (row != lo || kk != 0) ? 1u : 0u);
+                    }
                     tc_commit(empty_bar(stage));
                 }
                 __syncwarp();
@@ -197,13 +221,16 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
         }
     } else {
         // ------------------------------ epilogue: TMEM -> float32 rows --------------------------
+        // Two warps per TMEM lane quadrant; the chunks of 32 columns of a tile alternate between
+        // them.  The TMEM load of a warp's next chunk is in flight while it stores the current one.
         const int q = warp & 3;                       // TMEM lane quadrant this warp may read
+        const int grp = (warp - 2) >> 2;              // which of the quadrant's two warps
         float4* tbuf = reinterpret_cast<float4*>(epi_ptr + (warp - 2) * 4096);
         int acc = 0;
         uint32_t acc_phase = 0;
         bool alive = true;
         for (int w = w_begin; w < w_end; w += w_step) {
-            const Item it = decode(P, w);
+            const Item it = decode<MT>(P, w);
             const int M = P.p[it.q].M, N = P.p[it.q].N;
             float* out = P.p[it.q].out + (size_t)it.e * M * N;
             const bool empty = offsets[it.e + 1] == offsets[it.e];   // no MMA ran: gradient 0
@@ -212,18 +239,17 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
                 alive = __all_sync(0xffffffffu, ok);
             }
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * WN);
-#pragma unroll 1
-            for (int c = 0; c < WN && alive; c += 32) {
-                if (it.n0 + c >= N) break;
-                float v[32];
-                if (!empty) {
-                    tc_ld32(taddr + c, v);
-                    tc_wait_ld();
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = 0.f;
-                }
+            // chunk u = (128-row half, 32 columns): only those that hold outputs of the problem
+            const int cols_ok = min(WN / 32, (N - it.n0 + 31) / 32);
+            const int halves_ok = min(MT, (M - it.m0 + WM - 1) / WM);
+            const int n_u = alive ? halves_ok * cols_ok : 0;
+            const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * MT * WN);
+            auto load = [&](int u, float(&v)[32]) {
+                const int half = u / cols_ok, c = (u - half * cols_ok) * 32;
+                tc_ld32(tacc + (uint32_t)(half * WN + c), v);
+            };
+            auto store = [&](int u, float(&v)[32]) {
+                const int half = u / cols_ok, c = (u - half * cols_ok) * 32;
                 // the lane's row goes to shared memory in 16-byte pieces, piece j at slot
                 // j ^ (row & 7): conflict-free both for these stores and for the row reads below
 #pragma unroll
@@ -240,11 +266,30 @@ wgrad_kernel(const __grid_constant__ Params P, const int32_t* __restrict__ offse
 #pragma unroll
                 for (int rr = 0; rr < 8; ++rr) {
                     const int r = rr * 4 + (lane >> 3), j = lane & 7;
-                    const int m = it.m0 + q * 32 + r, n = it.n0 + c + 4 * j;
+                    const int m = it.m0 + half * WM + q * 32 + r, n = it.n0 + c + 4 * j;
                     if (m < M && n + 4 <= N)
                         *reinterpret_cast<float4*>(out + (size_t)m * N + n) = val[rr];
                 }
                 __syncwarp();
+            };
+            float va[32], vb[32];
+            if (empty) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) va[i] = vb[i] = 0.f;
+            }
+            int u = grp;
+            if (u < n_u && !empty) load(u, va);
+#pragma unroll 1
+            while (u < n_u) {
+                tc_wait_ld();
+                if (u + EPI_PER_Q < n_u && !empty) load(u + EPI_PER_Q, vb);
+                store(u, va);
+                u += EPI_PER_Q;
+                if (u >= n_u) break;
+                tc_wait_ld();
+                if (u + EPI_PER_Q < n_u && !empty) load(u + EPI_PER_Q, va);
+                store(u, vb);
+                u += EPI_PER_Q;
             }
             tc_fence_before();
             __syncwarp();
@@ -282,11 +327,16 @@ r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, c
     if (R == 0) return R3_OK;
     static PerDevice attr_set;
     if (!attr_set.done()) {
-        if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(wgrad_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Shape<1>::SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(wgrad_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Shape<2>::SMEM_BYTES) != cudaSuccess)
             return R3_ERR_CUDA;
         attr_set.mark();
     }
+    // the tall tile once an expert holds enough rows for its operand traffic to matter more than
+    // an epilogue that the next tile's MMAs do not hide
+    const int MT = R / (uint64_t)s->E >= (uint64_t)TALL_TILE_MIN_ROWS ? 2 : 1;
     Params P;
     const void* a_ptr[3] = {dout, da, db};
     const void* b_ptr[3] = {h, xp, xp};
@@ -301,7 +351,7 @@ r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, c
         p.out = out[q];
         p.M = Ms[q];
         p.N = Ns[q];
-        p.mt = (Ms[q] + WM - 1) / WM;
+        p.mt = (Ms[q] + MT * WM - 1) / (MT * WM);
         p.nt = (Ns[q] + WN - 1) / WN;
         p.tile0 = tiles;
         tiles += p.mt * p.nt;
@@ -311,7 +361,10 @@ r3_status launch_wgrad_tc(const r3_shape* s, const void* xp, const void* dout, c
     const int items = s->E * tiles;
     P.total_items = items;
     const int grid = items < sm_count() ? items : sm_count();
-    wgrad_kernel<<<grid, THREADS, SMEM_BYTES, cs>>>(P, offsets, dev_status);
+    if (MT == 2)
+        wgrad_kernel<2><<<grid, THREADS, Shape<2>::SMEM_BYTES, cs>>>(P, offsets, dev_status);
+    else
+        wgrad_kernel<1><<<grid, THREADS, Shape<1>::SMEM_BYTES, cs>>>(P, offsets, dev_status);
     return launch_status();
 }
 

@@ -195,6 +195,8 @@ def test_layer_backward_full_size_sampled_tokens(r3):
     (300, 2048, 16, 8, 768),      # the paper-like layer shape, ragged expert sizes
     (77, 136, 6, 3, 72),          # ragged d, F; experts smaller than one 64-row block
     (1500, 512, 3, 2, 264),       # experts spanning many 64-row blocks
+    (2300, 328, 3, 2, 520),       # over 1024 rows per expert: the 256-row tile, ragged d and F
+    (2100, 512, 2, 1, 256),       # the 256-row tile with full tiles only
 ])
 def test_expert_weight_gradients(r3, T, d, E, K, F):
     """r3_grouped_swiglu_bwd: dW_gate, dW_up, dW_down of every expert against the oracle, fed the
