@@ -250,11 +250,14 @@ def test_expert_weight_gradients(r3, T, d, E, K, F):
     assert all(torch.equal(p, q) for p, q in zip((dxp, dwg, dwu, dwd), again))
 
 
-def test_layer_backward_with_expert_weight_gradients(r3):
+@pytest.mark.parametrize("T,d,E,K,F", [
+    (700, 256, 16, 4, 136),       # 175 rows per expert: the 128-row weight-gradient tile
+    (2200, 320, 4, 2, 264),       # 1100 rows per expert: the 256-row tile, ragged d and F
+])
+def test_layer_backward_with_expert_weight_gradients(r3, T, d, E, K, F):
     from paper_2510_11370_b200 import synth
     from tests.helpers import Case
-    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_w", T=700, d=256, E=16, K=4,
-                     F=136)
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="bwd_w", T=T, d=d, E=E, K=K, F=F)
     case = Case(w)
     c = case.cuda()
     s = r3.shape_of(w)
