@@ -95,8 +95,12 @@ r3_status grouped_swiglu_keep_lists(const r3_shape* shape, const void* xp, const
                                     size_t ws_bytes, int32_t* dev_status, void* stream);
 
 // The row copy of the dispatch alone: xp[row_of_slot[t, j]] = x[t] (maps from an earlier r3_permute).
+// x_early = true only when the kernel launched just before on the stream does not write x and
+// cannot let this one start before everything in front of it has completed (the dispatch kernels):
+// the token rows are then fetched before the dependency wait.
 r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_t* row_of_slot,
-                              void* xp, cudaStream_t stream, int32_t* dev_status);
+                              void* xp, cudaStream_t stream, int32_t* dev_status,
+                              bool x_early = false);
 
 // Number of SMs of the current device (cached).
 int sm_count();

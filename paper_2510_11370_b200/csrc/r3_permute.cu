@@ -314,8 +314,11 @@ permute_maps_cluster_kernel(const IdxT* __restrict__ idx, int32_t* __restrict__ 
     for (int e = lt; e < E; e += kChunk) hist[e] = 0;
     for (int i = lt; i < E * kWords; i += kChunk) bits[i] = 0u;
     __syncthreads();
-    tc::grid_launch_dependents();
+    // The wait comes first here: once this grid lets its dependent start, everything before it
+    // in the stream has completed, so the row copy launched right behind it may fetch the token
+    // rows (which this kernel does not write) before its own wait.
     tc::grid_dependency_wait();                    // the record may come from the kernel before
+    tc::grid_launch_dependents();
     int kept[8];                                   // slots 0..7: the expert, or -1 for a dropped pair
 #pragma unroll
     for (int u = 0; u < 8; ++u) kept[u] = -1;
@@ -464,7 +467,7 @@ constexpr int kRowTokens = 8;
 __global__ void __launch_bounds__(32)
 permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ row_of_slot,
                            uint8_t* __restrict__ xp, int T, int K, uint32_t row_bytes,
-                           int32_t* dev_status) {
+                           int x_early, int32_t* dev_status) {
     extern __shared__ __align__(128) uint8_t smem_p[];
     const uint32_t bar = tc::smem_u32(smem_p);
     volatile int* flags = reinterpret_cast<volatile int*>(smem_p + 8);
@@ -479,13 +482,20 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
         tc::mbar_expect_tx(bar, row_bytes * (uint32_t)nt);
     }
     __syncwarp();
+    auto fetch_rows = [&]() {
+        if (lane < nt)
+            asm volatile(
+                "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                ::"r"(rows0 + (uint32_t)lane * row_bytes), "l"(x + (size_t)(t0 + lane) * row_bytes),
+                  "r"(row_bytes), "r"(bar) : "memory");
+    };
+    // x_early: the kernel before this one in the stream does not write x and lets this grid start
+    // only after everything before IT has completed (the dispatch kernels), so the token rows are
+    // fetched while the dispatch is still computing the maps.
+    if (x_early) fetch_rows();
     tc::grid_launch_dependents();
-    tc::grid_dependency_wait();            // x and the maps may come from the kernel before
-    if (lane < nt)
-        asm volatile(
-            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-            ::"r"(rows0 + (uint32_t)lane * row_bytes), "l"(x + (size_t)(t0 + lane) * row_bytes),
-              "r"(row_bytes), "r"(bar) : "memory");
+    tc::grid_dependency_wait();            // the maps (and, unless x_early, x) come from before
+    if (!x_early) fetch_rows();
     int32_t r[8];
     // destination rows of this lane's token, fetched while the copy flies; K > 8 goes in rounds
     const int32_t* rows = row_of_slot + (size_t)(t0 + (lane < nt ? lane : 0)) * K;
@@ -517,7 +527,7 @@ permute_rows_staged_kernel(const uint8_t* __restrict__ x, const int32_t* __restr
 }
 
 r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_t* row_of_slot,
-                              void* xp, cudaStream_t cs, int32_t* dev_status) {
+                              void* xp, cudaStream_t cs, int32_t* dev_status, bool x_early) {
     const int T = shape->T, K = shape->K;
     const size_t row_bytes = (size_t)shape->d * act_bytes(shape);
     if (row_bytes * kRowTokens <= 96 * 1024) {
@@ -533,7 +543,7 @@ r3_status launch_permute_rows(const r3_shape* shape, const void* x, const int32_
         if (tc::launch_dependent(permute_rows_staged_kernel, dim3((T + kRowTokens - 1) / kRowTokens),
                                  dim3(32), smem, cs, static_cast<const uint8_t*>(x), row_of_slot,
                                  static_cast<uint8_t*>(xp), T, K, (uint32_t)row_bytes,
-                                 dev_status) != cudaSuccess)
+                                 x_early ? 1 : 0, dev_status) != cudaSuccess)
             return R3_ERR_CUDA;
         return launch_status();
     }
@@ -666,7 +676,11 @@ r3_status r3::permute_impl(const r3_shape* shape, const void* idx, const void* x
             static_cast<const IdxT*>(idx), chunk_counts, offsets, row_of_slot, slot_of_row,
             T, E, K, NB));
     }
-    if (x) return r3::launch_permute_rows(shape, x, row_of_slot, xp, cs, dev_status);
+    // The kernel in front of the row copy is one of the dispatch kernels above: none writes x,
+    // the one-cluster form lets its dependent start only after its own wait and the others not
+    // before they end, so everything earlier in the stream has completed when the row copy starts
+    // and it may fetch the token rows before its wait.
+    if (x) return r3::launch_permute_rows(shape, x, row_of_slot, xp, cs, dev_status, true);
     return r3::launch_status();
 }
 
