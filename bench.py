@@ -1073,7 +1073,6 @@ def run_diag(args):
     from paper_2510_11370_b200 import build
     build.build()
     from paper_2510_11370_b200 import r3
-    from oracle import r3_diag_oracle as D
     if int(os.environ.get("RANK", "0")) != 0:
         return
     dev = torch.device("cuda", 0)
@@ -1114,6 +1113,8 @@ def run_diag(args):
     ms_g = timed(lambda: r3.record_gather(s, L, PT, pages, bt, cu, Ts, out=out_rec))
     pos0 = torch.zeros(Bq, dtype=torch.int32, device=dev)
     ms_a = timed(lambda: r3.record_append(s, L, PT, pages, bt, pos0, cu, out_rec))
+    # cpu_baseline leg: the oracle, as it stands, on a bounded sample
+    from oracle import r3_diag_oracle as D
     t0 = time.perf_counter()
     m = 2_000_000
     ref_kl = D.kl_k3(pt[:m].cpu().numpy(), pi[:m].cpu().numpy())
