@@ -275,3 +275,55 @@ def test_layer_backward_with_expert_weight_gradients(r3, T, d, E, K, F):
     y0, ds0, dx0, dwr0 = r3.replay_layer_train(s, c["x"], c["w_r"], c["idx"], c["w_gate"],
                                                c["w_up"], c["w_down"], c["dy"])
     assert torch.equal(dx, dx0) and torch.equal(dw_r, dwr0) and torch.equal(y, y0)
+
+
+def test_expert_weight_gradients_paper_shape_sampled_experts(r3):
+    """The 256-row weight-gradient tile at the paper-like layer shape (16384 tokens, 1024 rows per
+    expert on average, d=2048, F=768): the experts with the most and the fewest rows and one in
+    between, each of its three gradients in full against the oracle.  The inputs are drawn on the
+    device by torch; the stored pre-activations of the checked experts are formed on the host in
+    float64 and rounded to bf16 (those of the other experts are random: their gradients are not
+    looked at)."""
+    T, d, E, K, F = 16384, 2048, 128, 8, 768
+    R = T * K
+    dev = torch.device("cuda", 0)
+    bf = torch.bfloat16
+    rng = np.random.default_rng(11)
+    idx_np = np.argsort(rng.random((T, E)) * (0.5 + rng.random(E))[None, :], axis=1)[:, :K]
+    counts, offsets, ros, sor = O.permutation(idx_np, E)
+    g = torch.Generator(device=dev).manual_seed(11)
+    x = torch.randn(T, d, generator=g, device=dev).to(bf)
+    wg = (torch.randn(E, F, d, generator=g, device=dev) * 0.05).to(bf)
+    wu = (torch.randn(E, F, d, generator=g, device=dev) * 0.05).to(bf)
+    wd = (torch.randn(E, d, F, generator=g, device=dev) * 0.05).to(bf)
+    dout = torch.randn(R, d, generator=g, device=dev).to(bf)
+    a = torch.randn(R, F, generator=g, device=dev).to(bf)
+    b = torch.randn(R, F, generator=g, device=dev).to(bf)
+    xp = x[torch.from_numpy(sor.astype(np.int64)).to(dev) // K].contiguous()
+    order = np.argsort(counts)
+    picks = [int(order[-1]), int(order[0]), int(order[E // 2])]
+    assert counts[picks[0]] > 1024          # the 256-row tile is the one that runs
+    host = {}
+    for e in picks:
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        xe = f64(xp[lo:hi].cpu())
+        a[lo:hi] = torch.from_numpy(xe @ f64(wg[e].cpu()).T).to(bf).to(dev)
+        b[lo:hi] = torch.from_numpy(xe @ f64(wu[e].cpu()).T).to(bf).to(dev)
+        host[e] = (xe, f64(dout[lo:hi].cpu()))
+    s = r3.make_shape(T, d, E, K, F)
+    st = r3.new_status(dev)
+    dxp, dwg, dwu, dwd = r3.grouped_swiglu_bwd(s, xp, dout, a, b, torch.from_numpy(offsets).to(dev),
+                                               wg, wu, wd, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    worst = 0.0
+    for e in picks:
+        xe, de = host[e]
+        ref = O.swiglu_expert_bwd_weights(xe, de, f32(wg[e].cpu()), f32(wu[e].cpu()),
+                                          f32(wd[e].cpu()))
+        for k, got in enumerate((dwg, dwu, dwd)):
+            err = rel_err(f64(got[e].cpu()), ref[k])
+            worst = max(worst, err)
+            assert err < TOL_BF16, (e, k, err, int(counts[e]))
+    print(f"weight gradients at T={T}: rows of the checked experts "
+          f"{[int(counts[e]) for e in picks]}, worst error {worst:.2e}")
