@@ -601,7 +601,12 @@ def measure_layer(torch, r3, r3dist, inp, args, peaks, sampler, world=1, dev=Non
     r3dist.barrier()
     e2e_ms = r3dist.max_over_ranks(ev0.elapsed_time(ev1), dev)
     assert st.item() == 0
-    assert torch.equal(yh.to(dev), y), "host-buffer path disagrees with the device path"
+    # the host-buffer call sends a large batch through in chunks of tokens, whose router launches
+    # may split d differently from the whole batch's: equal up to a bf16 rounding step
+    y_dev, y_host = y.float(), yh.to(dev).float()
+    assert float((y_host - y_dev).abs().max()) <= 2.0 ** -7 * float(y_dev.abs().max()), \
+        "host-buffer path disagrees with the device path"
+    del y_dev, y_host
     e2e_rec = {"value": world * T * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": int(xh.numel() * es + dyh.numel() * es + idxh.numel() * idxh.element_size()),
                "d2h_bytes_per_step": int(yh.numel() * es + dlh.numel() * 4),
@@ -637,7 +642,8 @@ def measure_layer(torch, r3, r3dist, inp, args, peaks, sampler, world=1, dev=Non
     r3dist.barrier()
     pipe_ms = r3dist.max_over_ranks((tp1 - tp0) * 1e3, dev)
     assert st.item() == 0
-    assert all(torch.equal(ln["y"].to(dev), y) for ln in lanes)
+    # every lane ran the same chunked call as the single-batch measurement above: same bits
+    assert all(torch.equal(ln["y"], yh) for ln in lanes)
     e2e_rec["batches_in_flight"] = {
         "depth": depth, "value": world * T * e2e_steps / (pipe_ms * 1e-3), "unit": UNIT,
         "ms_per_step": pipe_ms / e2e_steps, "steps": e2e_steps,

@@ -294,7 +294,12 @@ r3_status r3_replay_stack(const r3_shape* shape, int32_t L, const void* x0, cons
 /* As r3_replay_layer, with the per-step tensors in HOST memory (pinned memory recommended):
  * x_host, idx_host, dy_host are copied to the device, y_host and dlogits_host are copied back,
  * and the stream is synchronised before returning.  Weights stay on the device.  The workspace
- * must hold r3_replay_layer_host_workspace_bytes(shape) bytes (device staging included). */
+ * must hold r3_replay_layer_host_workspace_bytes(shape) bytes (device staging included).
+ * From 16384 tokens on the batch goes through in chunks of at least 8192 tokens (at most 16
+ * chunks), each a layer of its own: the copies travel on two library-owned streams beside the
+ * kernels on `stream`, which ends behind the last result copy.  Every token's result is what a
+ * layer of its chunk alone gives; against one launch over the whole batch it may differ in the
+ * last bits (the router kernel sums d in another order for another token count). */
 size_t r3_replay_layer_host_workspace_bytes(const r3_shape* shape);
 r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host, const void* w_router,
                                const void* idx_host, const void* w_gate, const void* w_up,

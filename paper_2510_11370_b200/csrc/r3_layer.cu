@@ -13,10 +13,14 @@ namespace r3 {
 // per device, created at the first call on that device and kept until the process exits; the
 // helper is forked from and joined back into the caller's stream with the events, so the call as
 // a whole is still ordered on the caller's stream (and can be captured with it).
+constexpr int kHostChunksMax = 16;       // host-buffer entry point: token chunks in flight
+constexpr int kHostChunkTokens = 8192;   // ... and their least size
 struct SideStream {
     cudaStream_t stream = nullptr;
-    cudaStream_t copy = nullptr;   // host-buffer entry point: dy travels here beside the compute
+    cudaStream_t copy = nullptr;      // host-buffer entry point: inputs travel here beside the compute
+    cudaStream_t copy_out = nullptr;  // ... and results back on this one
     cudaEvent_t fork = nullptr, join = nullptr, copy_fork = nullptr, copied = nullptr;
+    cudaEvent_t in_ready[kHostChunksMax] = {}, done[kHostChunksMax] = {}, out_done = nullptr;
     int state = 0;                 // 0 = not tried, 1 = ready, -1 = unavailable
 };
 static SideStream* side_stream() {
@@ -27,13 +31,18 @@ static SideStream* side_stream() {
     std::lock_guard<std::mutex> lock(mu);
     SideStream& ss = per_device[dev];
     if (ss.state == 0) {
-        const bool ok =
+        bool ok =
             cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) == cudaSuccess &&
             cudaStreamCreateWithFlags(&ss.copy, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&ss.copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ss.out_done, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ss.copy_fork, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ss.copied, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) == cudaSuccess;
+        for (int c = 0; ok && c < kHostChunksMax; ++c)
+            ok = cudaEventCreateWithFlags(&ss.in_ready[c], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ss.done[c], cudaEventDisableTiming) == cudaSuccess;
         ss.state = ok ? 1 : -1;
         if (!ok) cudaGetLastError();
     }
@@ -493,13 +502,69 @@ extern "C" r3_status r3_replay_layer_host_enqueue(const r3_shape* shape, const v
     const r3::HostWs h = r3::carve_host(shape, workspace);
     const size_t T = shape->T, row = (size_t)shape->d * r3::act_bytes(shape);
     if (!x_host || !w_router || !w_gate || !w_up || !w_down) return R3_ERR_INVALID_ARG;
+    r3::SideStream* side = r3::side_stream();
+    if (side && T >= 2 * (size_t)r3::kHostChunkTokens) {
+        // A large batch goes through in chunks of tokens (every step of the layer is per token once
+        // the record is given, so the chunks are layers of their own): chunk c + 1 crosses the link
+        // while chunk c computes and chunk c - 1 returns, so the call takes about the time of its
+        // host-to-device bytes instead of the sum of copies and compute.
+        size_t chunk = (T + r3::kHostChunksMax - 1) / r3::kHostChunksMax;
+        chunk = (chunk + 255) / 256 * 256;
+        if (chunk < (size_t)r3::kHostChunkTokens) chunk = r3::kHostChunkTokens;
+        const size_t idx_row = (size_t)shape->K * r3::idx_bytes(shape);
+        if (cudaEventRecord(side->copy_fork, cs) != cudaSuccess ||
+            cudaStreamWaitEvent(side->copy, side->copy_fork, 0) != cudaSuccess ||
+            cudaStreamWaitEvent(side->copy_out, side->copy_fork, 0) != cudaSuccess)
+            return R3_ERR_CUDA;
+        int n_chunks = 0;
+        for (size_t t0 = 0; t0 < T; t0 += chunk, ++n_chunks) {
+            const size_t n = T - t0 < chunk ? T - t0 : chunk;
+            if (cudaMemcpyAsync(static_cast<char*>(h.x) + t0 * row,
+                                static_cast<const char*>(x_host) + t0 * row, n * row,
+                                cudaMemcpyHostToDevice, side->copy) != cudaSuccess ||
+                cudaMemcpyAsync(static_cast<char*>(h.idx) + t0 * idx_row,
+                                static_cast<const char*>(idx_host) + t0 * idx_row, n * idx_row,
+                                cudaMemcpyHostToDevice, side->copy) != cudaSuccess ||
+                cudaMemcpyAsync(static_cast<char*>(h.dy) + t0 * row,
+                                static_cast<const char*>(dy_host) + t0 * row, n * row,
+                                cudaMemcpyHostToDevice, side->copy) != cudaSuccess ||
+                cudaEventRecord(side->in_ready[n_chunks], side->copy) != cudaSuccess)
+                return R3_ERR_CUDA;
+        }
+        int c = 0;
+        for (size_t t0 = 0; t0 < T; t0 += chunk, ++c) {
+            const size_t n = T - t0 < chunk ? T - t0 : chunk;
+            r3_shape part = *shape;
+            part.T = (int32_t)n;
+            if (cudaStreamWaitEvent(cs, side->in_ready[c], 0) != cudaSuccess) return R3_ERR_CUDA;
+            st = r3::run_layer(&part, static_cast<char*>(h.x) + t0 * row, w_router,
+                               static_cast<char*>(h.idx) + t0 * idx_row, w_gate, w_up, w_down,
+                               static_cast<char*>(h.dy) + t0 * row, nullptr,
+                               static_cast<char*>(h.y) + t0 * row, h.dlogits + t0 * shape->E,
+                               nullptr, h.inner, dev_status, stream);
+            if (st != R3_OK) return st;
+            if (cudaEventRecord(side->done[c], cs) != cudaSuccess ||
+                cudaStreamWaitEvent(side->copy_out, side->done[c], 0) != cudaSuccess ||
+                cudaMemcpyAsync(static_cast<char*>(y_host) + t0 * row,
+                                static_cast<char*>(h.y) + t0 * row, n * row,
+                                cudaMemcpyDeviceToHost, side->copy_out) != cudaSuccess ||
+                cudaMemcpyAsync(dlogits_host + t0 * shape->E, h.dlogits + t0 * shape->E,
+                                n * shape->E * 4, cudaMemcpyDeviceToHost, side->copy_out) !=
+                    cudaSuccess)
+                return R3_ERR_CUDA;
+        }
+        // the caller's stream ends behind the last result copy
+        if (cudaEventRecord(side->out_done, side->copy_out) != cudaSuccess ||
+            cudaStreamWaitEvent(cs, side->out_done, 0) != cudaSuccess)
+            return R3_ERR_CUDA;
+        return R3_OK;
+    }
     if (cudaMemcpyAsync(h.x, x_host, T * row, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
         cudaMemcpyAsync(h.idx, idx_host, T * shape->K * r3::idx_bytes(shape),
                         cudaMemcpyHostToDevice, cs) != cudaSuccess)
         return R3_ERR_CUDA;
     // x and the record are needed at once; dy only by the last kernel: it follows x over the
     // link on a copy stream of its own while the layer computes
-    r3::SideStream* side = r3::side_stream();
     cudaEvent_t dy_ready = nullptr;
     if (side) {
         if (cudaEventRecord(side->copy_fork, cs) != cudaSuccess ||

@@ -338,6 +338,65 @@ def test_host_buffer_layer_and_two_batches_in_flight(r3):
     assert st.item() == 0
 
 
+def test_host_buffer_layer_in_token_chunks(r3):
+    """From 16384 tokens on r3_replay_layer_host sends the batch through in chunks of 8192 tokens
+    (copies of one chunk beside the compute of another).  Every step of the layer is per token, so
+    a chunk must come out with the bits of running it alone on the device path (the whole batch
+    in one launch may differ in the last bits: the router kernel splits d differently for another
+    token count, so that run is compared within a bf16 rounding step); two such calls in flight
+    on streams of their own must not disturb each other."""
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], T=40000, d=256, E=16, K=4, F=136)
+    chunk = 8192
+    cases = [Case(w, device="cuda")]
+    cases.append(copy.copy(cases[0]))
+    cases[1].x = cases[1].x.flip(0).contiguous()
+    cases[1].dy = cases[1].dy.flip(0).contiguous()
+    cases[1].idx = cases[1].idx.flip(0).contiguous()
+    s = r3.shape_of(w)
+    st = r3.new_status("cuda")
+    dev = {k: getattr(cases[0], k).cuda() for k in ("w_r", "w_gate", "w_up", "w_down")}
+    alone, bufs = [], []
+    for c in cases:
+        ys, dss = [], []
+        for t0 in range(0, w.T, chunk):
+            n = min(chunk, w.T - t0)
+            sp = r3.shape_of(synth.scaled(w, T=n))
+            y, ds, _ = r3.replay_layer(sp, c.x[t0:t0 + n].cuda(), dev["w_r"],
+                                       c.idx[t0:t0 + n].cuda(), dev["w_gate"], dev["w_up"],
+                                       dev["w_down"], c.dy[t0:t0 + n].cuda(), dev_status=st)
+            torch.cuda.synchronize()
+            ys.append(y.cpu())
+            dss.append(ds.cpu())
+        alone.append((torch.cat(ys), torch.cat(dss)))
+        bufs.append(dict(x=c.x.pin_memory(), dy=c.dy.pin_memory(), idx=c.idx.pin_memory(),
+                         y=torch.empty((w.T, w.d), dtype=c.x.dtype).pin_memory(),
+                         ds=torch.empty((w.T, w.E), dtype=torch.float32).pin_memory(),
+                         ws=r3.workspace(r3.replay_layer_host_workspace_bytes(s), "cuda"),
+                         stream=torch.cuda.Stream()))
+    c = cases[0]
+    y_whole, ds_whole, _ = r3.replay_layer(s, c.x.cuda(), dev["w_r"], c.idx.cuda(), dev["w_gate"],
+                                           dev["w_up"], dev["w_down"], c.dy.cuda(), dev_status=st)
+    b = bufs[0]
+    r3.replay_layer_host(s, b["x"], dev["w_r"], b["idx"], dev["w_gate"], dev["w_up"], dev["w_down"],
+                         b["dy"], b["y"], b["ds"], ws=b["ws"], dev_status=st)
+    assert torch.equal(b["y"], alone[0][0]) and torch.equal(b["ds"], alone[0][1])
+    assert rel_err(f64(b["y"]), f64(y_whole)) < 2.0 ** -7
+    assert rel_err(f64(b["ds"]), f64(ds_whole)) < 1e-4
+    for rounds in range(2):
+        for b in bufs:
+            b["y"].zero_()
+            b["ds"].zero_()
+        for b in bufs:
+            r3.replay_layer_host_enqueue(s, b["x"], dev["w_r"], b["idx"], dev["w_gate"],
+                                         dev["w_up"], dev["w_down"], b["dy"], b["y"], b["ds"],
+                                         ws=b["ws"], dev_status=st, stream=b["stream"])
+        for b in bufs:
+            b["stream"].synchronize()
+        for b, (y, ds) in zip(bufs, alone):
+            assert torch.equal(b["y"], y) and torch.equal(b["ds"], ds)
+    assert st.item() == 0
+
+
 @pytest.mark.parametrize("name,T", [("c1_tiny_fp32", 512), ("c2_layer_bf16", 1500)])
 def test_second_pass_over_the_same_record(r3, name, T):
     """r3_replay_layer_same_record uses the dispatch and the work lists that r3_replay_layer left
