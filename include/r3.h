@@ -295,12 +295,19 @@ r3_status r3_replay_stack(const r3_shape* shape, int32_t L, const void* x0, cons
  * x_host, idx_host, dy_host are copied to the device, y_host and dlogits_host are copied back,
  * and the stream is synchronised before returning.  Weights stay on the device.  The workspace
  * must hold r3_replay_layer_host_workspace_bytes(shape) bytes (device staging included).
- * From 16384 tokens on the batch goes through in chunks of at least 8192 tokens (at most 16
- * chunks), each a layer of its own: the copies travel on two library-owned streams beside the
- * kernels on `stream`, which ends behind the last result copy.  Every token's result is what a
- * layer of its chunk alone gives; against one launch over the whole batch it may differ in the
- * last bits (the router kernel sums d in another order for another token count). */
+ * From 16384 tokens on the batch goes through in chunks of tokens (r3_replay_layer_host_chunks),
+ * each a layer of its own: the copies travel on two library-owned streams beside the kernels on
+ * `stream`, which ends behind the last result copy.  Every token's result is what a layer of its
+ * chunk alone gives; against one launch over the whole batch it may differ in the last bits (the
+ * router kernel sums d in another order for another token count). */
 size_t r3_replay_layer_host_workspace_bytes(const r3_shape* shape);
+/* How r3_replay_layer_host cuts shape->T tokens: writes starts[0..n] (host memory, room for 17
+ * values; starts[0] = 0, starts[n] = T, chunk c holds tokens [starts[c], starts[c+1])) and returns
+ * n; 0 for a bad shape or a null pointer.  Equal chunks of at least 8192 tokens, multiples of
+ * 256, the last one cut into a half and two quarters (the compute and the result copy of the last
+ * chunk are what the call cannot hide under its input copies).  A host-side schedule: the paper
+ * has no counterpart. */
+int32_t r3_replay_layer_host_chunks(const r3_shape* shape, int64_t* starts);
 r3_status r3_replay_layer_host(const r3_shape* shape, const void* x_host, const void* w_router,
                                const void* idx_host, const void* w_gate, const void* w_up,
                                const void* w_down, const void* dy_host, void* y_host,

@@ -477,7 +477,39 @@ static HostWs carve_host(const r3_shape* s, void* base) {
     h.total = off;
     return h;
 }
+// Token chunks of the host-buffer call: starts[0..n] with starts[n] = T; n = 1 below
+// 2 * kHostChunkTokens tokens.  Equal chunks of at least kHostChunkTokens tokens (a multiple of
+// 256, at most 12 of them), except that the last one is cut into a half and two quarters: what the
+// call cannot hide is the compute and the result copy of its LAST chunk, so that one is small.
+static int host_chunks(int64_t T, int64_t* starts) {
+    starts[0] = 0;
+    if (T < 2 * (int64_t)kHostChunkTokens) {
+        starts[1] = T;
+        return 1;
+    }
+    int64_t chunk = ((T + 11) / 12 + 255) / 256 * 256;
+    if (chunk < kHostChunkTokens) chunk = kHostChunkTokens;
+    int n = 0;
+    int64_t t = 0;
+    while (T - t > chunk) {
+        t += chunk;
+        starts[++n] = t;
+    }
+    const int64_t rest = T - t;                      // 1 .. chunk tokens
+    if (rest >= 4096) {
+        const int64_t half = rest / 2 / 256 * 256, quarter = rest / 4 / 256 * 256;
+        starts[++n] = t + half;
+        starts[++n] = t + half + quarter;
+    }
+    starts[++n] = T;
+    return n;
+}
 }  // namespace r3
+
+extern "C" int32_t r3_replay_layer_host_chunks(const r3_shape* shape, int64_t* starts) {
+    if (r3::check_shape(shape) != R3_OK || !starts) return 0;
+    return r3::host_chunks(shape->T, starts);
+}
 
 extern "C" size_t r3_replay_layer_host_workspace_bytes(const r3_shape* shape) {
     if (r3::check_shape(shape) != R3_OK) return 0;
@@ -508,17 +540,15 @@ extern "C" r3_status r3_replay_layer_host_enqueue(const r3_shape* shape, const v
         // the record is given, so the chunks are layers of their own): chunk c + 1 crosses the link
         // while chunk c computes and chunk c - 1 returns, so the call takes about the time of its
         // host-to-device bytes instead of the sum of copies and compute.
-        size_t chunk = (T + r3::kHostChunksMax - 1) / r3::kHostChunksMax;
-        chunk = (chunk + 255) / 256 * 256;
-        if (chunk < (size_t)r3::kHostChunkTokens) chunk = r3::kHostChunkTokens;
+        int64_t starts[r3::kHostChunksMax + 1];
+        const int n_chunks = r3::host_chunks((int64_t)T, starts);
         const size_t idx_row = (size_t)shape->K * r3::idx_bytes(shape);
         if (cudaEventRecord(side->copy_fork, cs) != cudaSuccess ||
             cudaStreamWaitEvent(side->copy, side->copy_fork, 0) != cudaSuccess ||
             cudaStreamWaitEvent(side->copy_out, side->copy_fork, 0) != cudaSuccess)
             return R3_ERR_CUDA;
-        int n_chunks = 0;
-        for (size_t t0 = 0; t0 < T; t0 += chunk, ++n_chunks) {
-            const size_t n = T - t0 < chunk ? T - t0 : chunk;
+        for (int c = 0; c < n_chunks; ++c) {
+            const size_t t0 = (size_t)starts[c], n = (size_t)(starts[c + 1] - starts[c]);
             if (cudaMemcpyAsync(static_cast<char*>(h.x) + t0 * row,
                                 static_cast<const char*>(x_host) + t0 * row, n * row,
                                 cudaMemcpyHostToDevice, side->copy) != cudaSuccess ||
@@ -528,12 +558,11 @@ extern "C" r3_status r3_replay_layer_host_enqueue(const r3_shape* shape, const v
                 cudaMemcpyAsync(static_cast<char*>(h.dy) + t0 * row,
                                 static_cast<const char*>(dy_host) + t0 * row, n * row,
                                 cudaMemcpyHostToDevice, side->copy) != cudaSuccess ||
-                cudaEventRecord(side->in_ready[n_chunks], side->copy) != cudaSuccess)
+                cudaEventRecord(side->in_ready[c], side->copy) != cudaSuccess)
                 return R3_ERR_CUDA;
         }
-        int c = 0;
-        for (size_t t0 = 0; t0 < T; t0 += chunk, ++c) {
-            const size_t n = T - t0 < chunk ? T - t0 : chunk;
+        for (int c = 0; c < n_chunks; ++c) {
+            const size_t t0 = (size_t)starts[c], n = (size_t)(starts[c + 1] - starts[c]);
             r3_shape part = *shape;
             part.T = (int32_t)n;
             if (cudaStreamWaitEvent(cs, side->in_ready[c], 0) != cudaSuccess) return R3_ERR_CUDA;

@@ -37,6 +37,7 @@ EXPORTS = [
     "r3_replay_layer_workspace_bytes",
     "r3_replay_layer", "r3_replay_blocks", "r3_replay_stack_workspace_bytes", "r3_replay_stack",
     "r3_replay_layer_host_workspace_bytes", "r3_replay_layer_host", "r3_replay_layer_host_enqueue",
+    "r3_replay_layer_host_chunks",
     "r3_replay_layer_same_record",
     "r3_prob_discrepancy_workspace_bytes", "r3_prob_discrepancy", "r3_record_diff",
     "r3_sequence_diff", "r3_grouped_swiglu_bwd_workspace_bytes", "r3_grouped_swiglu_bwd_input",
@@ -128,7 +129,9 @@ lib.r3_pagepool_alloc.argtypes = [_P, _I32, _P]
 lib.r3_pagepool_publish.argtypes = [_P, _P, _I32, _P, _I32]
 lib.r3_pagepool_release.argtypes = [_P, _P, _I32]
 lib.r3_selftest_bounded_wait.argtypes = [ctypes.c_int64, _P, _P, _P]
-_NOT_STATUS = ("r3_status_string", "r3_pagepool_create", "r3_pagepool_destroy")
+lib.r3_replay_layer_host_chunks.argtypes = [_SP, _P]
+_NOT_STATUS = ("r3_status_string", "r3_pagepool_create", "r3_pagepool_destroy",
+               "r3_replay_layer_host_chunks")
 for _n in EXPORTS:
     if _n not in _NOT_STATUS and not _n.endswith("_bytes"):
         getattr(lib, _n).restype = ctypes.c_int
@@ -471,6 +474,16 @@ def replay_layer_same_record(s: Shape, x, w_router, idx, w_gate, w_up, w_down, d
 
 def replay_layer_host_workspace_bytes(s: Shape) -> int:
     return lib.r3_replay_layer_host_workspace_bytes(ctypes.byref(s))
+
+
+def replay_layer_host_chunks(s: Shape) -> list:
+    """Token offsets [0, ..., T] of the chunks r3_replay_layer_host sends one after the other."""
+    starts = (ctypes.c_int64 * 17)()
+    lib.r3_replay_layer_host_chunks.restype = ctypes.c_int32
+    n = lib.r3_replay_layer_host_chunks(ctypes.byref(s), starts)
+    if n <= 0:
+        raise R3Error(1)
+    return [int(starts[i]) for i in range(n + 1)]
 
 
 def replay_layer_host(s: Shape, x_host, w_router, idx_host, w_gate, w_up, w_down, dy_host,

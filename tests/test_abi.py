@@ -87,3 +87,19 @@ def test_workspace_sizes_scale_with_the_layer(r3):
     assert r3.replay_layer_workspace_bytes(s) >= 2 * R * 2048 * 2 + R * 768 * 2
     assert r3.replay_layer_host_workspace_bytes(s) > r3.replay_layer_workspace_bytes(s)
     assert r3.permute_workspace_bytes(s) == 128 * 16 * 4
+
+
+def test_host_call_chunk_schedule(r3):
+    """r3_replay_layer_host_chunks: one chunk below 16384 tokens; above, chunks that cover
+    [0, T) without gaps, start on multiples of 256, number at most 16, and end with small ones."""
+    for T in (1, 300, 8192, 16383):
+        assert r3.replay_layer_host_chunks(r3.make_shape(T, 64, 16, 2, 64)) == [0, T]
+    for T in (16384, 16385, 40000, 65536, 100000, 1 << 20):
+        st = r3.replay_layer_host_chunks(r3.make_shape(T, 64, 16, 2, 64))
+        sizes = [b - a for a, b in zip(st, st[1:])]
+        assert st[0] == 0 and st[-1] == T and all(n > 0 for n in sizes)
+        assert 2 <= len(sizes) <= 16
+        assert all(a % 256 == 0 for a in st[:-1])
+        assert sizes[-1] <= max(sizes) // 2 + 256
+    assert r3.replay_layer_host_chunks(r3.make_shape(65536, 64, 16, 2, 64)) == \
+        [0, 8192, 16384, 24576, 32768, 40960, 49152, 57344, 61440, 63488, 65536]

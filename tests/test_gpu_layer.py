@@ -339,27 +339,28 @@ def test_host_buffer_layer_and_two_batches_in_flight(r3):
 
 
 def test_host_buffer_layer_in_token_chunks(r3):
-    """From 16384 tokens on r3_replay_layer_host sends the batch through in chunks of 8192 tokens
+    """From 16384 tokens on r3_replay_layer_host sends the batch through in chunks of tokens
     (copies of one chunk beside the compute of another).  Every step of the layer is per token, so
     a chunk must come out with the bits of running it alone on the device path (the whole batch
     in one launch may differ in the last bits: the router kernel splits d differently for another
     token count, so that run is compared within a bf16 rounding step); two such calls in flight
     on streams of their own must not disturb each other."""
     w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], T=40000, d=256, E=16, K=4, F=136)
-    chunk = 8192
     cases = [Case(w, device="cuda")]
     cases.append(copy.copy(cases[0]))
     cases[1].x = cases[1].x.flip(0).contiguous()
     cases[1].dy = cases[1].dy.flip(0).contiguous()
     cases[1].idx = cases[1].idx.flip(0).contiguous()
     s = r3.shape_of(w)
+    starts = r3.replay_layer_host_chunks(s)
+    assert starts == [0, 8192, 16384, 24576, 32768, 36352, 38144, 40000]
     st = r3.new_status("cuda")
     dev = {k: getattr(cases[0], k).cuda() for k in ("w_r", "w_gate", "w_up", "w_down")}
     alone, bufs = [], []
     for c in cases:
         ys, dss = [], []
-        for t0 in range(0, w.T, chunk):
-            n = min(chunk, w.T - t0)
+        for t0, t1 in zip(starts, starts[1:]):
+            n = t1 - t0
             sp = r3.shape_of(synth.scaled(w, T=n))
             y, ds, _ = r3.replay_layer(sp, c.x[t0:t0 + n].cuda(), dev["w_r"],
                                        c.idx[t0:t0 + n].cuda(), dev["w_gate"], dev["w_up"],
