@@ -540,6 +540,10 @@ extern "C" r3_status r3_replay_layer_host_enqueue(const r3_shape* shape, const v
         // the record is given, so the chunks are layers of their own): chunk c + 1 crosses the link
         // while chunk c computes and chunk c - 1 returns, so the call takes about the time of its
         // host-to-device bytes instead of the sum of copies and compute.
+        // the events below belong to the device, not to the call: one enqueue at a time, so that
+        // every wait is paired with the record of its own call
+        static std::mutex enqueue_mu;
+        std::lock_guard<std::mutex> lock(enqueue_mu);
         int64_t starts[r3::kHostChunksMax + 1];
         const int n_chunks = r3::host_chunks((int64_t)T, starts);
         const size_t idx_row = (size_t)shape->K * r3::idx_bytes(shape);
