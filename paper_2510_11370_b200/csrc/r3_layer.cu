@@ -114,6 +114,10 @@ static r3_status run_layer(const r3_shape* shape, const void* x, const void* w_r
                            int32_t* dev_status, void* stream, cudaEvent_t dy_ready = nullptr,
                            void* pre_gate = nullptr, void* pre_up = nullptr,
                            bool same_record = false) {
+    // the helper stream's fork and join events are per device: one layer is enqueued at a time,
+    // so that host threads calling at once cannot pair a wait with another call's record
+    static std::mutex layer_mu;
+    std::lock_guard<std::mutex> layer_lock(layer_mu);
     const LayerWs w = carve(shape, workspace);
     float* gates = gates_out ? gates_out : w.gates;
     r3_status st;
