@@ -26,6 +26,8 @@
  *    device and kept until the process exits: the router logits run there beside the
  *    permutation.  The helper is forked from and joined back into `stream` with events, so the
  *    call as a whole is ordered on `stream` exactly as if everything had been enqueued there.
+ *    Host threads may call at once: the enqueue of a layer takes a process-wide lock for its
+ *    few microseconds, because the helper streams and their events belong to the device.
  *  - Matrices are row-major and dense.  Weights are stored output-major: W_r [E, d],
  *    W_gate/W_up [E, F, d], W_down [E, d, F].
  *  - Activations and expert weights have dtype `act_dtype` (R3_F32 or R3_BF16); W_r has dtype
