@@ -537,6 +537,238 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     }
 }
 
+
+// ---- CTA-pair form: tokens on the M side, one tile of 256 tokens per pair of SMs ---------------
+// tcgen05.mma cta_group::2 with M = 256: CTA r of the pair holds tokens [128 r, 128 r + 128) of
+// the tile as its 128 tensor-memory lanes, all E experts as columns.  Per k block it copies its own
+// 128 token rows and only HALF of the router rows (experts [r E/2, (r+1) E/2)): the tensor cores of
+// the two SMs exchange the halves themselves.  A layer's 256-token decode batch then costs a CTA
+// 512 KB of x and 256 KB of W_r (bf16, d = 2048), the bytes of the two-way k split, but every CTA
+// ends with the COMPLETE logits of its tokens: no partial sums travel, and lane = token means that
+// a thread reads a token's logits straight out of tensor memory, 32 experts at a time.
+// 16 warps: warp 0 lane 0 copies, warp 1 lane 0 of the leader issues the MMAs, then warp w takes
+// lane quadrant w % 4 and the experts 32 (w / 4), 32 (w / 4) + 128: a thread sorts its 32 (or 64)
+// packed candidates into a list of 8 (the networks of group_topk), the lists of a token's four
+// threads meet in shared memory and the thread of the first chunk merges them.  A token whose
+// packed order is not certain is done again from its full-precision logits (moved to a row buffer
+// by the threads that hold them) by one warp with warp_topk_exact, 16 tokens per round.
+namespace pairm {
+constexpr int TM = 128;                  // tokens per CTA
+constexpr int THREADS = 16 * 32;
+constexpr int PSTAGES = 8;               // most ring stages
+constexpr int X_BYTES = TM * BK * 2;     // 16 KB
+constexpr int LIST = 9;                  // 8 candidates + runner
+constexpr int REDO_ROWS = 16;
+constexpr int EPI_BYTES = 4 * TM * LIST * 4 + REDO_ROWS * 256 * 4 + (TM + 4) * 4;
+}  // namespace pairm
+
+template <typename IdxT>
+__global__ void __launch_bounds__(pairm::THREADS, 1)
+router_pair_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                   IdxT* __restrict__ idx_out, float* __restrict__ logits_out, int T, int d, int E,
+                   int K, int planes, int stages, uint32_t tmem_cols, int ring_bytes) {
+    using namespace pairm;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const int w_bytes = (E >> 1) * BK * 2;               // half of the router rows, one plane
+    const int stage_bytes = X_BYTES + planes * w_bytes;
+    const uint32_t bar0 = base + (uint32_t)ring_bytes;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (PSTAGES + s); };
+    const uint32_t acc_bar = bar0 + 8u * (2 * PSTAGES);
+    uint8_t* misc = base_ptr + ring_bytes + 8 * (2 * PSTAGES + 1);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(misc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 4);
+    // after the k loop the ring's place holds the lists, the row buffer and the redo list
+    float* lists = reinterpret_cast<float*>(base_ptr);                   // [4][TM][LIST]
+    float* rowbuf = lists + 4 * TM * LIST;                               // [REDO_ROWS][256]
+    int* redo_n = reinterpret_cast<int*>(rowbuf + REDO_ROWS * 256);      // count, then tokens
+    int* redo_tok = redo_n + 4;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int layer = blockIdx.y;
+    const uint32_t rank = cluster_ctarank();
+    const int t0 = (int)(blockIdx.x >> 1) * 2 * TM + (int)rank * TM;   // this CTA's first token
+    const int n_mine = max(0, min(TM, T - t0));
+    const int kblocks = (d + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(acc_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // nothing above touched global memory: it may have run beside the previous kernel of the stream
+    grid_dependency_wait();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < kblocks; ++kb) {
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, nullptr)) { ok = false; break; }
+                const uint32_t sx = base + stage * stage_bytes, sw = sx + X_BYTES;
+                const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
+                if (rank == 0) mbar_expect_tx(full_bar(stage), (uint32_t)(2 * stage_bytes));
+                tma_load_2d_pair(sx, &tmX, kb * BK, layer * T + t0, lead_full);
+                for (int p = 0; p < planes; ++p)
+                    tma_load_3d_pair(sw + p * w_bytes, &tmW, kb * BK, (int)rank * (E >> 1),
+                                     layer * planes + p, lead_full);
+                if (++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+            // every stage's release (signalled from the leader's tensor core) has landed
+            for (int s = 0; ok && s < stages && s < kblocks; ++s) {
+                ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, nullptr);
+                if (++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_bf16(2 * TM, E);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                if (!mbar_wait(full_bar(stage), phase, abort_flag, nullptr)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sx = base + stage * stage_bytes, sw = sx + X_BYTES;
+                const uint64_t da = smem_desc_sw128(sx);
+                for (int p = 0; p < planes; ++p) {
+                    const uint64_t db = smem_desc_sw128(sw + p * w_bytes);
+#pragma unroll
+                    for (int kk = 0; kk < BK / UK; ++kk)
+                        tc_mma_bf16_pair(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2),
+                                         idesc, (kb | p | kk) != 0 ? 1u : 0u);
+                }
+                tc_commit_pair(empty_bar(stage), 3);       // frees the stage in both CTAs
+                if (++stage == stages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok) tc_commit_pair(acc_bar, 3);            // accumulators complete, both CTAs
+        }
+        __syncwarp();
+    } else if (warp < 6) {
+        // the accumulator is complete: every copy has landed and every MMA has read its operands
+        __all_sync(0xffffffffu, mbar_wait(acc_bar, 0u, abort_flag, nullptr));
+    }
+    tc_fence_before();
+    __syncthreads();
+    // this grid has fetched its inputs: the next kernel of the stream may begin its set-up
+    grid_launch_dependents();
+    tc_fence_after();
+
+    // ------------------------------ epilogue -----------------------------------------------------
+    const int q = warp & 3, cg = warp >> 2;              // lane quadrant, chunk group
+    const int row = q * 32 + lane;                       // token of this thread within the CTA
+    const bool valid = row < n_mine && !*abort_flag;
+    const size_t out_row = (size_t)layer * T + t0 + row;
+    if (threadIdx.x == 0) *redo_n = 0;
+    TopList<8> list;
+    list.clear();
+    for (int c = cg * 32; c < E; c += 128) {             // uniform in the warp
+        float v[32];
+        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);
+        tc_wait_ld();
+        if (valid && logits_out) {
+            float4* dst = reinterpret_cast<float4*>(logits_out + out_row * E + c);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (c + 4 * i < E)                        // E is a multiple of 16
+                    dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        }
+        if (idx_out) {
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                if (c + 8 * b < E) {
+                    float cand[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) cand[i] = pack_candidate(v[8 * b + i], c + 8 * b + i);
+                    sort_desc<8>(cand);
+                    list.merge(cand, kNoCandidate);
+                }
+            }
+        }
+    }
+    if (idx_out) {
+        float* mine = lists + ((size_t)cg * TM + row) * LIST;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mine[i] = list.top[i];
+        mine[8] = list.runner;
+        __syncthreads();
+        if (cg == 0 && valid) {
+            for (int g = 1; g < 4 && g * 32 < E; ++g) {
+                const float* other = lists + ((size_t)g * TM + row) * LIST;
+                float o8[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o8[i] = other[i];
+                list.merge(o8, other[8]);
+            }
+            bool sure = true;
+            IdxT* out = idx_out + out_row * K;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float next = j + 1 < 8 ? list.top[j + 1 < 8 ? j + 1 : j] : list.runner;
+                if (j < K) {
+                    if ((__float_as_uint(list.top[j]) >> 8) == (__float_as_uint(next) >> 8)) sure = false;
+                    out[j] = (IdxT)candidate_expert(list.top[j]);
+                }
+            }
+            if (!sure) redo_tok[atomicAdd(redo_n, 1)] = row;
+        }
+        __syncthreads();
+        // tokens whose packed order was not certain: full-precision rows, one warp each
+        const int n_redo = *redo_n;
+        for (int r0 = 0; r0 < n_redo; r0 += REDO_ROWS) {
+            const int nb = min(REDO_ROWS, n_redo - r0);
+            for (int c = cg * 32; c < E; c += 128) {
+                float v[32];
+                tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);
+                tc_wait_ld();
+                for (int b = 0; b < nb; ++b) {
+                    if (redo_tok[r0 + b] == row) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) rowbuf[b * 256 + c + i] = v[i];
+                    }
+                }
+            }
+            __syncthreads();
+            if (warp < nb) {
+                Partials ps;
+                ps.p0 = rowbuf;
+                ps.p1 = rowbuf;
+                ps.stride = 0;
+                ps.n = 1;
+                const int tok = redo_tok[r0 + warp];
+                IdxT* out = idx_out + ((size_t)layer * T + t0 + tok) * K;
+                if (E <= 128) warp_topk_exact<IdxT, 4>(ps, 256, warp, lane, E, K, out);
+                else warp_topk_exact<IdxT, 8>(ps, 256, warp, lane, E, K, out);
+            }
+            __syncthreads();
+        }
+    }
+
+    // ------------------------------ teardown ---------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    cluster_sync_all();            // neither CTA leaves while the other may still signal it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, tmem_cols);
+    }
+}
+
 }  // namespace rt
 
 bool router_tc_supported(const r3_shape* s) {
@@ -596,6 +828,73 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
             total);
         wplanes = workspace;
     }
+    // The CTA-pair form (records of up to 8 experts; it writes the logits in 16-byte pieces).  It
+    // is taken below where the k-split form would put exactly two CTAs on a tile: with more CTAs
+    // per tile the split form is faster (one layer's decode batch: 16.5 us against 20.3 us), with
+    // one CTA per tile (many tiles) its coalesced logits stores are (65536 tokens: 0.075 against
+    // 0.10 ms).
+    // Returns R3_OK after a launch, R3_ERR_UNSUPPORTED when this device cannot run the pair form.
+    auto launch_pair_form = [&]() -> r3_status {
+        using namespace pairm;
+        const int stage_bytes = X_BYTES + planes * (s->E / 2) * BK * 2;
+        const int fixed = BAR_BYTES + 1024;
+        int stages = (SMEM_LIMIT - fixed) / stage_bytes;
+        if (stages > PSTAGES) stages = PSTAGES;
+        int ring = stages * stage_bytes;
+        if (ring < EPI_BYTES) ring = (EPI_BYTES + 127) & ~127;
+        uint32_t cols = 32;
+        while ((int)cols < s->E) cols <<= 1;
+        CUtensorMap px, pw;
+        if (!make_map_2d(&px, x, (uint64_t)L * s->T, (uint64_t)s->d, TM) ||
+            !make_map_3d(&pw, wplanes, (uint64_t)L * planes, (uint64_t)s->E, (uint64_t)s->d,
+                         (uint32_t)(s->E / 2)))
+            return R3_ERR_CUDA;
+        cudaLaunchConfig_t pc = {};
+        cudaLaunchAttribute pa[2];
+        pa[0].id = cudaLaunchAttributeClusterDimension;
+        pa[0].val.clusterDim.x = 2;
+        pa[0].val.clusterDim.y = 1;
+        pa[0].val.clusterDim.z = 1;
+        pa[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pa[1].val.programmaticStreamSerializationAllowed = 1;
+        const int tiles = (s->T + 2 * TM - 1) / (2 * TM);
+        pc.gridDim = dim3((unsigned)(2 * tiles), (unsigned)L);
+        pc.blockDim = dim3(pairm::THREADS);
+        pc.dynamicSmemBytes = (size_t)(ring + fixed);
+        pc.stream = cs;
+        pc.attrs = pa;
+        pc.numAttrs = 2;
+        static int pair_ok[64][2] = {};         // per device and index type: 0 untested, 1 yes, -1 no
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return R3_ERR_CUDA;
+        const int ti = s->idx_type == R3_IDX_U8 ? 0 : 1;
+        cudaError_t le = cudaSuccess;
+#define R3_RP(IDX)                                                                              \
+        do {                                                                                    \
+            auto kern = router_pair_kernel<IDX>;                                                \
+            if (pair_ok[dev][ti] == 0) {                                                        \
+                int n = 0;                                                                      \
+                cudaLaunchConfig_t probe = pc;                                                  \
+                probe.numAttrs = 1;                                                             \
+                probe.dynamicSmemBytes = (size_t)SMEM_LIMIT;                                    \
+                pair_ok[dev][ti] =                                                              \
+                    (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                                          SMEM_LIMIT) == cudaSuccess &&                         \
+                     cudaOccupancyMaxActiveClusters(&n, kern, &probe) == cudaSuccess && n >= 1) \
+                        ? 1 : -1;                                                               \
+                if (pair_ok[dev][ti] < 0) cudaGetLastError();                                   \
+            }                                                                                   \
+            if (pair_ok[dev][ti] == 1)                                                          \
+                le = cudaLaunchKernelEx(&pc, kern, px, pw, static_cast<IDX*>(idx_out),          \
+                                        logits_out, (int)s->T, (int)s->d, (int)s->E, (int)s->K, \
+                                        planes, stages, cols, ring);                            \
+        } while (0)
+        if (ti == 0) R3_RP(uint8_t); else R3_RP(int16_t);
+#undef R3_RP
+        if (pair_ok[dev][ti] == 1) return le == cudaSuccess ? launch_status() : R3_ERR_CUDA;
+        return R3_ERR_UNSUPPORTED;
+    };
+    const bool pair_form_fits = s->K <= 8 && aligned(logits_out, 16);
     // token tiles of a layer: as few as possible, of equal size (a multiple of 16); with two M
     // tiles (E > 128) the logits of 256 tokens would not fit in shared memory
     const int MT = (s->E + BME - 1) / BME;
@@ -656,6 +955,10 @@ r3_status launch_router_tc(const r3_shape* s, int L, const void* x, const void* 
         int ksplit = want >= 2 ? usable_split(kern, want, units) : 1;                           \
         while (ksplit > 1 && !fits(ksplit)) --ksplit;                                           \
         if (!fits(ksplit)) return R3_ERR_UNSUPPORTED;                                           \
+        if (ksplit == 2 && pair_form_fits) {                                                    \
+            const r3_status ps = launch_pair_form();                                            \
+            if (ps != R3_ERR_UNSUPPORTED) return ps;                                            \
+        }                                                                                       \
         int stages = (SMEM_LIMIT - fixed) / stage_bytes;                                        \
         if (stages > MAX_STAGES) stages = MAX_STAGES;                                           \
         int ring = stages * stage_bytes;                                                        \

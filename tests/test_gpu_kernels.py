@@ -330,6 +330,38 @@ def test_capture_batched_layers(r3):
         check_record_against_logits(idx[l].cpu().numpy(), ref_s, K)
 
 
+@pytest.mark.parametrize("L,T,d,E,K,rw", [
+    (50, 70, 256, 128, 8, torch.bfloat16),       # fewer tokens than one CTA of the pair holds
+    (60, 130, 320, 48, 3, torch.float32),        # two tokens for the second CTA, three weight planes
+    (50, 100, 256, 256, 8, torch.bfloat16),      # 256 experts: two column chunks per thread, int16 record
+    (47, 256, 512, 64, 1, torch.float32),        # a full tile, K = 1
+])
+def test_capture_batched_layers_pair_form(r3, L, T, d, E, K, rw):
+    """46 to 74 one-tile layers in a launch: the range in which the router kernel gives every tile a
+    pair of CTAs with the tokens on the M side of the MMA (the 48-layer decode batch of the paper's
+    setting is the full-size case).  Small-integer data, so logits and record must equal the
+    oracle's bit for bit; every token of layer 1 is a planted tie (experts 2, 5 and 17 share their
+    weights), which sends those tokens through the exact second selection, and layer 2 holds the
+    signed zeros."""
+    rng = np.random.default_rng(L + T + E)
+    x = torch.from_numpy(rng.integers(-3, 4, (L, T, d)).astype(np.float32)).to(torch.bfloat16)
+    w = torch.from_numpy(rng.integers(-2, 3, (L, E, d)).astype(np.float32)).to(rw)
+    w[1, 5] = w[1, 2]
+    w[1, 17] = w[1, 2]
+    w[1, E - 1] = w[1, 0]
+    plant_signed_zeros(x[2], w[2])
+    s = r3.make_shape(T, d, E, K, 8, router=rw, idx=idx_dtype(E))
+    idx, logits = r3.capture_topk_ws(s, L, x.cuda(), w.cuda(), want_logits=True)
+    for l in range(L):
+        ref_s = O.router_logits(f64(x[l]), f64(w[l]))
+        assert np.array_equal(logits[l].cpu().numpy().astype(np.float64), ref_s), l
+        assert np.array_equal(idx[l].cpu().numpy().astype(np.int64), O.topk_indices(ref_s, K)), l
+    only_idx, none = r3.capture_topk_ws(s, L, x.cuda(), w.cuda())
+    assert none is None and torch.equal(only_idx, idx)
+    _, only_logits = r3.capture_topk_ws(s, L, x.cuda(), w.cuda(), want_idx=False, want_logits=True)
+    assert torch.equal(only_logits, logits)
+
+
 # ------------------------------------------------------------------ grouped SwiGLU experts
 def run_swiglu_case(r3, T, d, E, K, F, act, tol, seed=0):
     rng = np.random.default_rng(seed + T)
