@@ -704,7 +704,7 @@ def measure_capture(torch, r3, synth, w, args, peaks, sampler, dev):
         "config": {"workload": w.name, "layers": L, "T": T, "d": d, "E": E, "K": K,
                    "l2": f"activations and router weights rotate over {reps} sets of "
                          f"{L * (T + E) * d * 2 / 1e6:.0f} MB (> L2 in all)"},
-        "roofline": {"bound": "hbm", "kernel": "router_tc_kernel (48 layers in one launch)",
+        "roofline": {"bound": "hbm", "kernel": "router_pair_kernel (48 layers in one launch)",
                      "achieved": round(bytes_b / ms_b / 1e6, 1), "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": round(bytes_b / ms_b / 1e6 / peaks["hbm_gbs"], 4),
                      "peak_kind": f"copy bandwidth, {peaks['source']}", "traffic": None},
