@@ -39,6 +39,9 @@ L2_BYTES = 126e6
 SUSTAINED_SECONDS = 0.6
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
+# DRAM bytes of one router_pair_kernel launch on the 48 x 256 decode capture (75.6 MB read +
+# 1.5 MB written; algorithmic 75.6 MB), from the ncu capture of that workload.
+CAPTURE_DRAM_TRAFFIC_BYTES = 77.05e6
 # DRAM bytes (read + write) of one launch of the up-projection GEMM kernel, from the ncu captures
 # summarised under profiles/ (a constant taken from the profile, not re-measured by a run)
 GEMM_UP_DRAM_TRAFFIC_BYTES = {"c2_layer_bf16": 988.8e6,     # 940.8 MB read + 48.0 MB written
@@ -707,7 +710,10 @@ def measure_capture(torch, r3, synth, w, args, peaks, sampler, dev):
         "roofline": {"bound": "hbm", "kernel": "router_pair_kernel (48 layers in one launch)",
                      "achieved": round(bytes_b / ms_b / 1e6, 1), "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": round(bytes_b / ms_b / 1e6 / peaks["hbm_gbs"], 4),
-                     "peak_kind": f"copy bandwidth, {peaks['source']}", "traffic": None},
+                     "peak_kind": f"copy bandwidth, {peaks['source']}",
+                     "traffic": CAPTURE_DRAM_TRAFFIC_BYTES if w.name == "c4_capture" else None,
+                     "traffic_source": "ncu capture summarised under profiles/ (a constant, not "
+                                       "re-measured by this run)"},
         "kernels": {"capture_batched": kern(ms_b),
                     "capture_one_layer": {"us_per_call": round(ms_1 * 1e3, 2)}},
         "record_bytes_per_step": L * T * K, "gpu_launches": steps,
