@@ -14,6 +14,7 @@ namespace r3 {
 
 constexpr int kMaxTaus = 16;
 constexpr int kDiagThreads = 256;
+constexpr int kFinalThreads = 1024;
 constexpr int kMaxDiffK = 32;
 
 // r - 1 - log r for r = a / b, in float32 without the cancellation of the literal form (for r
@@ -24,7 +25,9 @@ constexpr int kMaxDiffK = 32;
 // exact to 1e-16 but runs at a small fraction of the float32 rate: the kernel would be bound by
 // the float64 pipe, not by memory.
 __device__ __forceinline__ float k3_term(float a, float b) {
-    const float u = (a - b) / b;
+    // a - b is exact for values within a factor of two; the quotient may be two units off in its
+    // last place (the fast division), which is 2^-22 of the term: far inside its tolerance
+    const float u = __fdividef(a - b, b);
     if (fabsf(u) < 0.25f) {
         float p = 1.f / 13.f;
 #pragma unroll
@@ -34,41 +37,65 @@ __device__ __forceinline__ float k3_term(float a, float b) {
     return u - log1pf(u);
 }
 
+// NT = the number of thresholds rounded up to 4, 8 or 16 (unused ones are +inf: never exceeded).
+// A thread takes 16-byte pieces (four tokens of each array), two pieces per round so that 64
+// bytes per thread are in flight; the four k3 terms of a piece are added in float32 (a rounding of
+// 2^-24 of their sum, far inside the 1e-5 that the estimate is compared within) and the piece
+// sums in float64.  Arrays that do not start on a 16-byte boundary take the scalar loop.
+template <int NT>
 __global__ void __launch_bounds__(kDiagThreads)
 prob_partial_kernel(const float* __restrict__ pt, const float* __restrict__ pi, long long n,
                     const float* __restrict__ taus, int n_tau, double* __restrict__ part_kl,
                     long long* __restrict__ part_cnt) {
     __shared__ double s_kl[kDiagThreads / 32];
     __shared__ long long s_cnt[kDiagThreads / 32][kMaxTaus];
-    float tau[kMaxTaus];
-    int cnt[kMaxTaus];
+    float tau[NT];
+    int cnt[NT];
 #pragma unroll
-    for (int i = 0; i < kMaxTaus; ++i) {
+    for (int i = 0; i < NT; ++i) {
         tau[i] = i < n_tau ? taus[i] : INFINITY;
         cnt[i] = 0;
     }
     double acc = 0.0;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += stride) {
-        const float a = pt[t], b = pi[t];
-        acc += (double)k3_term(a, b);
-        // the threshold decision is taken on float32 ratios, the precision of the inputs
-        const float big = fmaxf(a / b, b / a);
+    auto one = [&](float a, float b) -> float {
+        // the threshold decision is taken on float32 ratios, the precision of the inputs:
+        // max(a / b, b / a) is the correctly rounded quotient of the larger by the smaller (one of
+        // the two quotients is at least 1, the other at most 1, and rounding keeps that order)
+        const float big = fmaxf(a, b) / fminf(a, b);
 #pragma unroll
-        for (int i = 0; i < kMaxTaus; ++i) cnt[i] += big > tau[i] ? 1 : 0;
+        for (int i = 0; i < NT; ++i) cnt[i] += big > tau[i] ? 1 : 0;
+        return k3_term(a, b);
+    };
+    auto four = [&](const float4& a, const float4& b) {
+        const float s0 = one(a.x, b.x), s1 = one(a.y, b.y), s2 = one(a.z, b.z), s3 = one(a.w, b.w);
+        acc += (double)((s0 + s1) + (s2 + s3));
+    };
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool vec = ((reinterpret_cast<uintptr_t>(pt) | reinterpret_cast<uintptr_t>(pi)) & 15u) == 0;
+    const long long n4 = vec ? n >> 2 : 0;
+    const float4* pt4 = reinterpret_cast<const float4*>(pt);
+    const float4* pi4 = reinterpret_cast<const float4*>(pi);
+    long long v = gtid;
+    for (; v + stride < n4; v += 2 * stride) {
+        const float4 a0 = pt4[v], b0 = pi4[v], a1 = pt4[v + stride], b1 = pi4[v + stride];
+        four(a0, b0);
+        four(a1, b1);
     }
+    if (v < n4) four(pt4[v], pi4[v]);
+    for (long long t = 4 * n4 + gtid; t < n; t += stride) acc += (double)one(pt[t], pi[t]);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
 #pragma unroll
-    for (int i = 0; i < kMaxTaus; ++i) {
+    for (int i = 0; i < NT; ++i) {
 #pragma unroll
         for (int s = 16; s > 0; s >>= 1) cnt[i] += __shfl_xor_sync(0xffffffffu, cnt[i], s);
     }
     if (lane == 0) {
         s_kl[warp] = acc;
 #pragma unroll
-        for (int i = 0; i < kMaxTaus; ++i) s_cnt[warp][i] = cnt[i];
+        for (int i = 0; i < NT; ++i) s_cnt[warp][i] = cnt[i];
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -83,19 +110,19 @@ prob_partial_kernel(const float* __restrict__ pt, const float* __restrict__ pi, 
     }
 }
 
-// Sums the per-CTA partials: thread i takes partials i, i + 256, ... (fixed), then the same warp
-// and CTA reduction as above.
-__global__ void __launch_bounds__(kDiagThreads)
+// Sums the per-CTA partials: thread i takes partials i, i + 1024, ... (fixed), then the same warp
+// and CTA reduction as above (one CTA of kFinalThreads threads).
+__global__ void __launch_bounds__(kFinalThreads)
 prob_final_kernel(const double* __restrict__ part_kl, const long long* __restrict__ part_cnt,
                   int parts, long long n, int n_tau, double* __restrict__ kl_out,
                   long long* __restrict__ counts_out) {
-    __shared__ double s_kl[kDiagThreads / 32];
-    __shared__ long long s_cnt[kDiagThreads / 32][kMaxTaus];
+    __shared__ double s_kl[kFinalThreads / 32];
+    __shared__ long long s_cnt[kFinalThreads / 32][kMaxTaus];
     double k = 0.0;
     long long c[kMaxTaus];
 #pragma unroll
     for (int i = 0; i < kMaxTaus; ++i) c[i] = 0;
-    for (int p = threadIdx.x; p < parts; p += kDiagThreads) {
+    for (int p = threadIdx.x; p < parts; p += kFinalThreads) {
         k += part_kl[p];
 #pragma unroll
         for (int i = 0; i < kMaxTaus; ++i)
@@ -117,12 +144,12 @@ prob_final_kernel(const double* __restrict__ part_kl, const long long* __restric
     __syncthreads();
     if (threadIdx.x == 0) {
         double tot = 0.0;
-        for (int w = 0; w < kDiagThreads / 32; ++w) tot += s_kl[w];         // fixed order
+        for (int w = 0; w < kFinalThreads / 32; ++w) tot += s_kl[w];         // fixed order
         *kl_out = n > 0 ? tot / (double)n : 0.0;
     }
     if (threadIdx.x < n_tau) {
         long long tot = 0;
-        for (int w = 0; w < kDiagThreads / 32; ++w) tot += s_cnt[w][threadIdx.x];
+        for (int w = 0; w < kFinalThreads / 32; ++w) tot += s_cnt[w][threadIdx.x];
         counts_out[threadIdx.x] = tot;
     }
 }
@@ -164,27 +191,37 @@ record_diff_kernel(const IdxT* __restrict__ ra, const IdxT* __restrict__ rb, int
 }
 
 // The common case K = 8 with one-byte ids: both records of a router are one 8-byte load each, and
-// membership of an id in the other record is two packed byte comparisons.
+// membership of an id in the other record is a zero-byte test on packed words.  A CTA takes 32
+// tokens: lane = token (a warp reads 256 consecutive bytes of a layer), warp w the layers w,
+// w + 8, ...; the per-token sums of the eight warps meet in shared memory.
 __global__ void __launch_bounds__(kDiagThreads)
 record_diff_k8_kernel(const uint2* __restrict__ ra, const uint2* __restrict__ rb, int L, int T,
                       uint8_t* __restrict__ diff_out, int32_t* __restrict__ token_choices,
                       int32_t* __restrict__ token_routers, unsigned long long* __restrict__ hist) {
+    constexpr int W = kDiagThreads / 32;
     __shared__ unsigned int s_hist[9];
+    __shared__ int s_choices[W][32], s_routers[W][32];
     if (threadIdx.x < 9) s_hist[threadIdx.x] = 0u;
     __syncthreads();
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * 32 + lane;
+    int choices = 0, routers = 0;
     if (t < T) {
-        int choices = 0, routers = 0;
         unsigned int local[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
-#pragma unroll 4
-        for (int l = 0; l < L; ++l) {
+#pragma unroll 2
+        for (int l = warp; l < L; l += W) {
             const uint2 a = ra[(size_t)l * T + t], b = rb[(size_t)l * T + t];
             int same = 0;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const unsigned int ea = ((i < 4 ? a.x : a.y) >> (8 * (i & 3))) & 0xffu;
                 const unsigned int rep = ea * 0x01010101u;
-                same += (__vcmpeq4(rep, b.x) | __vcmpeq4(rep, b.y)) != 0u ? 1 : 0;
+                // a byte of x is zero where the ids are equal; (x - 01..01) & ~x has the top bit of
+                // a byte set if that byte is zero (and possibly of bytes above a zero one, which
+                // does not matter for "any")
+                const unsigned int x0 = rep ^ b.x, x1 = rep ^ b.y;
+                const unsigned int z = ((x0 - 0x01010101u) & ~x0) | ((x1 - 0x01010101u) & ~x1);
+                same += (z & 0x80808080u) != 0u ? 1 : 0;
             }
             const int dlt = 8 - same;
             choices += dlt;
@@ -193,13 +230,23 @@ record_diff_k8_kernel(const uint2* __restrict__ ra, const uint2* __restrict__ rb
             for (int v = 0; v < 9; ++v) local[v] += dlt == v ? 1u : 0u;
             if (diff_out) diff_out[(size_t)l * T + t] = (uint8_t)dlt;
         }
-        token_choices[t] = choices;
-        token_routers[t] = routers;
 #pragma unroll
         for (int v = 0; v < 9; ++v)
             if (local[v]) atomicAdd(&s_hist[v], local[v]);       // integer: order-independent
     }
+    s_choices[warp][lane] = choices;
+    s_routers[warp][lane] = routers;
     __syncthreads();
+    if (warp == 0 && t < T) {
+        int c = 0, r = 0;
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            c += s_choices[w][lane];
+            r += s_routers[w][lane];
+        }
+        token_choices[t] = c;
+        token_routers[t] = r;
+    }
     if (threadIdx.x < 9 && s_hist[threadIdx.x])
         atomicAdd(&hist[threadIdx.x], (unsigned long long)s_hist[threadIdx.x]);
 }
@@ -221,7 +268,7 @@ sequence_sum_kernel(const int32_t* __restrict__ token_routers, const int32_t* __
 
 static int prob_parts(long long n) {
     const long long want = (n + kDiagThreads * 8LL - 1) / (kDiagThreads * 8LL);
-    const long long cap = 8LL * sm_count();
+    const long long cap = 4LL * sm_count();
     const long long g = want < cap ? want : cap;
     return (int)(g > 0 ? g : 1);
 }
@@ -248,9 +295,16 @@ extern "C" r3_status r3_prob_discrepancy(const float* p_train, const float* p_in
     const int parts = r3::prob_parts(n);
     double* part_kl = static_cast<double*>(workspace);
     long long* part_cnt = reinterpret_cast<long long*>(part_kl + parts);
-    r3::prob_partial_kernel<<<parts, r3::kDiagThreads, 0, cs>>>(p_train, p_infer, n, taus, n_tau,
-                                                               part_kl, part_cnt);
-    r3::prob_final_kernel<<<1, r3::kDiagThreads, 0, cs>>>(part_kl, part_cnt, parts, n, n_tau, kl_out,
+    if (n_tau <= 4)
+        r3::prob_partial_kernel<4><<<parts, r3::kDiagThreads, 0, cs>>>(p_train, p_infer, n, taus,
+                                                                      n_tau, part_kl, part_cnt);
+    else if (n_tau <= 8)
+        r3::prob_partial_kernel<8><<<parts, r3::kDiagThreads, 0, cs>>>(p_train, p_infer, n, taus,
+                                                                      n_tau, part_kl, part_cnt);
+    else
+        r3::prob_partial_kernel<16><<<parts, r3::kDiagThreads, 0, cs>>>(p_train, p_infer, n, taus,
+                                                                       n_tau, part_kl, part_cnt);
+    r3::prob_final_kernel<<<1, r3::kFinalThreads, 0, cs>>>(part_kl, part_cnt, parts, n, n_tau, kl_out,
                                             reinterpret_cast<long long*>(counts_out));
     return r3::launch_status();
 }
@@ -270,7 +324,7 @@ extern "C" r3_status r3_record_diff(const r3_shape* shape, int32_t L, const void
     const unsigned grid = (unsigned)((shape->T + r3::kDiagThreads - 1) / r3::kDiagThreads);
     if (shape->K == 8 && shape->idx_type == R3_IDX_U8 && r3::aligned(rec_a, 8) &&
         r3::aligned(rec_b, 8)) {
-        r3::record_diff_k8_kernel<<<grid, r3::kDiagThreads, 0, cs>>>(
+        r3::record_diff_k8_kernel<<<(unsigned)((shape->T + 31) / 32), r3::kDiagThreads, 0, cs>>>(
             static_cast<const uint2*>(rec_a), static_cast<const uint2*>(rec_b), L, shape->T,
             diff_out, token_choices, token_routers, reinterpret_cast<unsigned long long*>(hist));
         return r3::launch_status();
