@@ -249,3 +249,37 @@ def test_gate_bwd_refuses_a_misaligned_dlogits_instead_of_faulting(r3):
     ds = r3.replay_gate_bwd(s, g, dg, idx, dlogits=ok)
     ref = O.replay_gate_bwd(g.cpu().numpy(), dg.cpu().numpy(), idx.cpu().to(torch.int64).numpy(), E)
     assert rel_err(ds.cpu().numpy(), ref) < TOL_F32
+
+
+def test_inputs_written_by_the_kernel_just_before_the_call(r3):
+    """The dispatch, the row copy and the layer's first kernels are launched so that they may begin
+    before the kernel in front of them on the stream has ended, and the row copy fetches its token
+    rows before its own dependency wait.  Here the activations (and the record) are produced by
+    torch kernels enqueued directly in front of the call, without a synchronisation, forty times
+    with other data, into the SAME buffers: a fetch that did not wait for its producer would pick
+    up the rows of the round before."""
+    T, d, E, K, F = 4096, 512, 32, 4, 64
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="chain", T=T, d=d, E=E, K=K, F=F)
+    s = r3.shape_of(w)
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev).manual_seed(3)
+    base = torch.randn(T, d, generator=g, device=dev)
+    x = torch.empty(T, d, dtype=torch.bfloat16, device=dev)
+    idx = torch.empty(T, K, dtype=torch.uint8, device=dev)
+    keys = torch.rand(40, T, E, generator=g, device=dev)
+    ws = r3.workspace(r3.permute_workspace_bytes(s), dev)
+    st = r3.new_status(dev)
+    outs = []
+    for r in range(40):
+        # producers: one elementwise kernel for x, a top-k for the record, then the dispatch at once
+        x.copy_((base * (r + 1)).to(torch.bfloat16))
+        idx.copy_(keys[r].topk(K, dim=1).indices.to(torch.uint8))
+        counts, offsets, ros, sor, xp = r3.permute(s, idx, x, ws=ws, dev_status=st)
+        outs.append((idx.clone(), x.clone(), ros, xp))
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    for r, (idx_r, x_r, ros, xp) in enumerate(outs):
+        _, _, ros_ref, sor_ref = O.permutation(idx_r.cpu().numpy().astype(np.int64), E)
+        assert np.array_equal(ros.cpu().numpy(), ros_ref), r
+        want = x_r[torch.from_numpy(sor_ref.astype(np.int64)).to(dev) // K]
+        assert torch.equal(xp, want), r
