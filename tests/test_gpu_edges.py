@@ -283,3 +283,38 @@ def test_inputs_written_by_the_kernel_just_before_the_call(r3):
         assert np.array_equal(ros.cpu().numpy(), ros_ref), r
         want = x_r[torch.from_numpy(sor_ref.astype(np.int64)).to(dev) // K]
         assert torch.equal(xp, want), r
+
+
+def test_layer_fed_by_kernels_enqueued_directly_in_front_of_it(r3):
+    """The same for the whole layer (its first kernels on both streams start under the tail of
+    whatever precedes them): activations, upstream gradient and record rewritten by torch kernels
+    in front of every call, twelve rounds into the same buffers and the same workspace; every
+    round must give the bits of running its inputs alone after a synchronisation."""
+    w = synth.scaled(synth.WORKLOADS["c2_layer_bf16"], name="chain_layer", T=3000, d=512, E=32,
+                     K=4, F=128)
+    case = Case(w, device="cuda")
+    c = case.cuda()
+    s = r3.shape_of(w)
+    dev = torch.device("cuda", 0)
+    st = r3.new_status(dev)
+    ws = r3.workspace(r3.replay_layer_workspace_bytes(s), dev)
+    g = torch.Generator(device=dev).manual_seed(9)
+    keys = torch.rand(12, w.T, w.E, generator=g, device=dev)
+    x, dy, idx = c["x"].clone(), c["dy"].clone(), c["idx"].clone()
+    y = torch.empty_like(x)
+    ds = torch.empty((w.T, w.E), dtype=torch.float32, device=dev)
+    kept = []
+    for r in range(12):
+        x.copy_((c["x"].float() * (1.0 + 0.25 * r)).to(x.dtype))
+        dy.copy_((c["dy"].float() * (1.0 - 0.05 * r)).to(dy.dtype))
+        idx.copy_(keys[r].topk(w.K, dim=1).indices.to(idx.dtype))
+        r3.replay_layer(s, x, c["w_r"], idx, c["w_gate"], c["w_up"], c["w_down"], dy, y=y,
+                        dlogits=ds, ws=ws, dev_status=st)
+        kept.append((x.clone(), dy.clone(), idx.clone(), y.clone(), ds.clone()))
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    for r, (xr, dyr, idxr, yr, dsr) in enumerate(kept):
+        y1, ds1, _ = r3.replay_layer(s, xr, c["w_r"], idxr, c["w_gate"], c["w_up"], c["w_down"],
+                                     dyr, dev_status=st)
+        torch.cuda.synchronize()
+        assert torch.equal(y1, yr) and torch.equal(ds1, dsr), r
